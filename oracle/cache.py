@@ -1,0 +1,172 @@
+"""Oracle packed KV cache: append, dequantize, decode (test infrastructure).
+
+Mirrors the semantics of the library's three calls on NumPy arrays so that the
+tests can compare bytes and values one by one:
+
+* append: V is quantized token-wise at once.  K is quantized token-wise at once
+  (k_axis 0), or channel-wise per 128-token block (k_axis 1): tokens first go to
+  an fp16 residual tail (Sec. 4.1: recent tokens stay in full precision and are
+  flushed periodically); when the block is complete it is quantized with one
+  group per channel and written to its page.
+* dequantize: xhat = fmaf(code, scale, zero) rounded to the 16-bit input type.
+* decode: fp64 attention (App. A.1) over z + s*code exactly, the tail as stored.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from . import attention, layout, quantizer
+from .layout import PAGE_TOKENS, Layout
+
+ERR_CAPACITY_BIT = 1
+
+
+class OracleCache:
+    def __init__(self, batch, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, dtype, capacity_tokens):
+        assert capacity_tokens % PAGE_TOKENS == 0
+        assert not (k_axis == 1 and kb == 16)
+        self.B, self.H, self.D = batch, n_kv_heads, head_dim
+        self.dtype = dtype
+        self.capacity = capacity_tokens
+        self.L = Layout(head_dim, kb, vb, gk, gv, k_axis)
+        self.pages = np.zeros((batch, n_kv_heads, capacity_tokens // PAGE_TOKENS, self.L.page_bytes), np.uint8)
+        self.k_tail = np.zeros((batch, n_kv_heads, PAGE_TOKENS, head_dim), np.uint16) if k_axis == 1 else None
+        self.seq_len = np.zeros(batch, np.int32)
+        self.status = 0
+
+    # ------------------------------------------------------------------ append
+    def append(self, k_bits: np.ndarray, v_bits: np.ndarray):
+        """k_bits, v_bits: uint16 [B, Hkv, t_new, D] patterns of the input dtype."""
+        L = self.L
+        t_new = k_bits.shape[2]
+        for b in range(self.B):
+            t0 = int(self.seq_len[b])
+            if t0 + t_new > self.capacity:
+                self.status |= ERR_CAPACITY_BIT
+                continue
+            for h in range(self.H):
+                done = 0
+                while done < t_new:
+                    t = t0 + done
+                    p, slot = divmod(t, PAGE_TOKENS)
+                    n = min(PAGE_TOKENS - slot, t_new - done)
+                    slots = np.arange(slot, slot + n)
+                    page = self.pages[b, h, p]
+                    kx = k_bits[b, h, done:done + n]
+                    vx = v_bits[b, h, done:done + n]
+                    # values: always token-wise
+                    if L.vb == 16:
+                        layout.put_v_codes(page, L, slots, vx)
+                    else:
+                        c, s, z = quantizer.quantize_per_token(vx, self.dtype, L.vb, L.gv)
+                        layout.put_v_codes(page, L, slots, c)
+                        layout.put_v_meta_tokens(page, L, slots, s, z)
+                    # keys
+                    if L.k_axis == 0:
+                        if L.kb == 16:
+                            layout.put_k_codes(page, L, slots, kx)
+                        else:
+                            c, s, z = quantizer.quantize_per_token(kx, self.dtype, L.kb, L.gk)
+                            layout.put_k_codes(page, L, slots, c)
+                            layout.put_k_meta_tokens(page, L, slots, s, z)
+                    else:
+                        self.k_tail[b, h, slot:slot + n] = quantizer.to_tail_fp16_bits(kx, self.dtype)
+                        if slot + n == PAGE_TOKENS:      # block complete: flush the tail
+                            c, s, z = quantizer.quantize_per_channel_block(self.k_tail[b, h], L.kb)
+                            layout.put_k_codes(page, L, np.arange(PAGE_TOKENS), c)
+                            layout.put_k_meta_channels(page, L, s, z)
+                    done += n
+            self.seq_len[b] = t0 + t_new
+
+    # ------------------------------------------------------- page -> values
+    def _page_values(self, b, h, p, n_valid, exact: bool):
+        """Reconstruction of the first n_valid tokens of page p.
+        exact=True: fp64 z + s*c (for attention); False: fp32 fmaf (for dequantize).
+        Returns (K (n,D), V (n,D))."""
+        L, D = self.L, self.D
+        page = self.pages[b, h, p]
+        deq = quantizer.dequantize_groups_f64 if exact else quantizer.dequantize_groups
+        # V
+        if L.vb == 16:
+            V = quantizer.bits_to_f32(layout.get_v_codes(page, L), self.dtype)
+        else:
+            c = layout.get_v_codes(page, L).reshape(PAGE_TOKENS, D // L.gv, L.gv)
+            s, z = layout.get_v_meta(page, L)
+            V = deq(c, s, z).reshape(PAGE_TOKENS, D)
+        # K
+        tail_tokens = L.k_axis == 1 and n_valid < PAGE_TOKENS
+        if tail_tokens:
+            K = quantizer.bits_to_f32(self.k_tail[b, h], "fp16")
+        elif L.kb == 16:
+            K = quantizer.bits_to_f32(layout.get_k_codes(page, L), self.dtype)
+        elif L.k_axis == 0:
+            c = layout.get_k_codes(page, L).reshape(PAGE_TOKENS, D // L.gk, L.gk)
+            s, z = layout.get_k_meta(page, L)
+            K = deq(c, s, z).reshape(PAGE_TOKENS, D)
+        else:
+            c = layout.get_k_codes(page, L)            # (128, D), one group per channel
+            s, z = layout.get_k_meta(page, L)          # (D,)
+            K = deq(np.ascontiguousarray(c.T), s, z).T
+        if exact:
+            K = K.astype(np.float64)
+            V = V.astype(np.float64)
+        return K[:n_valid], V[:n_valid]
+
+    def values_f64(self):
+        """K-hat, V-hat as fp64 [B, Hkv, capacity, D]; zeros beyond seq_len."""
+        K = np.zeros((self.B, self.H, self.capacity, self.D), np.float64)
+        V = np.zeros_like(K)
+        for b in range(self.B):
+            n = int(self.seq_len[b])
+            for h in range(self.H):
+                for p in range((n + PAGE_TOKENS - 1) // PAGE_TOKENS):
+                    nv = min(PAGE_TOKENS, n - p * PAGE_TOKENS)
+                    k, v = self._page_values(b, h, p, nv, exact=True)
+                    K[b, h, p * PAGE_TOKENS: p * PAGE_TOKENS + nv] = k
+                    V[b, h, p * PAGE_TOKENS: p * PAGE_TOKENS + nv] = v
+        return K, V
+
+    # -------------------------------------------------------------- dequantize
+    def dequantize(self, k_out: np.ndarray, v_out: np.ndarray, t_begin: int, t_end: int):
+        """Writes 16-bit patterns of the input dtype into k_out, v_out
+        [B, Hkv, capacity, D] for tokens t_begin <= t < min(t_end, seq_len[b])."""
+        for b in range(self.B):
+            hi = min(t_end, int(self.seq_len[b]))
+            n = int(self.seq_len[b])
+            for h in range(self.H):
+                for p in range(t_begin // PAGE_TOKENS, (hi + PAGE_TOKENS - 1) // PAGE_TOKENS):
+                    nv = min(PAGE_TOKENS, n - p * PAGE_TOKENS)
+                    k, v = self._page_values(b, h, p, nv, exact=False)
+                    lo_t = max(t_begin, p * PAGE_TOKENS)
+                    hi_t = min(hi, p * PAGE_TOKENS + nv)
+                    sl = slice(lo_t - p * PAGE_TOKENS, hi_t - p * PAGE_TOKENS)
+                    k_out[b, h, lo_t:hi_t] = quantizer.f32_to_bits(k[sl], self.dtype)
+                    v_out[b, h, lo_t:hi_t] = quantizer.f32_to_bits(v[sl], self.dtype)
+
+    # ------------------------------------------------------------------ decode
+    def decode(self, q_bits: np.ndarray, scale=None) -> np.ndarray:
+        """q_bits uint16 [B, Hq, D] of the input dtype -> fp64 [B, Hq, D]."""
+        q = quantizer.bits_to_f32(q_bits, self.dtype).astype(np.float64)
+        K, V = self.values_f64()
+        return attention.decode_attention(q, K, V, self.seq_len, scale)
+
+    def decode_streams(self, q_bits: np.ndarray, streams, scale=None):
+        """Same as decode but only for the listed (b, kv_head) streams; returns
+        {(b, kv_head): fp64 (G, D)} (used to sample full-size workloads)."""
+        import math
+        q = quantizer.bits_to_f32(q_bits, self.dtype).astype(np.float64)
+        G = q.shape[1] // self.H
+        sc = scale if scale and scale > 0 else 1.0 / math.sqrt(self.D)
+        res = {}
+        for (b, h) in streams:
+            n = int(self.seq_len[b])
+            Ks, Vs = [], []
+            for p in range((n + PAGE_TOKENS - 1) // PAGE_TOKENS):
+                nv = min(PAGE_TOKENS, n - p * PAGE_TOKENS)
+                k, v = self._page_values(b, h, p, nv, exact=True)
+                Ks.append(k)
+                Vs.append(v)
+            K = np.concatenate(Ks) if Ks else np.zeros((0, self.D))
+            V = np.concatenate(Vs) if Vs else np.zeros((0, self.D))
+            res[(b, h)] = np.stack([attention.attend_one(q[b, h * G + j], K, V, sc) for j in range(G)])
+        return res

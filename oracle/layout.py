@@ -1,0 +1,193 @@
+"""Oracle packer / unpacker for the packed KV page (test infrastructure).
+
+Written from the layout's published index function, independently of the CUDA
+code.  The paper describes no packed layout; this one is the library's own
+(layout version 1):
+
+A page holds 128 consecutive tokens of one (batch, kv-head) stream as four
+regions, in this order, each a multiple of 16 bytes:
+
+    [K codes | K meta | V codes | V meta]
+
+All multi-byte quantities are little-endian.  A b-bit code field number f of a
+32-bit word occupies bits [f*b, f*b+b).  With ppw = 16/b ("pairs per word"):
+
+K codes (b = kb in {2,4,8}): token-major rows of D*b/8 bytes; a row is 4 chunks
+of D*b/32 bytes.  Channel d of a token lives in
+    chunk  = (d % 8) // 2
+    P      = 2*(d // 16) + (d % 16) // 8          pair index inside the chunk
+    word   = P // ppw,  field = P % ppw + ppw*(d % 2)
+V codes (b = vb in {2,4,8}): 8 tiles of 16 tokens, a tile is 32 chunks of
+D*b/16 bytes.  Channel d of token tau (0..15 inside its tile) lives in
+    chunk  = 4*(d % 8) + (tau % 8) // 2
+    P      = 4*(d // 16) + (d % 16) // 8 + 2*(tau // 8)
+    word   = P // ppw,  field = P % ppw + ppw*(tau % 2)
+b = 16 (either side): plain rows [token][D] of the input's 16-bit patterns.
+
+Meta: (scale fp16, zero fp16) pairs, 4 bytes each.  Per-token axis:
+[128 tokens][D/g groups]; per-channel K: [D channels] (one group per channel
+over the page's 128 tokens).  A 16-bit side has no meta.
+"""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+
+PAGE_TOKENS = 128
+
+
+@dataclasses.dataclass(frozen=True)
+class Layout:
+    D: int
+    kb: int
+    vb: int
+    gk: int
+    gv: int
+    k_axis: int = 0
+
+    @property
+    def k_codes_bytes(self):
+        return PAGE_TOKENS * self.D * self.kb // 8
+
+    @property
+    def k_meta_bytes(self):
+        if self.kb == 16:
+            return 0
+        return 4 * self.D if self.k_axis == 1 else PAGE_TOKENS * (self.D // self.gk) * 4
+
+    @property
+    def v_codes_bytes(self):
+        return PAGE_TOKENS * self.D * self.vb // 8
+
+    @property
+    def v_meta_bytes(self):
+        return 0 if self.vb == 16 else PAGE_TOKENS * (self.D // self.gv) * 4
+
+    @property
+    def k_meta_off(self):
+        return self.k_codes_bytes
+
+    @property
+    def v_codes_off(self):
+        return self.k_meta_off + self.k_meta_bytes
+
+    @property
+    def v_meta_off(self):
+        return self.v_codes_off + self.v_codes_bytes
+
+    @property
+    def page_bytes(self):
+        return self.v_meta_off + self.v_meta_bytes
+
+
+# ----------------------------------------------------------------------------
+# index functions: (token in page, channel) -> (byte offset in region, bit shift)
+# ----------------------------------------------------------------------------
+def k_code_pos(t, d, D, b):
+    t = np.asarray(t)
+    d = np.asarray(d)
+    ppw = 16 // b
+    chunk = (d % 8) // 2
+    P = 2 * (d // 16) + (d % 16) // 8
+    word = P // ppw
+    field = P % ppw + ppw * (d % 2)
+    bit = field * b
+    byte = t * (D * b // 8) + chunk * (D * b // 32) + 4 * word + bit // 8
+    return byte, bit % 8
+
+
+def v_code_pos(t, d, D, b):
+    t = np.asarray(t)
+    d = np.asarray(d)
+    ppw = 16 // b
+    tile = t // 16
+    tau = t % 16
+    chunk = 4 * (d % 8) + (tau % 8) // 2
+    P = 4 * (d // 16) + (d % 16) // 8 + 2 * (tau // 8)
+    word = P // ppw
+    field = P % ppw + ppw * (tau % 2)
+    bit = field * b
+    byte = tile * (16 * D * b // 8) + chunk * (D * b // 16) + 4 * word + bit // 8
+    return byte, bit % 8
+
+
+def _put_codes(region: np.ndarray, pos_fn, tokens: np.ndarray, codes: np.ndarray, D, b):
+    """OR b-bit codes (n, D) of the given page-local tokens into a code region."""
+    tt, dd = np.meshgrid(tokens, np.arange(D), indexing="ij")
+    if b == 16:
+        u = codes.astype(np.uint16)
+        region[tt * 2 * D + 2 * dd] = (u & 0xFF).astype(np.uint8)
+        region[tt * 2 * D + 2 * dd + 1] = (u >> 8).astype(np.uint8)
+        return
+    byte, shift = pos_fn(tt, dd, D, b)
+    mask = (1 << b) - 1
+    # clear, then set (fields never straddle bytes because b divides 8)
+    np.bitwise_and.at(region, byte.ravel(), (~(mask << shift.ravel()) & 0xFF).astype(np.uint8))
+    np.bitwise_or.at(region, byte.ravel(), ((codes.astype(np.uint32).ravel() & mask) << shift.ravel()).astype(np.uint8))
+
+
+def _get_codes(region: np.ndarray, pos_fn, D, b) -> np.ndarray:
+    tt, dd = np.meshgrid(np.arange(PAGE_TOKENS), np.arange(D), indexing="ij")
+    if b == 16:
+        lo = region[tt * 2 * D + 2 * dd].astype(np.uint16)
+        hi = region[tt * 2 * D + 2 * dd + 1].astype(np.uint16)
+        return lo | (hi << 8)
+    byte, shift = pos_fn(tt, dd, D, b)
+    return ((region[byte] >> shift.astype(np.uint8)) & ((1 << b) - 1)).astype(np.uint8)
+
+
+def put_k_codes(page: np.ndarray, L: Layout, tokens, codes):
+    _put_codes(page[: L.k_codes_bytes], k_code_pos, np.asarray(tokens), codes, L.D, L.kb)
+
+
+def put_v_codes(page: np.ndarray, L: Layout, tokens, codes):
+    _put_codes(page[L.v_codes_off: L.v_codes_off + L.v_codes_bytes], v_code_pos,
+               np.asarray(tokens), codes, L.D, L.vb)
+
+
+def get_k_codes(page: np.ndarray, L: Layout) -> np.ndarray:
+    return _get_codes(page[: L.k_codes_bytes], k_code_pos, L.D, L.kb)
+
+
+def get_v_codes(page: np.ndarray, L: Layout) -> np.ndarray:
+    return _get_codes(page[L.v_codes_off: L.v_codes_off + L.v_codes_bytes], v_code_pos, L.D, L.vb)
+
+
+def _meta_view(page: np.ndarray, off: int, nbytes: int) -> np.ndarray:
+    """uint16 view [n][2] = (scale bits, zero bits) of a meta region."""
+    return page[off: off + nbytes].view(np.uint16).reshape(-1, 2)
+
+
+def put_k_meta_tokens(page, L: Layout, tokens, s16, z16):
+    """per-token axis: s16, z16 (n, D/gk)."""
+    m = _meta_view(page, L.k_meta_off, L.k_meta_bytes).reshape(PAGE_TOKENS, L.D // L.gk, 2)
+    m[np.asarray(tokens), :, 0] = s16
+    m[np.asarray(tokens), :, 1] = z16
+
+
+def put_k_meta_channels(page, L: Layout, s16, z16):
+    """per-channel axis: s16, z16 (D,)."""
+    m = _meta_view(page, L.k_meta_off, L.k_meta_bytes)
+    m[:, 0] = s16
+    m[:, 1] = z16
+
+
+def put_v_meta_tokens(page, L: Layout, tokens, s16, z16):
+    m = _meta_view(page, L.v_meta_off, L.v_meta_bytes).reshape(PAGE_TOKENS, L.D // L.gv, 2)
+    m[np.asarray(tokens), :, 0] = s16
+    m[np.asarray(tokens), :, 1] = z16
+
+
+def get_k_meta(page, L: Layout):
+    """(s16, z16): (128, D/gk) for the per-token axis, (D,) for per-channel."""
+    m = _meta_view(page, L.k_meta_off, L.k_meta_bytes)
+    if L.k_axis == 1:
+        return m[:, 0].copy(), m[:, 1].copy()
+    m = m.reshape(PAGE_TOKENS, L.D // L.gk, 2)
+    return m[..., 0].copy(), m[..., 1].copy()
+
+
+def get_v_meta(page, L: Layout):
+    m = _meta_view(page, L.v_meta_off, L.v_meta_bytes).reshape(PAGE_TOKENS, L.D // L.gv, 2)
+    return m[..., 0].copy(), m[..., 1].copy()
