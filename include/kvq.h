@@ -1,0 +1,162 @@
+/*
+ * kvq - mixed-precision KV-cache quantization hot path for NVIDIA B200 (sm_100a).
+ *
+ * C-ABI of libkvq.so.  Plain C: POD structs, raw pointers, sizes.  No C++ or
+ * torch types cross this boundary.  All `void*` / `int32_t*` data pointers in
+ * kvq_cache and in the call arguments are DEVICE pointers owned by the caller;
+ * kvq_config and kvq_cache structs themselves are HOST memory, read during the
+ * call and never retained.  `cuda_stream` is a cudaStream_t passed as void*
+ * (NULL = the legacy default stream).
+ *
+ * What is computed (arxiv 2502.15075, "Quantize What Counts: More for Keys,
+ * Less for Values"): keys and values of the cache (K = X W^K, V = X W^V, one
+ * L x d_head matrix per head, Sec. 3 / App. B.3) are stored with a uniform scalar
+ * quantizer (App. B.1: scale = range / steps, Q = round(A / scale), A^ = scale Q)
+ * at independent bit widths b_K, b_V (Theorem 2: more bits for keys), in groups
+ * of 32/64/128 elements, token-wise or channel-wise, with recent tokens of an
+ * incomplete channel-wise block kept in 16-bit precision (Sec. 4.1).  A decode
+ * step computes softmax(q K^T / sqrt(d)) V (App. A.1 notation) over the
+ * reconstructed cache.
+ *
+ * Quantizer (fixed formula; every operation an individually rounded IEEE fp32
+ * operation, ties to even):
+ *     mn, mx  = min, max of the group, each + 0.0f   (-0 becomes +0)
+ *     s16     = fp16_rn((mx - mn) / qmax), z16 = fp16_rn(mn), saturating at +-65504
+ *     s, z    = (float)s16, (float)z16,  qmax = 2^b - 1
+ *     code    = 0 if s == 0, else clamp(rintf((x - z) * (1.0f / s)), 0, qmax)
+ *     x^      = fmaf(code, s, z)
+ * Inputs must be finite.
+ *
+ * Packed page (layout version 1): 128 consecutive tokens of one
+ * (batch, kv-head) stream, regions [K codes | K meta | V codes | V meta], each
+ * a multiple of 16 bytes, little-endian.  Field f of a 32-bit word holds bits
+ * [f*b, f*b+b); ppw = 16/b.
+ *   K codes, b in {2,4,8}: rows of D*b/8 bytes per token, each 4 chunks of
+ *     D*b/32 bytes; channel d: chunk (d%8)/2, P = 2*(d/16) + (d%16)/8,
+ *     word P/ppw, field P%ppw + ppw*(d%2).
+ *   V codes, b in {2,4,8}: 8 tiles of 16 tokens, each 32 chunks of D*b/16
+ *     bytes; channel d of tile-local token tau: chunk 4*(d%8) + (tau%8)/2,
+ *     P = 4*(d/16) + (d%16)/8 + 2*(tau/8), word P/ppw, field P%ppw + ppw*(tau%2).
+ *   b = 16: rows [token][D] of the input's 16-bit patterns, no meta.
+ *   Meta: (scale fp16, zero fp16) per group; per-token axis [128][D/g],
+ *     per-channel K [D].
+ * pages: [batch][n_kv_heads][capacity_tokens/128][page_bytes].
+ * k_tail (k_axis == 1 only): fp16 [batch][n_kv_heads][128][head_dim]; holds
+ *   fp16(x) of the keys of the incomplete last block; the block is quantized
+ *   (one group per channel over its 128 tokens) when it fills up.
+ */
+#ifndef KVQ_H_
+#define KVQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KVQ_LAYOUT_VERSION 1
+#define KVQ_PAGE_TOKENS 128
+
+/* return codes (0 = success) */
+#define KVQ_OK 0
+#define KVQ_ERR_INVALID_ARG (-1)
+#define KVQ_ERR_UNSUPPORTED (-2)
+#define KVQ_ERR_MISALIGNED (-3)
+#define KVQ_ERR_WORKSPACE_TOO_SMALL (-4)
+#define KVQ_ERR_CAPACITY (-5)
+#define KVQ_ERR_CUDA_LAUNCH (-6)
+#define KVQ_ERR_DEVICE_TIMEOUT (-7)
+
+/* bits that kernels OR into *kvq_cache.status (never trap) */
+#define KVQ_STATUS_CAPACITY 1u       /* an append would exceed capacity_tokens; that sequence was skipped */
+#define KVQ_STATUS_DEVICE_TIMEOUT 2u /* a bounded device-side wait expired */
+
+/* dtypes */
+#define KVQ_FP16 0
+#define KVQ_BF16 1
+#define KVQ_FP32 2 /* decode output only */
+
+typedef struct {
+  int32_t batch;
+  int32_t n_q_heads;       /* multiple of n_kv_heads; query head h reads KV head h / (n_q_heads/n_kv_heads);
+                              group size n_q_heads/n_kv_heads <= 8 */
+  int32_t n_kv_heads;
+  int32_t head_dim;        /* 64 or 128 */
+  int32_t kb, vb;          /* 2, 4, 8 quantized; 16 = unquantized passthrough */
+  int32_t gk, gv;          /* group size along head_dim: 32, 64 or 128, dividing head_dim (per-token axis) */
+  int32_t k_axis;          /* 0: keys token-wise; 1: keys channel-wise over 128-token blocks (needs kb != 16) */
+  int32_t in_dtype;        /* KVQ_FP16 or KVQ_BF16: type of k_new, v_new, q and of dequantize's outputs */
+  int32_t capacity_tokens; /* per sequence; multiple of 128 */
+} kvq_config;
+
+typedef struct {
+  void* pages;      /* device; 16-byte aligned; see layout above */
+  void* k_tail;     /* device fp16 tail, 16-byte aligned; NULL when k_axis == 0 */
+  int32_t* seq_len; /* device [batch]: tokens stored per sequence (quantized + tail) */
+  int32_t* status;  /* device, one word of KVQ_STATUS_* bits */
+} kvq_cache;        /* one per layer.  The caller zeroes seq_len and status for a fresh cache;
+                       pages must be zero-filled once before the first append. */
+
+/* Layout queries (host only, no GPU work).  All return KVQ_OK or KVQ_ERR_INVALID_ARG /
+ * KVQ_ERR_UNSUPPORTED for a config outside the documented ranges. */
+int kvq_layout_version(void);
+int kvq_page_bytes(const kvq_config* cfg, size_t* out);
+int kvq_cache_bytes(const kvq_config* cfg, size_t* pages_bytes, size_t* k_tail_bytes);
+/* Scratch needed by kvq_decode_attention for its split partial results. */
+int kvq_workspace_bytes(const kvq_config* cfg, size_t* out);
+
+/*
+ * Quantize and pack t_new new tokens per sequence and append them at position
+ * seq_len[b] (App. B.1 quantizer per group; Sec. 4.1 grouping and residual tail).
+ *   k_new, v_new: device, in_dtype, logical shape [batch][n_kv_heads][t_new][head_dim];
+ *     element (b,h,t,d) at offset b*stride_b + h*stride_h + t*stride_t + d (in elements);
+ *     head_dim contiguous, base pointers and strides such that every row is 16-byte aligned.
+ * Asynchronous on cuda_stream.  seq_len[b] += t_new for every sequence that fits; a sequence
+ * with seq_len[b] + t_new > capacity_tokens is left untouched and KVQ_STATUS_CAPACITY is set.
+ * Returns KVQ_OK or a host-detected argument / launch error (then nothing was launched).
+ * Not safe to call concurrently on the same cache.
+ */
+int kvq_quantize_append(const kvq_config* cfg, const kvq_cache* cache,
+                        const void* k_new, const void* v_new,
+                        int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                        int32_t t_new, void* cuda_stream);
+
+/*
+ * One decode step: out[b,h,:] = softmax_t(scale * q[b,h,:] . K^[b,h/G,t,:]) V^[b,h/G,t,:]
+ * over t < seq_len[b] (App. A.1: S = Q K^T / sqrt(d), A = softmax(S), A V), streaming the
+ * packed pages and reconstructing K^, V^ on the fly; tokens of an incomplete channel-wise
+ * key block are read from the fp16 tail.  Split over the sequence, partial results merged by
+ * log-sum-exp in a second pass.  seq_len[b] == 0 gives zeros.
+ *   q: device, in_dtype, [batch][n_q_heads][head_dim] contiguous.
+ *   out: device, [batch][n_q_heads][head_dim] contiguous, out_dtype (KVQ_FP16/BF16/FP32).
+ *   softmax_scale <= 0 selects 1/sqrt(head_dim).
+ *   workspace: device scratch of at least kvq_workspace_bytes(), 16-byte aligned; contents
+ *     need no initialisation and are undefined afterwards.
+ * Asynchronous on cuda_stream; reads the cache only.
+ */
+int kvq_decode_attention(const kvq_config* cfg, const kvq_cache* cache,
+                         const void* q, void* out, int32_t out_dtype, float softmax_scale,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Reconstruct tokens t_begin <= t < min(t_end, seq_len[b]) as x^ = fmaf(code, s, z) rounded to
+ * in_dtype (App. B.1: A^ = scale * Q); tail keys are converted from fp16.
+ *   k_out, v_out: device, in_dtype, [batch][n_kv_heads][capacity_tokens][head_dim] contiguous;
+ *     either may be NULL to skip it.  Elements outside the token range are not written.
+ * Asynchronous on cuda_stream; reads the cache only.
+ */
+int kvq_dequantize(const kvq_config* cfg, const kvq_cache* cache,
+                   void* k_out, void* v_out, int32_t t_begin, int32_t t_end, void* cuda_stream);
+
+/* Synchronises cuda_stream, reads *cache->status and returns KVQ_OK, KVQ_ERR_CAPACITY,
+ * KVQ_ERR_DEVICE_TIMEOUT or KVQ_ERR_CUDA_LAUNCH (a CUDA error surfaced by the sync). */
+int kvq_check_status(const kvq_cache* cache, void* cuda_stream);
+
+/* Static description of a return code. */
+const char* kvq_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVQ_H_ */

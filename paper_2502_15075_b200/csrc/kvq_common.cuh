@@ -1,0 +1,118 @@
+// Shared device/host definitions of libkvq: page geometry, the layout's index
+// functions and the fixed-formula group quantizer (App. B.1 uniform scalar
+// quantizer applied per group with a minimum offset).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvq.h"
+
+namespace kvq {
+
+constexpr int kPageTokens = KVQ_PAGE_TOKENS;
+constexpr int kMaxGroupHeads = 8;  // query heads per KV head
+
+// Everything a kernel needs to know about a cache, derived from kvq_config.
+struct Geom {
+  int B, Hq, Hkv, G, D;
+  int kb, vb, gk, gv, k_axis, in_dtype;
+  int capacity, n_pages;
+  int k_codes_bytes, k_meta_off, k_meta_bytes;
+  int v_codes_off, v_codes_bytes, v_meta_off, v_meta_bytes;
+  int page_bytes;
+};
+
+// Pointers of one cache (device memory).
+struct CachePtrs {
+  uint8_t* pages;
+  uint16_t* k_tail;
+  int32_t* seq_len;
+  uint32_t* status;
+};
+
+// ---------------------------------------------------------------- conversions
+__device__ __forceinline__ float bits16_to_f32(uint16_t u, int dtype) {
+  if (dtype == KVQ_FP16) return __half2float(__ushort_as_half(u));
+  return __uint_as_float(((uint32_t)u) << 16);
+}
+
+__device__ __forceinline__ uint16_t f32_to_fp16_sat_bits(float x) {
+  x = fminf(fmaxf(x, -65504.0f), 65504.0f);
+  return __half_as_ushort(__float2half_rn(x));
+}
+
+__device__ __forceinline__ uint16_t f32_to_bits16(float x, int dtype) {
+  if (dtype == KVQ_FP16) return __half_as_ushort(__float2half_rn(x));
+  return __bfloat16_as_ushort(__float2bfloat16_rn(x));
+}
+
+// ---------------------------------------------------------------- quantizer
+struct GroupParams {
+  float s, z, inv;     // fp32 values of the stored fp16 scale / zero, and 1/s (0 when s == 0)
+  uint32_t meta;       // s16 | z16 << 16
+};
+
+__device__ __forceinline__ GroupParams group_params(float mn, float mx, float qmax) {
+  mn = __fadd_rn(mn, 0.0f);
+  mx = __fadd_rn(mx, 0.0f);
+  float scale32 = __fdiv_rn(__fsub_rn(mx, mn), qmax);
+  uint16_t s16 = f32_to_fp16_sat_bits(scale32);
+  uint16_t z16 = f32_to_fp16_sat_bits(mn);
+  GroupParams p;
+  p.s = __half2float(__ushort_as_half(s16));
+  p.z = __half2float(__ushort_as_half(z16));
+  p.inv = (p.s != 0.0f) ? __fdiv_rn(1.0f, p.s) : 0.0f;
+  p.meta = (uint32_t)s16 | ((uint32_t)z16 << 16);
+  return p;
+}
+
+__device__ __forceinline__ uint32_t code_of(float x, const GroupParams& p, float qmax) {
+  float u = __fmul_rn(__fsub_rn(x, p.z), p.inv);
+  float r = rintf(u);
+  r = fminf(fmaxf(r, 0.0f), qmax);
+  return (uint32_t)r;
+}
+
+// ---------------------------------------------------------------- layout index functions
+// Byte offset (inside the K-code region of a page) of the 32-bit word holding
+// channel d of page-local token t, and the field's bit offset inside that word.
+__host__ __device__ __forceinline__ void k_code_pos(int t, int d, int D, int b, int& word_byte, int& bit) {
+  int ppw = 16 / b;
+  int chunk = (d & 7) >> 1;
+  int P = 2 * (d >> 4) + ((d & 15) >> 3);
+  word_byte = t * (D * b / 8) + chunk * (D * b / 32) + 4 * (P / ppw);
+  bit = (P % ppw + ppw * (d & 1)) * b;
+}
+
+__host__ __device__ __forceinline__ void v_code_pos(int t, int d, int D, int b, int& word_byte, int& bit) {
+  int ppw = 16 / b;
+  int tile = t >> 4, tau = t & 15;
+  int chunk = 4 * (d & 7) + ((tau & 7) >> 1);
+  int P = 4 * (d >> 4) + ((d & 15) >> 3) + 2 * (tau >> 3);
+  word_byte = tile * (16 * D * b / 8) + chunk * (D * b / 16) + 4 * (P / ppw);
+  bit = (P % ppw + ppw * (tau & 1)) * b;
+}
+
+// Inverse maps: which channel (and tile-local token) sits in field f of a word.
+__device__ __forceinline__ int k_field_channel(int chunk, int word, int f, int b) {
+  int ppw = 16 / b;
+  int P = word * ppw + (f % ppw);
+  return 16 * (P >> 1) + 8 * (P & 1) + 2 * chunk + (f / ppw);
+}
+
+__device__ __forceinline__ void v_field_pos(int chunk, int word, int f, int b, int& tau, int& d) {
+  int ppw = 16 / b;
+  int P = word * ppw + (f % ppw);
+  d = 16 * (P >> 2) + 8 * (P & 1) + (chunk >> 2);
+  tau = 8 * ((P & 3) >> 1) + 2 * (chunk & 3) + (f / ppw);
+}
+
+__device__ __forceinline__ uint32_t load_code(const uint8_t* region, int word_byte, int bit, int b) {
+  uint32_t w = *reinterpret_cast<const uint32_t*>(region + word_byte);
+  return (w >> bit) & ((1u << b) - 1u);
+}
+
+}  // namespace kvq

@@ -1,0 +1,27 @@
+// Internal launch interface between the C-ABI layer (kvq_host.cu) and the kernels.
+#pragma once
+
+#include "kvq_common.cuh"
+
+namespace kvq {
+
+int launch_quantize_append(const Geom& g, const CachePtrs& c, const void* k_new, const void* v_new,
+                           int64_t sb, int64_t sh, int64_t st, int t_new, cudaStream_t stream);
+
+int launch_dequantize(const Geom& g, const CachePtrs& c, void* k_out, void* v_out, int t_begin, int t_end,
+                      cudaStream_t stream);
+
+// Number of sequence splits the decode kernels use for this geometry (also sizes the workspace).
+int decode_num_splits(const Geom& g);
+size_t decode_workspace_bytes(const Geom& g);
+int launch_decode_attention(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
+                            float softmax_scale, void* workspace, cudaStream_t stream);
+
+}  // namespace kvq
+
+namespace kvq {
+// kernels behind launch_decode_attention
+int launch_decode_generic(const Geom& g, const CachePtrs& c, const void* q, float scale_log2e, float* ws,
+                          int n_split, cudaStream_t stream);
+int launch_merge(const Geom& g, const float* ws, void* out, int out_dtype, int n_split, cudaStream_t stream);
+}  // namespace kvq
