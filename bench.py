@@ -333,7 +333,9 @@ def oracle_leg(kvq, w, cfg, cache, q, out_gpu):
     pages = cache.pages_view()
     qb = q.cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
     seq = cache.seq_len.cpu().numpy()
-    streams = [(0, 0), (B - 1, H - 1), (B // 2, H // 2), (B // 3, 1 % H)]
+    n_streams = B * H
+    order = [(i * 37) % n_streams for i in range(min(n_streams, 48))]      # a fixed spread over the streams
+    streams = [(s // H, s % H) for s in dict.fromkeys(order)]
     got_all = out_gpu.double().cpu().numpy()
     t_used, n_done, errs = 0.0, 0, []
     with threadpool_limits(limits=1):
@@ -349,7 +351,7 @@ def oracle_leg(kvq, w, cfg, cache, q, out_gpu):
             n_done += 1
             got = got_all[b:b + 1, h * G:(h + 1) * G]
             errs.append((float(np.linalg.norm(got - want) / np.linalg.norm(want)), float(np.abs(got - want).max())))
-            if t_used > 20.0:
+            if t_used > 12.0:
                 break
     sample_bytes = n_done * w.context * wl.packed_bytes_per_token(w)
     return {"baseline": {"value": sample_bytes / t_used / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
