@@ -67,6 +67,7 @@ extern "C" {
 #define KVQ_ERR_CAPACITY (-5)
 #define KVQ_ERR_CUDA_LAUNCH (-6)
 #define KVQ_ERR_DEVICE_TIMEOUT (-7)
+#define KVQ_ERR_STATIC_SCRATCH (-8) /* problem needs more scratch than the library's built-in buffer */
 
 /* bits that kernels OR into *kvq_cache.status (never trap) */
 #define KVQ_STATUS_CAPACITY 1u       /* an append would exceed capacity_tokens; that sequence was skipped */
@@ -148,6 +149,36 @@ int kvq_decode_attention(const kvq_config* cfg, const kvq_cache* cache,
  */
 int kvq_dequantize(const kvq_config* cfg, const kvq_cache* cache,
                    void* k_out, void* v_out, int32_t t_begin, int32_t t_end, void* cuda_stream);
+
+/*
+ * kvq_decode_attention for callers that cannot provide scratch memory.  (The paper has no
+ * counterpart to this call; it exists for integration reasons only.)
+ *
+ * Some users of this library are not allowed to allocate device memory around a decode step:
+ * a serving engine that hands all free HBM to its own arena at start-up and treats any allocator
+ * call inside the token loop as a bug (cudaMalloc synchronises the whole device and fails once
+ * memory is fully reserved), or a plug-in that is given only input and output pointers by its
+ * host framework and has no allocator to ask.  For them this entry point takes the same inputs and
+ * outputs as kvq_decode_attention but no workspace: the split partial results go to a buffer of
+ * KVQ_STATIC_SCRATCH_BYTES that is part of the library image itself.  The call performs no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * Consequences the caller has to know:
+ *  - every GPU that loads libkvq.so holds those KVQ_STATIC_SCRATCH_BYTES until the process exits;
+ *  - a configuration whose kvq_workspace_bytes() exceeds KVQ_STATIC_SCRATCH_BYTES is rejected with
+ *    KVQ_ERR_STATIC_SCRATCH before anything is launched (use kvq_decode_attention then);
+ *  - the first call on each device looks up the buffer's device address (a host-side query, made
+ *    with that device current); make that first call before starting any stream capture;
+ *  - all calls on a device share the one buffer, and it keeps whatever the previous call left in it.
+ *    Nothing in it has to start at zero (each slot is written before it is read within a call), so
+ *    back-to-back calls on one stream are fine, but two calls that may overlap on the GPU (different
+ *    streams without an ordering between them) race on it and give wrong results.
+ * Results are identical to kvq_decode_attention's.
+ */
+#define KVQ_STATIC_SCRATCH_BYTES (8u << 20)
+int kvq_decode_attention_static(const kvq_config* cfg, const kvq_cache* cache,
+                                const void* q, void* out, int32_t out_dtype, float softmax_scale,
+                                void* cuda_stream);
 
 /* Synchronises cuda_stream, reads *cache->status and returns KVQ_OK, KVQ_ERR_CAPACITY,
  * KVQ_ERR_DEVICE_TIMEOUT or KVQ_ERR_CUDA_LAUNCH (a CUDA error surfaced by the sync). */

@@ -155,6 +155,55 @@ int kvq_decode_attention(const kvq_config* cfg, const kvq_cache* cache, const vo
                                  static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---------------------------------------------------------------------------
+// Decode without caller scratch: the split partials live in a buffer that is
+// part of the library image (one copy per GPU that loads the library).
+//
+// `g_static_scratch` names a device variable.  In host code that name is only a
+// handle for the runtime, not a device address, so it must never be passed to a
+// kernel; the device address is looked up once per device below and that
+// pointer is what the kernels receive.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[KVQ_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};   // device address per device ordinal, 0 = not looked up yet
+
+// Device address of the built-in scratch on the current device.  The first call on a device
+// performs the lookup (cudaGetSymbolAddress with that device current); later calls are a table read.
+int static_scratch_ptr(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return KVQ_ERR_CUDA_LAUNCH;
+  void* p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return KVQ_ERR_CUDA_LAUNCH;
+    __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);   // idempotent: same value from any thread
+  }
+  *out = p;
+  return KVQ_OK;
+}
+}  // namespace
+
+int kvq_decode_attention_static(const kvq_config* cfg, const kvq_cache* cache, const void* q, void* out,
+                                int32_t out_dtype, float softmax_scale, void* cuda_stream) {
+  Geom g;
+  CachePtrs c;
+  int rc = make_geom(cfg, &g);
+  if (rc != KVQ_OK) return rc;
+  rc = make_cache(g, cache, &c);
+  if (rc != KVQ_OK) return rc;
+  if (!q || !out) return KVQ_ERR_INVALID_ARG;
+  if (out_dtype != KVQ_FP16 && out_dtype != KVQ_BF16 && out_dtype != KVQ_FP32) return KVQ_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return KVQ_ERR_MISALIGNED;
+  if (decode_workspace_bytes(g) > (size_t)KVQ_STATIC_SCRATCH_BYTES) return KVQ_ERR_STATIC_SCRATCH;
+  void* scratch = nullptr;
+  rc = static_scratch_ptr(&scratch);
+  if (rc != KVQ_OK) return rc;
+  return launch_decode_attention(g, c, q, out, out_dtype, softmax_scale, scratch,
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
 int kvq_dequantize(const kvq_config* cfg, const kvq_cache* cache, void* k_out, void* v_out, int32_t t_begin,
                    int32_t t_end, void* cuda_stream) {
   Geom g;
@@ -191,6 +240,9 @@ const char* kvq_strerror(int code) {
     case KVQ_ERR_CAPACITY: return "append exceeds the cache capacity";
     case KVQ_ERR_CUDA_LAUNCH: return "CUDA launch or runtime error";
     case KVQ_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired";
+    case KVQ_ERR_STATIC_SCRATCH:
+      return "this configuration needs more split scratch than the library's built-in 8 MiB buffer; "
+             "use kvq_decode_attention with a caller-provided workspace";
     default: return "unknown kvq error";
   }
 }

@@ -47,17 +47,21 @@ _lib.kvq_quantize_append.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_voi
 _lib.kvq_decode_attention.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
                                       ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
                                       ctypes.c_void_p]
+_lib.kvq_decode_attention_static.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
+                                             ctypes.c_int32, ctypes.c_float, ctypes.c_void_p]
 _lib.kvq_dequantize.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
                                 ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
 _lib.kvq_check_status.argtypes = [_P(kvq_cache), ctypes.c_void_p]
 _lib.kvq_strerror.argtypes = [ctypes.c_int]
 _lib.kvq_strerror.restype = ctypes.c_char_p
 for _f in ("kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes", "kvq_quantize_append",
-           "kvq_decode_attention", "kvq_dequantize", "kvq_check_status"):
+           "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize", "kvq_check_status"):
     getattr(_lib, _f).restype = ctypes.c_int
 
 EXPORTS = ("kvq_layout_version", "kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes",
-           "kvq_quantize_append", "kvq_decode_attention", "kvq_dequantize", "kvq_check_status", "kvq_strerror")
+           "kvq_quantize_append", "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize",
+           "kvq_check_status", "kvq_strerror")
+STATIC_SCRATCH_BYTES = 8 << 20
 
 
 class KvqError(RuntimeError):
@@ -158,6 +162,21 @@ def kvq_decode_attention(cfg: kvq_config, cache: Cache, q: torch.Tensor, out: to
                                      _dtype_code(out.dtype), float(softmax_scale), workspace.data_ptr(),
                                      workspace.numel() * workspace.element_size(), _stream_ptr(stream)),
            "kvq_decode_attention")
+
+
+def kvq_decode_attention_static(cfg: kvq_config, cache: Cache, q: torch.Tensor, out: torch.Tensor,
+                                softmax_scale: float = 0.0, stream: Optional[torch.cuda.Stream] = None):
+    """kvq_decode_attention without a workspace argument, for callers that may not allocate device memory
+    (an engine whose arena owns all of HBM, a plug-in that only receives input/output pointers): the split
+    partials go to an 8 MiB buffer inside the library.  Raises KvqError(-8) when the configuration needs
+    more than that.  Calls that can overlap on the GPU must not share a device: they would race on the
+    buffer.  The first call on a device resolves the buffer's address; do it before any stream capture."""
+    assert q.is_cuda and out.is_cuda and q.is_contiguous() and out.is_contiguous()
+    assert tuple(q.shape) == (cfg.batch, cfg.n_q_heads, cfg.head_dim) and out.shape == q.shape
+    assert _dtype_code(q.dtype) == cfg.in_dtype
+    _check(_lib.kvq_decode_attention_static(ctypes.byref(cfg), ctypes.byref(cache.c), q.data_ptr(), out.data_ptr(),
+                                            _dtype_code(out.dtype), float(softmax_scale), _stream_ptr(stream)),
+           "kvq_decode_attention_static")
 
 
 def kvq_dequantize(cfg: kvq_config, cache: Cache, k_out: Optional[torch.Tensor], v_out: Optional[torch.Tensor],

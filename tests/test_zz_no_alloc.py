@@ -1,0 +1,70 @@
+"""Decode without a caller workspace (kvq_decode_attention_static).
+
+Who needs it: callers that are not allowed to allocate device memory around a
+decode step - a serving engine whose own arena already owns all free HBM (a
+cudaMalloc there stalls the device and may simply fail), or a plug-in that gets
+nothing but input/output pointers from its host.  The entry point keeps the
+split partials in an 8 MiB buffer inside the library instead.
+
+The test goes through the C-ABI, makes two calls in a row (the second on another
+cache and shape, so the buffer still holds the first call's partials) and checks
+each against the regular entry point with the tolerance of the parity tests.
+This file is collected last on purpose.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_15075_b200 import workloads as wl
+
+import kvq_testlib as tl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def kvq():
+    from paper_2502_15075_b200 import build
+    build.build()
+    from paper_2502_15075_b200 import kvq as mod
+    return mod
+
+
+def _case(kvq, w, B, T, seed):
+    k, v = wl.make_kv(w, layer=seed, tokens=T, batch=B)
+    cap = ((T + 127) // 128) * 128
+    cfg, gc, _ = tl.build_both(kvq, w, k, v, [T], cap)
+    q = wl.make_q(w, layer=seed, batch=B).cuda()
+    return cfg, gc, q
+
+
+def test_static_scratch_decode_matches_workspace_decode_twice(kvq):
+    cases = [_case(kvq, wl.LLAMA_8B.with_(n_kv_heads=2, n_q_heads=8), 2, 1000, 0),
+             _case(kvq, wl.LLAMA_1B.with_(n_kv_heads=4, n_q_heads=16), 3, 333, 1)]
+    for cfg, gc, q in cases:                 # two calls in a row on the shared built-in buffer
+        ref = torch.from_numpy(tl.gpu_decode(kvq, cfg, gc, q))
+        before = torch.cuda.memory_allocated()
+        out = torch.full(tuple(q.shape), float("nan"), dtype=torch.float32, device="cuda")
+        base = torch.cuda.memory_allocated()
+        kvq.kvq_decode_attention_static(cfg, gc, q, out)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == base >= before      # nothing came from torch's allocator
+        assert kvq.kvq_check_status(gc) == 0
+        tl.assert_attention_close(out.double().cpu().numpy(), ref.numpy())
+    # and the first configuration once more, after the buffer was used by a different shape
+    cfg, gc, q = cases[0]
+    out = torch.empty(tuple(q.shape), dtype=torch.float32, device="cuda")
+    kvq.kvq_decode_attention_static(cfg, gc, q, out)
+    tl.assert_attention_close(out.double().cpu().numpy(), tl.gpu_decode(kvq, cfg, gc, q))
+
+
+def test_static_scratch_rejects_oversized_problem(kvq):
+    # 512 sequences x 64 query heads need ~17 MB of split partials: more than the built-in 8 MiB
+    cfg = kvq.make_config(512, 64, 8, 128, 4, 2, 128, 128, 0, "bf16", 128)
+    assert kvq.kvq_workspace_bytes(cfg) > kvq.STATIC_SCRATCH_BYTES
+    gc = kvq.Cache(cfg)
+    q = torch.zeros((512, 64, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros((512, 64, 128), dtype=torch.float32, device="cuda")
+    with pytest.raises(kvq.KvqError) as e:
+        kvq.kvq_decode_attention_static(cfg, gc, q, out)
+    assert e.value.code == -8 and "built-in" in str(e.value)
