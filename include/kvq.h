@@ -31,12 +31,14 @@
  * (batch, kv-head) stream, regions [K codes | K meta | V codes | V meta], each
  * a multiple of 16 bytes, little-endian.  Field f of a 32-bit word holds bits
  * [f*b, f*b+b); ppw = 16/b.
- *   K codes, b in {2,4,8}: rows of D*b/8 bytes per token, each 4 chunks of
- *     D*b/32 bytes; channel d: chunk (d%8)/2, P = 2*(d/16) + (d%16)/8,
+ *   K codes, b in {2,4,8}: rows of D*b/8 bytes per token, each holding 4 chunks of
+ *     wpc = D*b/128 words; channel d: chunk (d%8)/2, P = 2*(d/16) + (d%16)/8,
  *     word P/ppw, field P%ppw + ppw*(d%2).
- *   V codes, b in {2,4,8}: 8 tiles of 16 tokens, each 32 chunks of D*b/16
- *     bytes; channel d of tile-local token tau: chunk 4*(d%8) + (tau%8)/2,
+ *   V codes, b in {2,4,8}: 8 tiles of 16 tokens, each holding 32 chunks of
+ *     wpc = D*b/64 words; channel d of tile-local token tau: chunk 4*(d%8) + (tau%8)/2,
  *     P = 4*(d/16) + (d%16)/8 + 2*(tau/8), word P/ppw, field P%ppw + ppw*(tau%2).
+ *   (chunk, word) inside a row / tile of nchunks chunks, with qw = min(wpc, 4):
+ *     byte = (word/4)*(nchunks*4*qw) + chunk*(4*qw) + (word%4)*4   (quads of words, quad-major).
  *   b = 16: rows [token][D] of the input's 16-bit patterns, no meta.
  *   Meta: (scale fp16, zero fp16) per group; per-token axis [128][D/g],
  *     per-channel K [D].

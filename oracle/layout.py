@@ -12,16 +12,20 @@ regions, in this order, each a multiple of 16 bytes:
 All multi-byte quantities are little-endian.  A b-bit code field number f of a
 32-bit word occupies bits [f*b, f*b+b).  With ppw = 16/b ("pairs per word"):
 
-K codes (b = kb in {2,4,8}): token-major rows of D*b/8 bytes; a row is 4 chunks
-of D*b/32 bytes.  Channel d of a token lives in
+K codes (b = kb in {2,4,8}): token-major rows of D*b/8 bytes; a row holds 4
+chunks of wpc = D*b/128 words.  Channel d of a token lives in
     chunk  = (d % 8) // 2
     P      = 2*(d // 16) + (d % 16) // 8          pair index inside the chunk
     word   = P // ppw,  field = P % ppw + ppw*(d % 2)
-V codes (b = vb in {2,4,8}): 8 tiles of 16 tokens, a tile is 32 chunks of
-D*b/16 bytes.  Channel d of token tau (0..15 inside its tile) lives in
+V codes (b = vb in {2,4,8}): 8 tiles of 16 tokens, a tile holds 32 chunks of
+wpc = D*b/64 words.  Channel d of token tau (0..15 inside its tile) lives in
     chunk  = 4*(d % 8) + (tau % 8) // 2
     P      = 4*(d // 16) + (d % 16) // 8 + 2*(tau // 8)
     word   = P // ppw,  field = P % ppw + ppw*(tau % 2)
+Placement of (chunk, word) inside its row / tile of `nchunks` chunks: words are
+kept in quads of qw = min(wpc, 4) words, quad-major:
+    byte   = (word // 4)*(nchunks*4*qw) + chunk*(4*qw) + (word % 4)*4
+(for wpc <= 4 this is simply chunk-major).
 b = 16 (either side): plain rows [token][D] of the input's 16-bit patterns.
 
 Meta: (scale fp16, zero fp16) pairs, 4 bytes each.  Per-token axis:
@@ -84,6 +88,11 @@ class Layout:
 # ----------------------------------------------------------------------------
 # index functions: (token in page, channel) -> (byte offset in region, bit shift)
 # ----------------------------------------------------------------------------
+def _chunk_word_byte(chunk, word, wpc, nchunks):
+    qw = min(wpc, 4)
+    return (word // 4) * (nchunks * 4 * qw) + chunk * (4 * qw) + (word % 4) * 4
+
+
 def k_code_pos(t, d, D, b):
     t = np.asarray(t)
     d = np.asarray(d)
@@ -93,7 +102,7 @@ def k_code_pos(t, d, D, b):
     word = P // ppw
     field = P % ppw + ppw * (d % 2)
     bit = field * b
-    byte = t * (D * b // 8) + chunk * (D * b // 32) + 4 * word + bit // 8
+    byte = t * (D * b // 8) + _chunk_word_byte(chunk, word, D * b // 128, 4) + bit // 8
     return byte, bit % 8
 
 
@@ -108,7 +117,7 @@ def v_code_pos(t, d, D, b):
     word = P // ppw
     field = P % ppw + ppw * (tau % 2)
     bit = field * b
-    byte = tile * (16 * D * b // 8) + chunk * (D * b // 16) + 4 * word + bit // 8
+    byte = tile * (16 * D * b // 8) + _chunk_word_byte(chunk, word, D * b // 64, 32) + bit // 8
     return byte, bit % 8
 
 

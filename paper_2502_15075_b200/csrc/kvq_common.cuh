@@ -79,11 +79,18 @@ __device__ __forceinline__ uint32_t code_of(float x, const GroupParams& p, float
 // ---------------------------------------------------------------- layout index functions
 // Byte offset (inside the K-code region of a page) of the 32-bit word holding
 // channel d of page-local token t, and the field's bit offset inside that word.
+// Byte offset of (chunk, word) inside a K row (nchunks = 4) or a V tile (nchunks = 32): words are kept
+// in quads of min(wpc, 4) words, quad-major, so that a lane's 16-byte load never conflicts with its neighbours'.
+__host__ __device__ __forceinline__ int chunk_word_byte(int chunk, int word, int wpc, int nchunks) {
+  int qw = wpc < 4 ? wpc : 4;
+  return (word >> 2) * (nchunks * 4 * qw) + chunk * (4 * qw) + (word & 3) * 4;
+}
+
 __host__ __device__ __forceinline__ void k_code_pos(int t, int d, int D, int b, int& word_byte, int& bit) {
   int ppw = 16 / b;
   int chunk = (d & 7) >> 1;
   int P = 2 * (d >> 4) + ((d & 15) >> 3);
-  word_byte = t * (D * b / 8) + chunk * (D * b / 32) + 4 * (P / ppw);
+  word_byte = t * (D * b / 8) + chunk_word_byte(chunk, P / ppw, D * b / 128, 4);
   bit = (P % ppw + ppw * (d & 1)) * b;
 }
 
@@ -92,7 +99,7 @@ __host__ __device__ __forceinline__ void v_code_pos(int t, int d, int D, int b, 
   int tile = t >> 4, tau = t & 15;
   int chunk = 4 * (d & 7) + ((tau & 7) >> 1);
   int P = 4 * (d >> 4) + ((d & 15) >> 3) + 2 * (tau >> 3);
-  word_byte = tile * (16 * D * b / 8) + chunk * (D * b / 16) + 4 * (P / ppw);
+  word_byte = tile * (16 * D * b / 8) + chunk_word_byte(chunk, P / ppw, D * b / 64, 32);
   bit = (P % ppw + ppw * (tau & 1)) * b;
 }
 

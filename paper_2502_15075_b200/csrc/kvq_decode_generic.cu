@@ -74,8 +74,8 @@ decode_generic_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float
           const uint32_t* roww = reinterpret_cast<const uint32_t*>(spage + (size_t)tp * (D * bk / 8));
           const uint32_t* meta = reinterpret_cast<const uint32_t*>(spage + g.k_meta_off);
           for (int wi = 0; wi < wpr; ++wi) {
-            uint32_t w = roww[wi];
             int chunkk = wi / wpc, word = wi % wpc;
+            uint32_t w = roww[chunk_word_byte(chunkk, word, wpc, 4) / 4];
             for (int f = 0; f < nf; ++f) {
               int d = k_field_channel(chunkk, word, f, bk);
               uint32_t mm = meta[g.k_axis == 1 ? d : tp * (D / g.gk) + d / g.gk];

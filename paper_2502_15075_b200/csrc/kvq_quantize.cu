@@ -61,7 +61,7 @@ __device__ __forceinline__ void pack_k_rows(const uint8_t* codes, int code_strid
       int d = k_field_channel(chunk, word, f, b);
       w |= (uint32_t)codes[r * code_stride + d] << (f * b);
     }
-    *reinterpret_cast<uint32_t*>(kregion + (size_t)(slot0 + r) * (D * b / 8) + wi * 4) = w;
+    *reinterpret_cast<uint32_t*>(kregion + (size_t)(slot0 + r) * (D * b / 8) + chunk_word_byte(chunk, word, wpc, 4)) = w;
   }
 }
 
@@ -111,13 +111,14 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
     const uint32_t fm = (1u << b_) - 1u;
     for (int wi = tid; wi < wpt; wi += kThreads) {
       int chunk = wi / wpc, word = wi % wpc;
-      uint32_t w = full ? 0u : vt[wi];
+      uint32_t* wp = vt + chunk_word_byte(chunk, word, wpc, 32) / 4;
+      uint32_t w = full ? 0u : *wp;
       for (int f = 0; f < nf; ++f) {
         int tau, d;
         v_field_pos(chunk, word, f, b_, tau, d);
         if (tau >= lo && tau < hi) w = (w & ~(fm << (f * b_))) | ((uint32_t)sV[tau][d] << (f * b_));
       }
-      vt[wi] = w;
+      *wp = w;
     }
   }
 }

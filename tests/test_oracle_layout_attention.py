@@ -96,6 +96,18 @@ def test_single_field_encoding_is_little_endian_words():
     assert ol.v_code_pos(0, 32, 128, 2) == (4, 0)
     # next tile of 16 tokens: 16*128*2/8 = 512 bytes further
     assert ol.v_code_pos(16, 0, 128, 2) == (512, 0)
+    # quad-major word placement when a chunk has more than 4 words:
+    # K, D=128, 8-bit (8 words per chunk): d=2 -> chunk 1 -> byte 16; d=64 -> P=8 -> word 4 -> second quad
+    # -> byte 4 chunks * 16 = 64; d=66 -> 64 + 16; d=1 -> field 0 + ppw(2) = 2 -> byte 2
+    assert ol.k_code_pos(0, 2, 128, 8) == (16, 0)
+    assert ol.k_code_pos(0, 64, 128, 8) == (64, 0)
+    assert ol.k_code_pos(0, 66, 128, 8) == (80, 0)
+    assert ol.k_code_pos(0, 1, 128, 8) == (2, 0)
+    assert ol.k_code_pos(1, 0, 128, 8) == (128, 0)
+    # V, D=128, 4-bit (8 words per chunk): d=64 -> P=16 -> word 4 -> second quad -> byte 32 chunks * 16 = 512
+    assert ol.v_code_pos(0, 64, 128, 4) == (512, 0)
+    assert ol.v_code_pos(2, 64, 128, 4) == (528, 0)
+    assert ol.v_code_pos(0, 16, 128, 4) == (4, 0)
 
 
 def test_memory_ratio_k4v2_vs_k4v4():
