@@ -1,45 +1,70 @@
-"""Build libkvq.so (sm_100a) in-tree with nvcc.  `python -m paper_2502_15075_b200.build`."""
+"""Build libkvq.so (sm_100a) in-tree with nvcc.  `python -m paper_2502_15075_b200.build [--force] [-v]`."""
 from __future__ import annotations
 
 import glob
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 LIB = os.path.join(HERE, "libkvq.so")
+OBJ_DIR = os.path.join(HERE, "_build")
 
 
 def sources():
     return sorted(glob.glob(os.path.join(HERE, "csrc", "*.cu")))
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def headers():
+    deps = []
+    for pat in ("*.h", "*.cuh", "*.inc"):
+        deps += glob.glob(os.path.join(HERE, "csrc", pat))
+    return deps + glob.glob(os.path.join(ROOT, "include", "*.h"))
+
+
+def _stale(target: str, deps) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(HERE, "csrc", "*.h")) + glob.glob(os.path.join(HERE, "csrc", "*.cuh"))
-    deps += glob.glob(os.path.join(ROOT, "include", "*.h"))
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(p) > t for p in deps)
+
+
+def needs_build() -> bool:
+    return _stale(LIB, sources() + headers())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"),
-           "-I", os.path.join(HERE, "csrc"), "-o", LIB]
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+             "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(HERE, "csrc")]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += sources()
-    res = subprocess.run(cmd, capture_output=True, text=True)
+        flags += ["-Xptxas", "-v"]
+    hdrs = headers()
+
+    def compile_one(src: str):
+        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        if not force and not _stale(obj, [src] + hdrs):
+            return obj, 0, ""
+        res = subprocess.run([nvcc] + flags + ["-c", src, "-o", obj], capture_output=True, text=True)
+        return obj, res.returncode, res.stdout + res.stderr
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 4)) as ex:
+        results = list(ex.map(compile_one, sources()))
+    log = "".join(r[2] for r in results)
+    if any(r[1] != 0 for r in results):
+        sys.stderr.write(log)
+        raise RuntimeError("nvcc failed building libkvq.so")
+    res = subprocess.run([nvcc, "-shared", "-o", LIB] + [r[0] for r in results], capture_output=True, text=True)
     if res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)
-        raise RuntimeError("nvcc failed building libkvq.so")
+        raise RuntimeError("linking libkvq.so failed")
     if verbose:
-        sys.stderr.write(res.stdout + res.stderr)
+        sys.stderr.write(log)
     return LIB
 
 

@@ -1,0 +1,104 @@
+// Dispatch of the fast decode path and its merge pass.
+#include "kvq_decode_mma_kernel.cuh"
+
+namespace kvq {
+namespace mma {
+
+// Instantiation units (kvq_decode_mma_inst_*.cu).
+#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NW)                                                              \
+  extern template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NW>(const Geom&, const CachePtrs&, const void*, \
+                                                                       float, float*, int, int, cudaStream_t);
+#include "kvq_decode_mma_list.inc"
+#undef KVQ_MMA_DECL
+
+// out[b,h,:] = sum_j 2^(m_j - m*) o_j / sum_j 2^(m_j - m*) l_j over the slots the flat split gave this stream.
+__global__ void merge_flat_kernel(Geom g, const int32_t* __restrict__ seq_len, const float* __restrict__ ws,
+                                  void* __restrict__ out, int out_dtype, int grid, int s_cap) {
+  const int bh = blockIdx.x, d = threadIdx.x;
+  const int b = bh / g.Hq, hq = bh % g.Hq;
+  const int h = hq / g.G, gh = hq % g.G;
+  const int D = g.D;
+  long long N = 0, before = 0;
+  int pages_max = 0, pages_b = 0;
+  for (int i = 0; i < g.B; ++i) {
+    int p = (seq_len[i] + kPageTokens - 1) >> 7;
+    if (i < b) before += p;
+    if (i == b) pages_b = p;
+    N += p;
+    pages_max = max(pages_max, p);
+  }
+  N *= g.Hkv;
+  before *= g.Hkv;
+  float r = 0.f;
+  if (pages_b > 0) {
+    const FlatPlan plan = make_plan(N, pages_max, grid, s_cap);
+    const long long xs = before + (long long)h * pages_b;
+    const int c_first = plan.cta_of(xs), c_last = plan.cta_of(xs + pages_b - 1);
+    const int n = min(c_last - c_first + 1, s_cap);
+    const float* base = ws + (((size_t)(b * g.Hkv + h) * s_cap) * g.G + gh) * (D + 2);
+    const size_t slot_stride = (size_t)g.G * (D + 2);
+    float mstar = -INFINITY;
+    for (int j = 0; j < n; ++j) mstar = fmaxf(mstar, base[j * slot_stride]);
+    float num = 0.f, den = 0.f;
+    if (mstar != -INFINITY) {
+      for (int j = 0; j < n; ++j) {
+        const float* pj = base + j * slot_stride;
+        const float mj = pj[0];
+        if (mj == -INFINITY) continue;
+        const float w = exp2f(mj - mstar);
+        num = fmaf(w, pj[2 + d], num);
+        den = fmaf(w, pj[1], den);
+      }
+    }
+    r = den > 0.f ? num / den : 0.f;
+  }
+  const size_t oi = (size_t)bh * D + d;
+  if (out_dtype == KVQ_FP32) static_cast<float*>(out)[oi] = r;
+  else static_cast<uint16_t*>(out)[oi] = f32_to_bits16(r, out_dtype);
+}
+
+}  // namespace mma
+
+constexpr int kFlatGrid = 2 * 148;   // two resident CTAs on each of the 148 SMs
+
+int flat_slot_cap(const Geom& g) {
+  const int streams = g.B * g.Hkv;
+  int s = (2 * kFlatGrid + streams - 1) / streams + 2;
+  if (s > g.n_pages + 1) s = g.n_pages + 1;
+  return s;
+}
+
+size_t flat_workspace_bytes(const Geom& g) {
+  return (size_t)g.B * g.Hkv * flat_slot_cap(g) * g.G * (g.D + 2) * sizeof(float);
+}
+
+static int pick(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap,
+                cudaStream_t stream, bool probe) {
+  const int ngk = (g.k_axis == 1 || g.kb == 16) ? 1 : g.D / g.gk;
+  const int ngv = (g.vb == 16) ? 1 : g.D / g.gv;
+#define KVQ_MMA_DECL(D_, KB_, VB_, KAXIS_, NGK_, NGV_, NW_)                                              \
+  if (g.D == D_ && g.kb == KB_ && g.vb == VB_ && g.k_axis == KAXIS_ && ngk == NGK_ && ngv == NGV_) {      \
+    if (probe) return KVQ_OK;                                                                             \
+    return mma::launch_mma_inst<D_, KB_, VB_, KAXIS_, NGK_, NGV_, NW_>(g, c, q, c1, ws, kFlatGrid, s_cap, stream); \
+  }
+#include "kvq_decode_mma_list.inc"
+#undef KVQ_MMA_DECL
+  return KVQ_ERR_UNSUPPORTED;
+}
+
+bool decode_mma_supported(const Geom& g) {
+  if (g.B > mma::kMaxBatchFlat) return false;
+  CachePtrs none{};
+  return pick(g, none, nullptr, 0.f, nullptr, 0, nullptr, true) == KVQ_OK;
+}
+
+int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype, float c1,
+                      float* ws, cudaStream_t stream) {
+  const int s_cap = flat_slot_cap(g);
+  int rc = pick(g, c, q, c1, ws, s_cap, stream, false);
+  if (rc != KVQ_OK) return rc;
+  mma::merge_flat_kernel<<<g.B * g.Hq, g.D, 0, stream>>>(g, c.seq_len, ws, out, out_dtype, kFlatGrid, s_cap);
+  return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
+}
+
+}  // namespace kvq

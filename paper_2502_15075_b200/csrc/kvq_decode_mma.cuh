@@ -1,0 +1,165 @@
+// Fused low-bit decode attention, fast path: softmax(q K^T / sqrt(d)) V
+// (App. A.1) over the packed cache, with K^ = z + s*code and V^ likewise
+// reconstructed inside the contraction.
+//
+// Structure (one CTA = NW consumer warps + 1 producer warp):
+//  * the producer streams whole 128-token pages into a shared-memory ring with
+//    cp.async.bulk (one bulk copy per page, completion on an mbarrier);
+//  * each consumer warp owns 16-token tiles of every page: it loads its operand
+//    fragments with 16-byte shared loads (the page layout already is fragment
+//    order), turns the codes into integer-valued fp16 with LOP3/PRMT + one HFMA2
+//    per pair, and runs QK^T and PV on the tensor cores (mma.m16n8k16, fp32
+//    accumulate) for the <= 8 query heads that share the KV head;
+//  * scale and zero-point never touch the codes:  q.K^_t = s_t (q.c_t) + z_t sum(q)
+//    and  o = sum_t (p_t s_t) c_t + sum_t p_t z_t ;
+//  * the sequence is split flat over the grid: CTA i takes the i-th equal share of
+//    all pages of all streams, writes one unnormalised partial (m, l, o) per stream
+//    it touches, and a merge pass combines them by log-sum-exp.
+// Every wait on an mbarrier is bounded in time; on expiry the kernel sets
+// KVQ_STATUS_DEVICE_TIMEOUT, keeps arriving at its barriers without computing, and returns.
+#pragma once
+
+#include "kvq_internal.h"
+
+namespace kvq {
+namespace mma {
+
+constexpr unsigned long long kWaitTimeoutNs = 2000000000ull;   // 2 s
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Wait for the phase with the given parity; gives up after kWaitTimeoutNs.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (globaltimer_ns() - t0 > kWaitTimeoutNs) return false;
+  }
+}
+// One bulk copy global -> this CTA's shared memory, completion counted in bytes on `bar`.
+// dst, src and bytes are multiples of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// D += A(16x16, row) * B(16x8, col), fp16 operands, fp32 accumulate.
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// Transpose an 8x8 matrix of 16-bit elements held one row-pair per lane.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ------------------------------------------------------------------ half2 helpers on raw registers
+__device__ __forceinline__ __half2 as_h2(uint32_t u) { return *reinterpret_cast<__half2*>(&u); }
+__device__ __forceinline__ uint32_t as_u32(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
+__device__ __forceinline__ uint32_t h2fma(uint32_t a, uint32_t b, uint32_t c) {
+  return as_u32(__hfma2(as_h2(a), as_h2(b), as_h2(c)));
+}
+__device__ __forceinline__ uint32_t pack_h2(float lo, float hi) { return as_u32(__floats2half2_rn(lo, hi)); }
+
+// ------------------------------------------------------------------ code -> fp16 conversion
+// A word holds 32/B fields; pair i = (field i, field i + 16/B) becomes one half2 register holding the two
+// codes as exact fp16 integers: the field bits are OR-ed into the mantissa of 1024.0 (0x6400), which yields
+// 1024 + code * 2^shift, and one HFMA2 with (2^-shift, -1024 * 2^-shift) brings that back to `code` exactly.
+constexpr uint32_t kMagic = 0x64006400u;   // (1024.0, 1024.0)
+
+template <int B> struct Unpack;
+
+template <> struct Unpack<4> {
+  static constexpr int PPW = 4;
+  __device__ static __forceinline__ void run(uint32_t x, uint32_t (&o)[4]) {
+    const uint32_t y = x >> 8;
+    o[0] = h2fma((x & 0x000f000fu) | kMagic, 0x3c003c00u, 0xe400e400u);   // * 1     - 1024
+    o[1] = h2fma((x & 0x00f000f0u) | kMagic, 0x2c002c00u, 0xd400d400u);   // * 1/16  - 64
+    o[2] = h2fma((y & 0x000f000fu) | kMagic, 0x3c003c00u, 0xe400e400u);
+    o[3] = h2fma((y & 0x00f000f0u) | kMagic, 0x2c002c00u, 0xd400d400u);
+  }
+};
+
+template <> struct Unpack<2> {
+  static constexpr int PPW = 8;
+  __device__ static __forceinline__ void run(uint32_t x, uint32_t (&o)[8]) {
+    const uint32_t y = x >> 10;
+    o[0] = h2fma((x & 0x00030003u) | kMagic, 0x3c003c00u, 0xe400e400u);   // * 1     - 1024
+    o[1] = h2fma((x & 0x000c000cu) | kMagic, 0x34003400u, 0xdc00dc00u);   // * 1/4   - 256
+    o[2] = h2fma((x & 0x00300030u) | kMagic, 0x2c002c00u, 0xd400d400u);   // * 1/16  - 64
+    o[3] = h2fma((x & 0x00c000c0u) | kMagic, 0x24002400u, 0xcc00cc00u);   // * 1/64  - 16
+    o[4] = h2fma((x & 0x03000300u) | kMagic, 0x1c001c00u, 0xc400c400u);   // * 1/256 - 4
+    o[5] = h2fma((y & 0x00030003u) | kMagic, 0x3c003c00u, 0xe400e400u);
+    o[6] = h2fma((y & 0x000c000cu) | kMagic, 0x34003400u, 0xdc00dc00u);
+    o[7] = h2fma((y & 0x00300030u) | kMagic, 0x2c002c00u, 0xd400d400u);
+  }
+};
+
+template <> struct Unpack<8> {
+  static constexpr int PPW = 2;
+  __device__ static __forceinline__ void run(uint32_t x, uint32_t (&o)[2]) {
+    // bytes (b0, 0x64, b2, 0x64) and (b1, 0x64, b3, 0x64): 1024 + code in each half
+    o[0] = h2fma(__byte_perm(x, 0x64646464u, 0x4240), 0x3c003c00u, 0xe400e400u);
+    o[1] = h2fma(__byte_perm(x, 0x64646464u, 0x4341), 0x3c003c00u, 0xe400e400u);
+  }
+};
+
+// Load a lane's NWORDS words of chunk `chunk` from a row / tile that holds `nchunks` chunks (quad-major).
+template <int NWORDS>
+__device__ __forceinline__ void load_chunk(const uint8_t* base, int chunk, int nchunks, uint32_t (&w)[NWORDS]) {
+  if constexpr (NWORDS >= 4) {
+#pragma unroll
+    for (int qd = 0; qd < NWORDS / 4; ++qd) {
+      uint4 v = *reinterpret_cast<const uint4*>(base + qd * (nchunks * 16) + chunk * 16);
+      w[4 * qd + 0] = v.x; w[4 * qd + 1] = v.y; w[4 * qd + 2] = v.z; w[4 * qd + 3] = v.w;
+    }
+  } else if constexpr (NWORDS == 2) {
+    uint2 v = *reinterpret_cast<const uint2*>(base + chunk * 8);
+    w[0] = v.x; w[1] = v.y;
+  } else {
+    w[0] = *reinterpret_cast<const uint32_t*>(base + chunk * 4);
+  }
+}
+
+__device__ __forceinline__ float meta_s(uint32_t m) { return __half2float(__ushort_as_half((uint16_t)(m & 0xFFFF))); }
+__device__ __forceinline__ float meta_z(uint32_t m) { return __half2float(__ushort_as_half((uint16_t)(m >> 16))); }
+
+}  // namespace mma
+}  // namespace kvq

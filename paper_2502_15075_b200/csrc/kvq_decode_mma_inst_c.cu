@@ -1,0 +1,13 @@
+// Explicit instantiations of the fast decode kernel (split over several files to compile in parallel).
+#include "kvq_decode_mma_kernel.cuh"
+
+namespace kvq {
+namespace mma {
+#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NW) \
+  template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NW>(const Geom&, const CachePtrs&, const void*, float, \
+                                                               float*, int, int, cudaStream_t);
+KVQ_MMA_DECL(64, 4, 2, 0, 2, 2, 8)
+KVQ_MMA_DECL(64, 4, 2, 0, 1, 1, 8)
+#undef KVQ_MMA_DECL
+}  // namespace mma
+}  // namespace kvq

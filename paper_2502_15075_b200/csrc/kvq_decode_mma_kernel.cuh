@@ -1,0 +1,475 @@
+// The templated fast decode kernel (see kvq_decode_mma.cuh for the design).
+#pragma once
+
+#include "kvq_decode_mma.cuh"
+
+namespace kvq {
+namespace mma {
+
+constexpr int kMaxBatchFlat = 1024;   // the flat partition keeps a per-batch prefix in shared memory
+
+// Flat split of all pages over the grid, identical in the decode and the merge kernel.
+struct FlatPlan {
+  long long N;       // total pages over all streams
+  int c_eff;         // CTAs that take part
+  __device__ __forceinline__ int cta_of(long long x) const { return (int)(((x + 1) * c_eff - 1) / N); }
+  __device__ __forceinline__ long long lo(int c) const { return (long long)c * N / c_eff; }
+};
+
+__device__ __forceinline__ FlatPlan make_plan(long long N, int pages_max, int grid, int s_cap) {
+  FlatPlan p;
+  p.N = N;
+  long long cap = pages_max > 0 ? (long long)(s_cap - 1) * N / pages_max : 0;
+  long long ce = grid;
+  if (ce > N) ce = N;
+  if (ce > cap) ce = cap;
+  p.c_eff = (int)ce;
+  return p;
+}
+
+// Shared-memory carve-up (dynamic): ring | barriers | prefix | combine buffer
+struct SmemLayout {
+  int page_stride, ring_bytes, bar_off, pref_off, misc_off, comb_off, total;
+};
+__host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, int nw, int D) {
+  SmemLayout s;
+  s.page_stride = (page_bytes + 127) & ~127;
+  s.ring_bytes = s.page_stride * stages;
+  s.bar_off = s.ring_bytes;
+  s.pref_off = s.bar_off + 16 * 8 * 2;                      // up to 16 stages x (full, empty)
+  s.misc_off = s.pref_off + (kMaxBatchFlat + 1) * 4;
+  s.comb_off = (s.misc_off + 64 + 127) & ~127;
+  int per_warp = (D / 16 * 4 + 4) * 32 * 4;                 // O fragments + m, l per lane
+  s.total = s.comb_off + (nw / 2 > 0 ? nw / 2 : 1) * per_warp;
+  return s;
+}
+
+template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NW>
+__global__ void __launch_bounds__((NW + 1) * 32, 2)
+decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1, float* __restrict__ ws,
+                  int s_cap, int stages) {
+  constexpr int KSTEPS = D / 16;            // k-steps of QK^T
+  constexpr int MT = D / 16;                // m-tiles of PV (channels)
+  constexpr int KW = D * KB / 128;          // K words per lane per token row
+  constexpr int VW = D * VB / 64;           // V words per lane per 16-token tile
+  constexpr int KPPW = Unpack<KB>::PPW;
+  constexpr int VPPW = Unpack<VB>::PPW;
+  constexpr int K_ROW_BYTES = D * KB / 8;
+  constexpr int V_TILE_BYTES = 16 * D * VB / 8;
+  constexpr int NCONS = NW * 32;
+  constexpr uint32_t FULL = 0xffffffffu;
+
+  extern __shared__ __align__(128) uint8_t smem[];
+  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sl.bar_off);   // full[0..stages), empty[0..stages)
+  int* sPref = reinterpret_cast<int*>(smem + sl.pref_off);
+  int* sMisc = reinterpret_cast<int*>(smem + sl.misc_off);           // [0] pages_max, [1] abort flag
+  float* sComb = reinterpret_cast<float*>(smem + sl.comb_off);
+
+  const int tid_ = threadIdx.x, lane = tid_ & 31, warp = tid_ >> 5;
+  const int gid = lane >> 2, tid = lane & 3;
+  const int B = g.B, Hkv = g.Hkv, G = g.G;
+
+  // ---- plan: pages per sequence, prefix over the batch
+  if (tid_ == 0) { sPref[0] = 0; sMisc[0] = 0; sMisc[1] = 0; }
+  __syncthreads();
+  for (int b = tid_; b < B; b += blockDim.x) {
+    int pages = (c.seq_len[b] + kPageTokens - 1) >> 7;
+    sPref[b + 1] = pages * Hkv;
+    atomicMax(&sMisc[0], pages);
+  }
+  __syncthreads();
+  if (warp == 0) {
+    int carry = 0;
+    for (int base = 0; base < B; base += 32) {
+      int i = base + lane;
+      int v = (i < B) ? sPref[i + 1] : 0;
+      for (int off = 1; off < 32; off <<= 1) {
+        int u = __shfl_up_sync(FULL, v, off);
+        if (lane >= off) v += u;
+      }
+      if (i < B) sPref[i + 1] = v + carry;
+      carry += __shfl_sync(FULL, v, 31);
+    }
+  }
+  if (tid_ == 0) {
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(smem_u32(&bars[s]), 1);
+      mbar_init(smem_u32(&bars[stages + s]), NW);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const FlatPlan plan = make_plan(sPref[B], sMisc[0], gridDim.x, s_cap);
+  if (plan.N == 0 || (int)blockIdx.x >= plan.c_eff) return;
+  const long long x_lo = plan.lo(blockIdx.x), x_hi = plan.lo(blockIdx.x + 1);
+
+  // ---- cursor: first page of this CTA -> (b, h, page)
+  int b = 0;
+  {
+    int lo_ = 0, hi_ = B - 1;            // last b with sPref[b] <= x_lo
+    while (lo_ < hi_) {
+      int mid = (lo_ + hi_ + 1) >> 1;
+      if (sPref[mid] <= x_lo) lo_ = mid; else hi_ = mid - 1;
+    }
+    b = lo_;
+  }
+  int pages_b = (sPref[b + 1] - sPref[b]) / Hkv;
+  int h = (int)((x_lo - sPref[b]) / pages_b);
+  int page = (int)((x_lo - sPref[b]) % pages_b);
+  const uint32_t ring = smem_u32(smem);
+  volatile int* abort_flag = sMisc + 1;
+
+  // =========================================================== producer warp
+  if (warp == NW) {
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (long long x = x_lo; x < x_hi && ok; ++x, ++it) {
+        const int stage = it % stages, round = it / stages;
+        if (round > 0) {
+          ok = mbar_wait(smem_u32(&bars[stages + stage]), (round - 1) & 1);
+          if (!ok || *abort_flag) { ok = false; break; }
+        }
+        const uint8_t* src = c.pages + ((size_t)(b * Hkv + h) * g.n_pages + page) * (size_t)g.page_bytes;
+        const uint32_t fb = smem_u32(&bars[stage]);
+        mbar_expect_tx(fb, (uint32_t)g.page_bytes);
+        bulk_load(ring + stage * sl.page_stride, src, (uint32_t)g.page_bytes, fb);
+        if (++page == pages_b) {
+          page = 0;
+          if (++h == Hkv) {
+            h = 0;
+            do { ++b; } while (b < B && sPref[b + 1] == sPref[b]);
+            if (b < B) pages_b = (sPref[b + 1] - sPref[b]) / Hkv;
+          }
+        }
+      }
+      if (!ok) {
+        // gave up: flag it, then let the copies already in flight land before the CTA exits
+        *abort_flag = 1;
+        atomicOr(c.status, KVQ_STATUS_DEVICE_TIMEOUT);
+        for (int k = 1; k <= stages && k <= it; ++k) {
+          const int j = it - k;
+          mbar_wait(smem_u32(&bars[j % stages]), (j / stages) & 1);
+        }
+      }
+    }
+    return;
+  }
+
+  // =========================================================== consumer warps
+  uint32_t qf[2 * KSTEPS];                   // B fragments of q (fp16), heads >= G are zero
+  float qsum[2][NGK];                        // sum of q over each key group, heads (2 tid, 2 tid + 1)
+  float O[MT][4];
+  float zacc[2][NGV];
+  float m0, m1, l0, l1;
+  int it = 0;
+  bool aborted = false;
+
+  for (long long x = x_lo; x < x_hi;) {
+    const int seg_pages = (int)min((long long)(pages_b - page), x_hi - x);
+    const int n_tok = c.seq_len[b];
+    const int stream = b * Hkv + h;
+
+    // ---- segment start: q fragments and group sums for this stream's heads
+    {
+      float part[NGK];
+#pragma unroll
+      for (int j = 0; j < NGK; ++j) part[j] = 0.f;
+      const uint16_t* qrow = q + ((size_t)b * g.Hq + (size_t)h * G + gid) * D;
+#pragma unroll
+      for (int s = 0; s < KSTEPS; ++s) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          uint32_t v = 0;
+          if (gid < G) {
+            uint32_t raw = *reinterpret_cast<const uint32_t*>(qrow + 16 * s + 2 * tid + 8 * hh);
+            float f0 = bits16_to_f32((uint16_t)(raw & 0xFFFF), g.in_dtype);
+            float f1 = bits16_to_f32((uint16_t)(raw >> 16), g.in_dtype);
+            v = pack_h2(f0, f1);
+            __half2 hv = as_h2(v);
+            part[s / (KSTEPS / NGK)] += __low2float(hv) + __high2float(hv);
+          }
+          qf[2 * s + hh] = v;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < NGK; ++j) {
+        float v = part[j];
+        v += __shfl_xor_sync(FULL, v, 1);
+        v += __shfl_xor_sync(FULL, v, 2);
+        qsum[0][j] = __shfl_sync(FULL, v, (2 * tid) * 4);
+        qsum[1][j] = __shfl_sync(FULL, v, (2 * tid + 1) * 4);
+      }
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) { O[mt][0] = O[mt][1] = O[mt][2] = O[mt][3] = 0.f; }
+#pragma unroll
+      for (int j = 0; j < NGV; ++j) { zacc[0][j] = zacc[1][j] = 0.f; }
+      m0 = m1 = -INFINITY;
+      l0 = l1 = 0.f;
+    }
+
+    for (int pp = 0; pp < seg_pages; ++pp, ++it) {
+      const int pg = page + pp;
+      const int nv = min(kPageTokens, n_tok - pg * kPageTokens);
+      const int stage = it % stages;
+      if (!aborted) {
+        const bool got = !*abort_flag && mbar_wait(smem_u32(&bars[stage]), (it / stages) & 1);
+        if (!__all_sync(FULL, got)) {
+          aborted = true;
+          *abort_flag = 1;
+          if (lane == 0) atomicOr(c.status, KVQ_STATUS_DEVICE_TIMEOUT);
+        }
+      }
+      if (!aborted) {
+        const uint8_t* sp = smem + stage * sl.page_stride;
+        const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
+        const int ntiles = (nv + 15) >> 4;
+
+        // ---- channel-wise keys: per page, fold the channel scales into q and get sum_d q_d z_d by one more mma
+        uint32_t qs[(KAXIS == 1) ? 2 * KSTEPS : 1];
+        float zq0 = 0.f, zq1 = 0.f;
+        if constexpr (KAXIS == 1) {
+          if (!tail_k) {
+            const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
+            float sz[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int s = 0; s < KSTEPS; ++s) {
+              uint32_t zf[2];
+#pragma unroll
+              for (int hh = 0; hh < 2; ++hh) {
+                uint2 mm = *reinterpret_cast<const uint2*>(km + 16 * s + 2 * tid + 8 * hh);
+                uint32_t sc2 = __byte_perm(mm.x, mm.y, 0x5410);
+                zf[hh] = __byte_perm(mm.x, mm.y, 0x7632);
+                qs[2 * s + hh] = as_u32(__hmul2(as_h2(qf[2 * s + hh]), as_h2(sc2)));
+              }
+              mma16816(sz, zf[0], zf[0], zf[1], zf[1], qf[2 * s], qf[2 * s + 1]);
+            }
+            zq0 = sz[0];
+            zq1 = sz[1];
+          }
+        }
+
+        for (int tile = warp; tile < ntiles; tile += NW) {
+          const int tok0 = tile * 16 + gid;            // page-local tokens of this lane's two rows
+          const bool v0 = tok0 < nv, v1 = tok0 + 8 < nv;
+          float L[4];
+
+          // ---------------- logits
+          if (KAXIS == 1 && tail_k) {
+            const uint16_t* tl = c.k_tail + ((size_t)stream * kPageTokens + tok0) * D;
+            float S[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int s = 0; s < KSTEPS; ++s) {
+              const int col = 16 * s + 2 * tid;
+              uint32_t a0 = v0 ? *reinterpret_cast<const uint32_t*>(tl + col) : 0u;
+              uint32_t a1 = v1 ? *reinterpret_cast<const uint32_t*>(tl + 8 * D + col) : 0u;
+              uint32_t a2 = v0 ? *reinterpret_cast<const uint32_t*>(tl + col + 8) : 0u;
+              uint32_t a3 = v1 ? *reinterpret_cast<const uint32_t*>(tl + 8 * D + col + 8) : 0u;
+              mma16816(S, a0, a1, a2, a3, qf[2 * s], qf[2 * s + 1]);
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) L[r] = c1 * S[r];
+          } else {
+            uint32_t ka[KW], kb2[KW];
+            const uint8_t* krow = sp + (size_t)tok0 * K_ROW_BYTES;
+            load_chunk<KW>(krow, tid, 4, ka);
+            load_chunk<KW>(krow + 8 * K_ROW_BYTES, tid, 4, kb2);
+            float S[NGK][4];
+#pragma unroll
+            for (int j = 0; j < NGK; ++j) { S[j][0] = S[j][1] = S[j][2] = S[j][3] = 0.f; }
+#pragma unroll
+            for (int w = 0; w < KW; ++w) {
+              uint32_t pa[KPPW], pb[KPPW];
+              Unpack<KB>::run(ka[w], pa);
+              Unpack<KB>::run(kb2[w], pb);
+#pragma unroll
+              for (int i = 0; i < KPPW; i += 2) {
+                const int s = (w * KPPW + i) / 2;
+                if constexpr (KAXIS == 1)
+                  mma16816(S[0], pa[i], pb[i], pa[i + 1], pb[i + 1], qs[2 * s], qs[2 * s + 1]);
+                else
+                  mma16816(S[s / (KSTEPS / NGK)], pa[i], pb[i], pa[i + 1], pb[i + 1], qf[2 * s], qf[2 * s + 1]);
+              }
+            }
+            if constexpr (KAXIS == 1) {
+              L[0] = c1 * (S[0][0] + zq0); L[1] = c1 * (S[0][1] + zq1);
+              L[2] = c1 * (S[0][2] + zq0); L[3] = c1 * (S[0][3] + zq1);
+            } else {
+              const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
+              L[0] = L[1] = L[2] = L[3] = 0.f;
+#pragma unroll
+              for (int j = 0; j < NGK; ++j) {
+                const uint32_t ma = km[tok0 * NGK + j], mb = km[(tok0 + 8) * NGK + j];
+                const float sa = c1 * meta_s(ma), za = c1 * meta_z(ma);
+                const float sb = c1 * meta_s(mb), zb = c1 * meta_z(mb);
+                L[0] += sa * S[j][0] + za * qsum[0][j];
+                L[1] += sa * S[j][1] + za * qsum[1][j];
+                L[2] += sb * S[j][2] + zb * qsum[0][j];
+                L[3] += sb * S[j][3] + zb * qsum[1][j];
+              }
+            }
+          }
+          if (!v0) { L[0] = -INFINITY; L[1] = -INFINITY; }
+          if (!v1) { L[2] = -INFINITY; L[3] = -INFINITY; }
+
+          // ---------------- online softmax (rescale only when some logit exceeds the running max)
+          const bool grow = (L[0] > m0) | (L[2] > m0) | (L[1] > m1) | (L[3] > m1);
+          if (__any_sync(FULL, grow)) {
+            float t0 = fmaxf(L[0], L[2]), t1 = fmaxf(L[1], L[3]);
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+              t0 = fmaxf(t0, __shfl_xor_sync(FULL, t0, off));
+              t1 = fmaxf(t1, __shfl_xor_sync(FULL, t1, off));
+            }
+            const float n0 = fmaxf(m0, t0), n1 = fmaxf(m1, t1);
+            const float a0 = (n0 == -INFINITY) ? 1.f : ex2(m0 - n0);
+            const float a1 = (n1 == -INFINITY) ? 1.f : ex2(m1 - n1);
+            m0 = n0; m1 = n1;
+            l0 *= a0; l1 *= a1;
+#pragma unroll
+            for (int j = 0; j < NGV; ++j) { zacc[0][j] *= a0; zacc[1][j] *= a1; }
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) { O[mt][0] *= a0; O[mt][1] *= a1; O[mt][2] *= a0; O[mt][3] *= a1; }
+          }
+          float p[4];
+          p[0] = ex2(L[0] - m0); p[1] = ex2(L[1] - m1); p[2] = ex2(L[2] - m0); p[3] = ex2(L[3] - m1);
+          l0 += p[0] + p[2];
+          l1 += p[1] + p[3];
+
+          // ---------------- values: fold the scale into p, keep the zero-point term as a scalar per group
+          const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + g.v_meta_off);
+          uint32_t bw[NGV][2];
+#pragma unroll
+          for (int j = 0; j < NGV; ++j) {
+            const uint32_t ma = v0 ? vm[tok0 * NGV + j] : 0u;
+            const uint32_t mb = v1 ? vm[(tok0 + 8) * NGV + j] : 0u;
+            const float sa = meta_s(ma), za = meta_z(ma), sb = meta_s(mb), zb = meta_z(mb);
+            zacc[0][j] += p[0] * za + p[2] * zb;
+            zacc[1][j] += p[1] * za + p[3] * zb;
+            bw[j][0] = movmatrix_trans(pack_h2(p[0] * sa, p[1] * sa));
+            bw[j][1] = movmatrix_trans(pack_h2(p[2] * sb, p[3] * sb));
+          }
+          uint32_t vw[VW];
+          load_chunk<VW>(sp + g.v_codes_off + (size_t)tile * V_TILE_BYTES, lane, 32, vw);
+          uint32_t pv[4 * MT];
+#pragma unroll
+          for (int w = 0; w < VW; ++w) {
+            uint32_t t[VPPW];
+            Unpack<VB>::run(vw[w], t);
+#pragma unroll
+            for (int i = 0; i < VPPW; ++i) pv[w * VPPW + i] = t[i];
+          }
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            const int j = mt / (MT / NGV);
+            mma16816(O[mt], pv[4 * mt], pv[4 * mt + 1], pv[4 * mt + 2], pv[4 * mt + 3], bw[j][0], bw[j][1]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars[stages + stage]));
+    }
+
+    // ---- segment end: finish this warp's state, combine the NW warps, write the partial
+    {
+#pragma unroll
+      for (int off = 4; off < 32; off <<= 1) {
+        l0 += __shfl_xor_sync(FULL, l0, off);
+        l1 += __shfl_xor_sync(FULL, l1, off);
+#pragma unroll
+        for (int j = 0; j < NGV; ++j) {
+          zacc[0][j] += __shfl_xor_sync(FULL, zacc[0][j], off);
+          zacc[1][j] += __shfl_xor_sync(FULL, zacc[1][j], off);
+        }
+      }
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        const int j = mt / (MT / NGV);
+        O[mt][0] += zacc[0][j]; O[mt][1] += zacc[1][j]; O[mt][2] += zacc[0][j]; O[mt][3] += zacc[1][j];
+      }
+      constexpr int PER_LANE = MT * 4 + 4;
+#pragma unroll
+      for (int step = NW / 2; step >= 1; step >>= 1) {
+        if (warp >= step && warp < 2 * step) {
+          float* dst = sComb + (size_t)(warp - step) * PER_LANE * 32 + lane;
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+            for (int r = 0; r < 4; ++r) dst[(mt * 4 + r) * 32] = O[mt][r];
+          }
+          dst[(MT * 4 + 0) * 32] = m0; dst[(MT * 4 + 1) * 32] = m1;
+          dst[(MT * 4 + 2) * 32] = l0; dst[(MT * 4 + 3) * 32] = l1;
+        }
+        named_bar_sync(1, NCONS);
+        if (warp < step) {
+          const float* src = sComb + (size_t)warp * PER_LANE * 32 + lane;
+          const float om0 = src[(MT * 4 + 0) * 32], om1 = src[(MT * 4 + 1) * 32];
+          const float n0 = fmaxf(m0, om0), n1 = fmaxf(m1, om1);
+          const float fa0 = (n0 == -INFINITY) ? 0.f : ex2(m0 - n0), fb0 = (n0 == -INFINITY) ? 0.f : ex2(om0 - n0);
+          const float fa1 = (n1 == -INFINITY) ? 0.f : ex2(m1 - n1), fb1 = (n1 == -INFINITY) ? 0.f : ex2(om1 - n1);
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            O[mt][0] = O[mt][0] * fa0 + src[(mt * 4 + 0) * 32] * fb0;
+            O[mt][1] = O[mt][1] * fa1 + src[(mt * 4 + 1) * 32] * fb1;
+            O[mt][2] = O[mt][2] * fa0 + src[(mt * 4 + 2) * 32] * fb0;
+            O[mt][3] = O[mt][3] * fa1 + src[(mt * 4 + 3) * 32] * fb1;
+          }
+          l0 = l0 * fa0 + src[(MT * 4 + 2) * 32] * fb0;
+          l1 = l1 * fa1 + src[(MT * 4 + 3) * 32] * fb1;
+          m0 = n0; m1 = n1;
+        }
+        named_bar_sync(1, NCONS);
+      }
+      if (warp == 0) {
+        const long long xs = (long long)sPref[b] + (long long)h * pages_b;     // first page of this stream
+        const int slot = (int)blockIdx.x - plan.cta_of(xs);
+        if (slot >= 0 && slot < s_cap) {
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int head = 2 * tid + e;
+            if (head < G) {
+              float* dst = ws + (((size_t)stream * s_cap + slot) * G + head) * (D + 2);
+              if (gid == 0) { dst[0] = e ? m1 : m0; dst[1] = e ? l1 : l0; }
+#pragma unroll
+              for (int mt = 0; mt < MT; ++mt) {
+                dst[2 + 16 * mt + gid] = O[mt][e];
+                dst[2 + 16 * mt + gid + 8] = O[mt][2 + e];
+              }
+            }
+          }
+        }
+      }
+    }
+
+    // ---- advance the cursor past this segment
+    x += seg_pages;
+    page += seg_pages;
+    if (page == pages_b) {
+      page = 0;
+      if (++h == Hkv) {
+        h = 0;
+        do { ++b; } while (b < B && sPref[b + 1] == sPref[b]);
+        if (b < B) pages_b = (sPref[b + 1] - sPref[b]) / Hkv;
+      }
+    }
+  }
+}
+
+// Launches one instantiation; defined per instantiation unit.
+template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NW>
+int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int grid, int s_cap,
+                    cudaStream_t stream) {
+  int stages = (112 * 1024 - smem_layout(0, 0, NW, D).total) / ((g.page_bytes + 127) & ~127);
+  if (stages > 8) stages = 8;
+  if (stages < 2) return KVQ_ERR_UNSUPPORTED;
+  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D);
+  auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NW>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
+    return KVQ_ERR_CUDA_LAUNCH;
+  kern<<<grid, (NW + 1) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap, stages);
+  return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
+}
+
+}  // namespace mma
+}  // namespace kvq

@@ -1,6 +1,7 @@
 // C-ABI layer of libkvq: argument validation, geometry, dispatch.  No device
 // memory is allocated or retained here; all work is queued on the caller's stream.
 #include <math.h>
+#include <stdlib.h>
 
 #include "kvq_internal.h"
 
@@ -71,15 +72,21 @@ int decode_num_splits(const Geom& g) {
 }
 
 size_t decode_workspace_bytes(const Geom& g) {
-  return (size_t)g.B * g.Hq * decode_num_splits(g) * (g.D + 2) * sizeof(float);
+  size_t generic = (size_t)g.B * g.Hq * decode_num_splits(g) * (g.D + 2) * sizeof(float);
+  size_t flat = flat_workspace_bytes(g);
+  return generic > flat ? generic : flat;
 }
 
 int launch_decode_attention(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
                             float softmax_scale, void* workspace, cudaStream_t stream) {
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)g.D);
   const float scale_log2e = scale * 1.4426950408889634f;
-  const int n_split = decode_num_splits(g);
   float* ws = static_cast<float*>(workspace);
+  // KVQ_DECODE_GENERIC=1 (debugging aid) routes every configuration through the plain-ALU kernel.
+  const char* force_generic = getenv("KVQ_DECODE_GENERIC");
+  const bool use_mma = decode_mma_supported(g) && !(force_generic && force_generic[0] == '1');
+  if (use_mma) return launch_decode_mma(g, c, q, out, out_dtype, scale_log2e, ws, stream);
+  const int n_split = decode_num_splits(g);
   int rc = launch_decode_generic(g, c, q, scale_log2e, ws, n_split, stream);
   if (rc != KVQ_OK) return rc;
   return launch_merge(g, ws, out, out_dtype, n_split, stream);

@@ -25,3 +25,11 @@ int launch_decode_generic(const Geom& g, const CachePtrs& c, const void* q, floa
                           int n_split, cudaStream_t stream);
 int launch_merge(const Geom& g, const float* ws, void* out, int out_dtype, int n_split, cudaStream_t stream);
 }  // namespace kvq
+
+namespace kvq {
+// fast (tensor-core) decode path: flat split over the grid
+bool decode_mma_supported(const Geom& g);
+size_t flat_workspace_bytes(const Geom& g);
+int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
+                      float scale_log2e, float* ws, cudaStream_t stream);
+}  // namespace kvq
