@@ -5,9 +5,10 @@ namespace kvq {
 namespace mma {
 
 // Instantiation units (kvq_decode_mma_inst_*.cu).
-#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NW)                                                              \
-  extern template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NW>(const Geom&, const CachePtrs&, const void*, \
-                                                                       float, float*, int, int, cudaStream_t);
+#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NW, MINB)                                                 \
+  extern template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NW, MINB>(const Geom&, const CachePtrs&,    \
+                                                                             const void*, float, float*, int, \
+                                                                             cudaStream_t);
 #include "kvq_decode_mma_list.inc"
 #undef KVQ_MMA_DECL
 
@@ -59,7 +60,7 @@ __global__ void merge_flat_kernel(Geom g, const int32_t* __restrict__ seq_len, c
 
 }  // namespace mma
 
-constexpr int kFlatGrid = 2 * 148;   // two resident CTAs on each of the 148 SMs
+constexpr int kFlatGrid = 2 * 148;   // slot capacity is sized for grids up to twice this
 
 int flat_slot_cap(const Geom& g) {
   const int streams = g.B * g.Hkv;
@@ -72,14 +73,16 @@ size_t flat_workspace_bytes(const Geom& g) {
   return (size_t)g.B * g.Hkv * flat_slot_cap(g) * g.G * (g.D + 2) * sizeof(float);
 }
 
+// Finds the instantiation for this geometry; launches it unless `probe`.  *grid = CTAs of the launch.
 static int pick(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap,
-                cudaStream_t stream, bool probe) {
+                cudaStream_t stream, bool probe, int* grid) {
   const int ngk = (g.k_axis == 1 || g.kb == 16) ? 1 : g.D / g.gk;
   const int ngv = (g.vb == 16) ? 1 : g.D / g.gv;
-#define KVQ_MMA_DECL(D_, KB_, VB_, KAXIS_, NGK_, NGV_, NW_)                                              \
-  if (g.D == D_ && g.kb == KB_ && g.vb == VB_ && g.k_axis == KAXIS_ && ngk == NGK_ && ngv == NGV_) {      \
-    if (probe) return KVQ_OK;                                                                             \
-    return mma::launch_mma_inst<D_, KB_, VB_, KAXIS_, NGK_, NGV_, NW_>(g, c, q, c1, ws, kFlatGrid, s_cap, stream); \
+#define KVQ_MMA_DECL(D_, KB_, VB_, KAXIS_, NGK_, NGV_, NW_, MINB_)                                            \
+  if (g.D == D_ && g.kb == KB_ && g.vb == VB_ && g.k_axis == KAXIS_ && ngk == NGK_ && ngv == NGV_) {           \
+    *grid = 148 * MINB_;                                                                                       \
+    if (probe) return KVQ_OK;                                                                                  \
+    return mma::launch_mma_inst<D_, KB_, VB_, KAXIS_, NGK_, NGV_, NW_, MINB_>(g, c, q, c1, ws, s_cap, stream); \
   }
 #include "kvq_decode_mma_list.inc"
 #undef KVQ_MMA_DECL
@@ -89,15 +92,17 @@ static int pick(const Geom& g, const CachePtrs& c, const void* q, float c1, floa
 bool decode_mma_supported(const Geom& g) {
   if (g.B > mma::kMaxBatchFlat) return false;
   CachePtrs none{};
-  return pick(g, none, nullptr, 0.f, nullptr, 0, nullptr, true) == KVQ_OK;
+  int grid = 0;
+  return pick(g, none, nullptr, 0.f, nullptr, 0, nullptr, true, &grid) == KVQ_OK;
 }
 
 int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype, float c1,
                       float* ws, cudaStream_t stream) {
   const int s_cap = flat_slot_cap(g);
-  int rc = pick(g, c, q, c1, ws, s_cap, stream, false);
+  int grid = 0;
+  int rc = pick(g, c, q, c1, ws, s_cap, stream, false, &grid);
   if (rc != KVQ_OK) return rc;
-  mma::merge_flat_kernel<<<g.B * g.Hq, g.D, 0, stream>>>(g, c.seq_len, ws, out, out_dtype, kFlatGrid, s_cap);
+  mma::merge_flat_kernel<<<g.B * g.Hq, g.D, 0, stream>>>(g, c.seq_len, ws, out, out_dtype, grid, s_cap);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
 

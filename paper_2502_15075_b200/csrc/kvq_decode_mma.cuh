@@ -47,19 +47,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// Same, letting the hardware park the thread for up to `hint_ns` while the phase is pending.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ unsigned long long globaltimer_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Wait for the phase with the given parity; gives up after kWaitTimeoutNs.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
+// Slow path of a wait: poll with a parking hint, give up after kWaitTimeoutNs.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
   const unsigned long long t0 = globaltimer_ns();
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
     if (globaltimer_ns() - t0 > kWaitTimeoutNs) return false;
   }
+}
+// Wait for the phase with the given parity; bounded in time (false = gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity);
 }
 // One bulk copy global -> this CTA's shared memory, completion counted in bytes on `bar`.
 // dst, src and bytes are multiples of 16.
@@ -104,16 +118,24 @@ __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) { return as_u32(
 // 1024 + code * 2^shift, and one HFMA2 with (2^-shift, -1024 * 2^-shift) brings that back to `code` exactly.
 constexpr uint32_t kMagic = 0x64006400u;   // (1024.0, 1024.0)
 
+// (x & MASK) | 0x64006400 as one LOP3 (truth table 0xEA = (a & b) | c).
+template <uint32_t MASK>
+__device__ __forceinline__ uint32_t field_to_magic(uint32_t x) {
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "n"(MASK), "r"(kMagic));
+  return d;
+}
+
 template <int B> struct Unpack;
 
 template <> struct Unpack<4> {
   static constexpr int PPW = 4;
   __device__ static __forceinline__ void run(uint32_t x, uint32_t (&o)[4]) {
     const uint32_t y = x >> 8;
-    o[0] = h2fma((x & 0x000f000fu) | kMagic, 0x3c003c00u, 0xe400e400u);   // * 1     - 1024
-    o[1] = h2fma((x & 0x00f000f0u) | kMagic, 0x2c002c00u, 0xd400d400u);   // * 1/16  - 64
-    o[2] = h2fma((y & 0x000f000fu) | kMagic, 0x3c003c00u, 0xe400e400u);
-    o[3] = h2fma((y & 0x00f000f0u) | kMagic, 0x2c002c00u, 0xd400d400u);
+    o[0] = h2fma(field_to_magic<0x000f000fu>(x), 0x3c003c00u, 0xe400e400u);   // * 1     - 1024
+    o[1] = h2fma(field_to_magic<0x00f000f0u>(x), 0x2c002c00u, 0xd400d400u);   // * 1/16  - 64
+    o[2] = h2fma(field_to_magic<0x000f000fu>(y), 0x3c003c00u, 0xe400e400u);
+    o[3] = h2fma(field_to_magic<0x00f000f0u>(y), 0x2c002c00u, 0xd400d400u);
   }
 };
 
@@ -121,14 +143,14 @@ template <> struct Unpack<2> {
   static constexpr int PPW = 8;
   __device__ static __forceinline__ void run(uint32_t x, uint32_t (&o)[8]) {
     const uint32_t y = x >> 10;
-    o[0] = h2fma((x & 0x00030003u) | kMagic, 0x3c003c00u, 0xe400e400u);   // * 1     - 1024
-    o[1] = h2fma((x & 0x000c000cu) | kMagic, 0x34003400u, 0xdc00dc00u);   // * 1/4   - 256
-    o[2] = h2fma((x & 0x00300030u) | kMagic, 0x2c002c00u, 0xd400d400u);   // * 1/16  - 64
-    o[3] = h2fma((x & 0x00c000c0u) | kMagic, 0x24002400u, 0xcc00cc00u);   // * 1/64  - 16
-    o[4] = h2fma((x & 0x03000300u) | kMagic, 0x1c001c00u, 0xc400c400u);   // * 1/256 - 4
-    o[5] = h2fma((y & 0x00030003u) | kMagic, 0x3c003c00u, 0xe400e400u);
-    o[6] = h2fma((y & 0x000c000cu) | kMagic, 0x34003400u, 0xdc00dc00u);
-    o[7] = h2fma((y & 0x00300030u) | kMagic, 0x2c002c00u, 0xd400d400u);
+    o[0] = h2fma(field_to_magic<0x00030003u>(x), 0x3c003c00u, 0xe400e400u);   // * 1     - 1024
+    o[1] = h2fma(field_to_magic<0x000c000cu>(x), 0x34003400u, 0xdc00dc00u);   // * 1/4   - 256
+    o[2] = h2fma(field_to_magic<0x00300030u>(x), 0x2c002c00u, 0xd400d400u);   // * 1/16  - 64
+    o[3] = h2fma(field_to_magic<0x00c000c0u>(x), 0x24002400u, 0xcc00cc00u);   // * 1/64  - 16
+    o[4] = h2fma(field_to_magic<0x03000300u>(x), 0x1c001c00u, 0xc400c400u);   // * 1/256 - 4
+    o[5] = h2fma(field_to_magic<0x00030003u>(y), 0x3c003c00u, 0xe400e400u);
+    o[6] = h2fma(field_to_magic<0x000c000cu>(y), 0x34003400u, 0xdc00dc00u);
+    o[7] = h2fma(field_to_magic<0x00300030u>(y), 0x2c002c00u, 0xd400d400u);
   }
 };
 

@@ -3,12 +3,12 @@
 
 namespace kvq {
 namespace mma {
-#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NW) \
-  template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NW>(const Geom&, const CachePtrs&, const void*, float, \
-                                                               float*, int, int, cudaStream_t);
-KVQ_MMA_DECL(128, 4, 2, 0, 1, 1, 8)
-KVQ_MMA_DECL(128, 2, 4, 0, 1, 1, 8)
-KVQ_MMA_DECL(128, 4, 4, 0, 1, 1, 8)
+#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NW, MINB)                                          \
+  template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NW, MINB>(const Geom&, const CachePtrs&, const void*, \
+                                                                     float, float*, int, cudaStream_t);
+KVQ_MMA_DECL(128, 4, 2, 0, 1, 1, 8, 2)
+KVQ_MMA_DECL(128, 2, 4, 0, 1, 1, 8, 2)
+KVQ_MMA_DECL(128, 4, 4, 0, 1, 1, 8, 2)
 #undef KVQ_MMA_DECL
 }  // namespace mma
 }  // namespace kvq

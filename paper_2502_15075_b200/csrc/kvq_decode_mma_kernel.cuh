@@ -1,6 +1,8 @@
 // The templated fast decode kernel (see kvq_decode_mma.cuh for the design).
 #pragma once
 
+#include <type_traits>
+
 #include "kvq_decode_mma.cuh"
 
 namespace kvq {
@@ -44,8 +46,8 @@ __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, in
   return s;
 }
 
-template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NW>
-__global__ void __launch_bounds__((NW + 1) * 32, 2)
+template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NW, int MINB>
+__global__ void __launch_bounds__((NW + 1) * 32, MINB)
 decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1, float* __restrict__ ws,
                   int s_cap, int stages) {
   constexpr int KSTEPS = D / 16;            // k-steps of QK^T
@@ -118,23 +120,25 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   int h = (int)((x_lo - sPref[b]) / pages_b);
   int page = (int)((x_lo - sPref[b]) % pages_b);
   const uint32_t ring = smem_u32(smem);
+  const uint32_t bar0 = smem_u32(bars);
   volatile int* abort_flag = sMisc + 1;
 
   // =========================================================== producer warp
   if (warp == NW) {
     if (lane == 0) {
-      int it = 0;
+      int it = 0, stage = 0;
+      uint32_t phase = 1;                // parity of the previous round of `empty`
       bool ok = true;
-      for (long long x = x_lo; x < x_hi && ok; ++x, ++it) {
-        const int stage = it % stages, round = it / stages;
-        if (round > 0) {
-          ok = mbar_wait(smem_u32(&bars[stages + stage]), (round - 1) & 1);
+      for (long long x = x_lo; x < x_hi; ++x, ++it) {
+        if (it >= stages) {
+          ok = mbar_wait(bar0 + 8 * (stages + stage), phase);
           if (!ok || *abort_flag) { ok = false; break; }
         }
         const uint8_t* src = c.pages + ((size_t)(b * Hkv + h) * g.n_pages + page) * (size_t)g.page_bytes;
-        const uint32_t fb = smem_u32(&bars[stage]);
+        const uint32_t fb = bar0 + 8 * stage;
         mbar_expect_tx(fb, (uint32_t)g.page_bytes);
         bulk_load(ring + stage * sl.page_stride, src, (uint32_t)g.page_bytes, fb);
+        if (++stage == stages) { stage = 0; phase ^= 1; }
         if (++page == pages_b) {
           page = 0;
           if (++h == Hkv) {
@@ -150,7 +154,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         atomicOr(c.status, KVQ_STATUS_DEVICE_TIMEOUT);
         for (int k = 1; k <= stages && k <= it; ++k) {
           const int j = it - k;
-          mbar_wait(smem_u32(&bars[j % stages]), (j / stages) & 1);
+          mbar_wait(bar0 + 8 * (j % stages), (j / stages) & 1);
         }
       }
     }
@@ -159,11 +163,12 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
   // =========================================================== consumer warps
   uint32_t qf[2 * KSTEPS];                   // B fragments of q (fp16), heads >= G are zero
-  float qsum[2][NGK];                        // sum of q over each key group, heads (2 tid, 2 tid + 1)
+  float qsum[2][NGK];                        // c1 * sum of q over each key group, heads (2 tid, 2 tid + 1)
   float O[MT][4];
   float zacc[2][NGV];
   float m0, m1, l0, l1;
-  int it = 0;
+  int stage = 0;
+  uint32_t phase = 0;
   bool aborted = false;
 
   for (long long x = x_lo; x < x_hi;) {
@@ -198,8 +203,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         float v = part[j];
         v += __shfl_xor_sync(FULL, v, 1);
         v += __shfl_xor_sync(FULL, v, 2);
-        qsum[0][j] = __shfl_sync(FULL, v, (2 * tid) * 4);
-        qsum[1][j] = __shfl_sync(FULL, v, (2 * tid + 1) * 4);
+        qsum[0][j] = c1 * __shfl_sync(FULL, v, (2 * tid) * 4);
+        qsum[1][j] = c1 * __shfl_sync(FULL, v, (2 * tid + 1) * 4);
       }
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) { O[mt][0] = O[mt][1] = O[mt][2] = O[mt][3] = 0.f; }
@@ -209,12 +214,10 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       l0 = l1 = 0.f;
     }
 
-    for (int pp = 0; pp < seg_pages; ++pp, ++it) {
-      const int pg = page + pp;
-      const int nv = min(kPageTokens, n_tok - pg * kPageTokens);
-      const int stage = it % stages;
+    for (int pp = 0; pp < seg_pages; ++pp) {
+      const int nv = min(kPageTokens, n_tok - (page + pp) * kPageTokens);
       if (!aborted) {
-        const bool got = !*abort_flag && mbar_wait(smem_u32(&bars[stage]), (it / stages) & 1);
+        const bool got = mbar_wait(bar0 + 8 * stage, phase);
         if (!__all_sync(FULL, got)) {
           aborted = true;
           *abort_flag = 1;
@@ -245,14 +248,16 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               }
               mma16816(sz, zf[0], zf[0], zf[1], zf[1], qf[2 * s], qf[2 * s + 1]);
             }
-            zq0 = sz[0];
-            zq1 = sz[1];
+            zq0 = c1 * sz[0];
+            zq1 = c1 * sz[1];
           }
         }
 
-        for (int tile = warp; tile < ntiles; tile += NW) {
+        // One 16-token tile: logits -> online softmax -> PV.  MASKED handles a partially filled page.
+        auto do_tile = [&](const int tile, auto masked_tag) {
+          constexpr bool MASKED = decltype(masked_tag)::value;
           const int tok0 = tile * 16 + gid;            // page-local tokens of this lane's two rows
-          const bool v0 = tok0 < nv, v1 = tok0 + 8 < nv;
+          const bool v0 = !MASKED || tok0 < nv, v1 = !MASKED || tok0 + 8 < nv;
           float L[4];
 
           // ---------------- logits
@@ -293,36 +298,38 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               }
             }
             if constexpr (KAXIS == 1) {
-              L[0] = c1 * (S[0][0] + zq0); L[1] = c1 * (S[0][1] + zq1);
-              L[2] = c1 * (S[0][2] + zq0); L[3] = c1 * (S[0][3] + zq1);
+              L[0] = fmaf(c1, S[0][0], zq0); L[1] = fmaf(c1, S[0][1], zq1);
+              L[2] = fmaf(c1, S[0][2], zq0); L[3] = fmaf(c1, S[0][3], zq1);
             } else {
               const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
               L[0] = L[1] = L[2] = L[3] = 0.f;
 #pragma unroll
               for (int j = 0; j < NGK; ++j) {
-                const uint32_t ma = km[tok0 * NGK + j], mb = km[(tok0 + 8) * NGK + j];
-                const float sa = c1 * meta_s(ma), za = c1 * meta_z(ma);
-                const float sb = c1 * meta_s(mb), zb = c1 * meta_z(mb);
-                L[0] += sa * S[j][0] + za * qsum[0][j];
-                L[1] += sa * S[j][1] + za * qsum[1][j];
-                L[2] += sb * S[j][2] + zb * qsum[0][j];
-                L[3] += sb * S[j][3] + zb * qsum[1][j];
+                const float2 ma = __half22float2(as_h2(km[tok0 * NGK + j]));          // (scale, zero)
+                const float2 mb = __half22float2(as_h2(km[(tok0 + 8) * NGK + j]));
+                const float sa = c1 * ma.x, sb = c1 * mb.x;
+                L[0] += fmaf(sa, S[j][0], ma.y * qsum[0][j]);
+                L[1] += fmaf(sa, S[j][1], ma.y * qsum[1][j]);
+                L[2] += fmaf(sb, S[j][2], mb.y * qsum[0][j]);
+                L[3] += fmaf(sb, S[j][3], mb.y * qsum[1][j]);
               }
             }
           }
-          if (!v0) { L[0] = -INFINITY; L[1] = -INFINITY; }
-          if (!v1) { L[2] = -INFINITY; L[3] = -INFINITY; }
+          if (MASKED) {
+            if (!v0) { L[0] = -INFINITY; L[1] = -INFINITY; }
+            if (!v1) { L[2] = -INFINITY; L[3] = -INFINITY; }
+          }
 
           // ---------------- online softmax (rescale only when some logit exceeds the running max)
-          const bool grow = (L[0] > m0) | (L[2] > m0) | (L[1] > m1) | (L[3] > m1);
-          if (__any_sync(FULL, grow)) {
-            float t0 = fmaxf(L[0], L[2]), t1 = fmaxf(L[1], L[3]);
+          const float t0 = fmaxf(L[0], L[2]), t1 = fmaxf(L[1], L[3]);
+          if (__any_sync(FULL, (t0 > m0) | (t1 > m1))) {
+            float u0 = t0, u1 = t1;
 #pragma unroll
             for (int off = 4; off < 32; off <<= 1) {
-              t0 = fmaxf(t0, __shfl_xor_sync(FULL, t0, off));
-              t1 = fmaxf(t1, __shfl_xor_sync(FULL, t1, off));
+              u0 = fmaxf(u0, __shfl_xor_sync(FULL, u0, off));
+              u1 = fmaxf(u1, __shfl_xor_sync(FULL, u1, off));
             }
-            const float n0 = fmaxf(m0, t0), n1 = fmaxf(m1, t1);
+            const float n0 = fmaxf(m0, u0), n1 = fmaxf(m1, u1);
             const float a0 = (n0 == -INFINITY) ? 1.f : ex2(m0 - n0);
             const float a1 = (n1 == -INFINITY) ? 1.f : ex2(m1 - n1);
             m0 = n0; m1 = n1;
@@ -339,16 +346,19 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
           // ---------------- values: fold the scale into p, keep the zero-point term as a scalar per group
           const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + g.v_meta_off);
+          const uint32_t pa01 = pack_h2(p[0], p[1]), pb01 = pack_h2(p[2], p[3]);
           uint32_t bw[NGV][2];
 #pragma unroll
           for (int j = 0; j < NGV; ++j) {
             const uint32_t ma = v0 ? vm[tok0 * NGV + j] : 0u;
             const uint32_t mb = v1 ? vm[(tok0 + 8) * NGV + j] : 0u;
-            const float sa = meta_s(ma), za = meta_z(ma), sb = meta_s(mb), zb = meta_z(mb);
+            const float za = meta_z(ma), zb = meta_z(mb);
             zacc[0][j] += p[0] * za + p[2] * zb;
             zacc[1][j] += p[1] * za + p[3] * zb;
-            bw[j][0] = movmatrix_trans(pack_h2(p[0] * sa, p[1] * sa));
-            bw[j][1] = movmatrix_trans(pack_h2(p[2] * sb, p[3] * sb));
+            // (p * s) in fp16: both heads of a row share the row's scale
+            const uint32_t sa2 = __byte_perm(ma, ma, 0x1010), sb2 = __byte_perm(mb, mb, 0x1010);
+            bw[j][0] = movmatrix_trans(as_u32(__hmul2(as_h2(pa01), as_h2(sa2))));
+            bw[j][1] = movmatrix_trans(as_u32(__hmul2(as_h2(pb01), as_h2(sb2))));
           }
           uint32_t vw[VW];
           load_chunk<VW>(sp + g.v_codes_off + (size_t)tile * V_TILE_BYTES, lane, 32, vw);
@@ -365,10 +375,19 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             const int j = mt / (MT / NGV);
             mma16816(O[mt], pv[4 * mt], pv[4 * mt + 1], pv[4 * mt + 2], pv[4 * mt + 3], bw[j][0], bw[j][1]);
           }
+        };
+
+        if (nv == kPageTokens) {
+#pragma unroll 1
+          for (int tile = warp; tile < kPageTokens / 16; tile += NW) do_tile(tile, std::false_type{});
+        } else {
+#pragma unroll 1
+          for (int tile = warp; tile < ntiles; tile += NW) do_tile(tile, std::true_type{});
         }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars[stages + stage]));
+      if (lane == 0) mbar_arrive(bar0 + 8 * (stages + stage));
+      if (++stage == stages) { stage = 0; phase ^= 1; }
     }
 
     // ---- segment end: finish this warp's state, combine the NW warps, write the partial
@@ -457,17 +476,19 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 }
 
 // Launches one instantiation; defined per instantiation unit.
-template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NW>
-int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int grid, int s_cap,
+template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NW, int MINB>
+int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap,
                     cudaStream_t stream) {
-  int stages = (112 * 1024 - smem_layout(0, 0, NW, D).total) / ((g.page_bytes + 127) & ~127);
+  const int budget = (227 * 1024) / MINB - 1024;            // shared memory per CTA for MINB resident CTAs per SM
+  int stages = (budget - smem_layout(0, 0, NW, D).total) / ((g.page_bytes + 127) & ~127);
   if (stages > 8) stages = 8;
   if (stages < 2) return KVQ_ERR_UNSUPPORTED;
   const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D);
-  auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NW>;
+  auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NW, MINB>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
     return KVQ_ERR_CUDA_LAUNCH;
-  kern<<<grid, (NW + 1) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap, stages);
+  kern<<<148 * MINB, (NW + 1) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap,
+                                                         stages);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
 
