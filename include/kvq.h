@@ -30,10 +30,11 @@
  * Packed page (layout version 1): 128 consecutive tokens of one
  * (batch, kv-head) stream, regions [K codes | K meta | V codes | V meta], each
  * a multiple of 16 bytes, little-endian.  Field f of a 32-bit word holds bits
- * [f*b, f*b+b); ppw = 16/b.
+ * [f*b, f*b+b); ppw = 16/b (V codes).
  *   K codes, b in {2,4,8}: rows of D*b/8 bytes per token, each holding 4 chunks of
- *     wpc = D*b/128 words; channel d: chunk (d%8)/2, P = 2*(d/16) + (d%16)/8,
- *     word P/ppw, field P%ppw + ppw*(d%2).
+ *     wpc = D*b/128 words; with fpb = 8/b fields per byte, channel d: chunk (d%16)/4,
+ *     r = d/16, word r/fpb, bit 8*(d%4) + b*(r%fpb)  (byte j of a word holds channels
+ *     16r + 4*chunk + j: one mask per field gives four consecutive channels as four bytes).
  *   V codes, b in {2,4,8}: 8 tiles of 16 tokens, each holding 32 chunks of
  *     wpc = D*b/64 words; channel d of tile-local token tau: chunk 4*(d%8) + (tau%8)/2,
  *     P = 4*(d/16) + (d%16)/8 + 2*(tau/8), word P/ppw, field P%ppw + ppw*(tau%2).

@@ -13,10 +13,14 @@ All multi-byte quantities are little-endian.  A b-bit code field number f of a
 32-bit word occupies bits [f*b, f*b+b).  With ppw = 16/b ("pairs per word"):
 
 K codes (b = kb in {2,4,8}): token-major rows of D*b/8 bytes; a row holds 4
-chunks of wpc = D*b/128 words.  Channel d of a token lives in
-    chunk  = (d % 8) // 2
-    P      = 2*(d // 16) + (d % 16) // 8          pair index inside the chunk
-    word   = P // ppw,  field = P % ppw + ppw*(d % 2)
+chunks of wpc = D*b/128 words.  With fpb = 8/b fields per byte, channel d of a
+token lives in
+    chunk  = (d % 16) // 4
+    r      = d // 16                               register index inside the chunk
+    word   = r // fpb,  bit = 8*(d % 4) + b*(r % fpb)
+(byte j of a word holds channels 16r + 4*chunk + j for the fpb values of r that
+share the word: masking one field out of every byte yields four consecutive
+channels as four bytes).
 V codes (b = vb in {2,4,8}): 8 tiles of 16 tokens, a tile holds 32 chunks of
 wpc = D*b/64 words.  Channel d of token tau (0..15 inside its tile) lives in
     chunk  = 4*(d % 8) + (tau % 8) // 2
@@ -96,12 +100,11 @@ def _chunk_word_byte(chunk, word, wpc, nchunks):
 def k_code_pos(t, d, D, b):
     t = np.asarray(t)
     d = np.asarray(d)
-    ppw = 16 // b
-    chunk = (d % 8) // 2
-    P = 2 * (d // 16) + (d % 16) // 8
-    word = P // ppw
-    field = P % ppw + ppw * (d % 2)
-    bit = field * b
+    fpb = 8 // b                      # fields per byte
+    chunk = (d % 16) // 4
+    r = d // 16
+    word = r // fpb
+    bit = 8 * (d % 4) + b * (r % fpb)
     byte = t * (D * b // 8) + _chunk_word_byte(chunk, word, D * b // 128, 4) + bit // 8
     return byte, bit % 8
 

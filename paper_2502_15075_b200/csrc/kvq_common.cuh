@@ -87,11 +87,11 @@ __host__ __device__ __forceinline__ int chunk_word_byte(int chunk, int word, int
 }
 
 __host__ __device__ __forceinline__ void k_code_pos(int t, int d, int D, int b, int& word_byte, int& bit) {
-  int ppw = 16 / b;
-  int chunk = (d & 7) >> 1;
-  int P = 2 * (d >> 4) + ((d & 15) >> 3);
-  word_byte = t * (D * b / 8) + chunk_word_byte(chunk, P / ppw, D * b / 128, 4);
-  bit = (P % ppw + ppw * (d & 1)) * b;
+  int fpb = 8 / b;              // fields per byte
+  int chunk = (d & 15) >> 2;
+  int r = d >> 4;               // register index inside the chunk
+  word_byte = t * (D * b / 8) + chunk_word_byte(chunk, r / fpb, D * b / 128, 4);
+  bit = 8 * (d & 3) + b * (r % fpb);
 }
 
 __host__ __device__ __forceinline__ void v_code_pos(int t, int d, int D, int b, int& word_byte, int& bit) {
@@ -105,9 +105,9 @@ __host__ __device__ __forceinline__ void v_code_pos(int t, int d, int D, int b, 
 
 // Inverse maps: which channel (and tile-local token) sits in field f of a word.
 __device__ __forceinline__ int k_field_channel(int chunk, int word, int f, int b) {
-  int ppw = 16 / b;
-  int P = word * ppw + (f % ppw);
-  return 16 * (P >> 1) + 8 * (P & 1) + 2 * chunk + (f / ppw);
+  int fpb = 8 / b;
+  int r = word * fpb + (f % fpb);
+  return 16 * r + 4 * chunk + (f / fpb);
 }
 
 __device__ __forceinline__ void v_field_pos(int chunk, int word, int f, int b, int& tau, int& d) {

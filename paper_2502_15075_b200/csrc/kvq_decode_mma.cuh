@@ -92,6 +92,13 @@ __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+// D += A(16x32, row, unsigned bytes) * B(32x8, col, signed bytes), int32 accumulate.
+__device__ __forceinline__ void mma16832_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 // Transpose an 8x8 matrix of 16-bit elements held one row-pair per lane.
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
   uint32_t d;
@@ -124,6 +131,21 @@ __device__ __forceinline__ uint32_t field_to_magic(uint32_t x) {
   uint32_t d;
   asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "n"(MASK), "r"(kMagic));
   return d;
+}
+
+// Key codes as unsigned-byte MMA operands: masking one field out of every byte of a packed word yields the
+// codes of four consecutive channels as four bytes, ready for an integer MMA (8-bit codes need nothing at all).
+// key_slot(kw, r): the four code bytes of register slot r (channels 16 r + 4 chunk + {0..3}) of a lane's KW
+// packed words; r is a constant after unrolling.
+template <int B, int KW>
+__device__ __forceinline__ uint32_t key_slot(const uint32_t (&kw)[KW], int r) {
+  if constexpr (B == 8) {
+    return kw[r];
+  } else {
+    constexpr int FPB = 8 / B;
+    constexpr uint32_t MASK = ((1u << B) - 1u) * 0x01010101u;
+    return (kw[r / FPB] >> (B * (r % FPB))) & MASK;
+  }
 }
 
 template <int B> struct Unpack;

@@ -3,12 +3,11 @@
 
 namespace kvq {
 namespace mma {
-#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NW, MINB)                                          \
-  template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NW, MINB>(const Geom&, const CachePtrs&, const void*, \
-                                                                     float, float*, int, cudaStream_t);
-KVQ_MMA_DECL(128, 4, 2, 0, 4, 1, 8, 2)
-KVQ_MMA_DECL(128, 4, 2, 0, 1, 4, 8, 2)
-KVQ_MMA_DECL(128, 4, 2, 0, 2, 2, 8, 2)
+#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB)                                          \
+  template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB>(const Geom&, const CachePtrs&, const void*, \
+                                                                         float, float*, int, cudaStream_t);
+KVQ_MMA_DECL(128, 4, 2, 0, 1, 4, 3, 4, 3)
+KVQ_MMA_DECL(128, 4, 2, 0, 2, 2, 3, 4, 3)
 #undef KVQ_MMA_DECL
 }  // namespace mma
 }  // namespace kvq

@@ -46,20 +46,26 @@ __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, in
   return s;
 }
 
-template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NW, int MINB>
+// Template parameters: head_dim, key bits, value bits, key axis (0 token-wise: keys go through integer MMAs
+// on the raw code bytes with q in 22-bit fixed point split into NL = 3 signed bytes; 1 channel-wise: fp16 MMAs
+// with the channel scales folded into q per page), key / value groups per row, q limbs, consumer warps,
+// resident CTAs per SM.
+template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NL, int NW, int MINB>
 __global__ void __launch_bounds__((NW + 1) * 32, MINB)
 decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1, float* __restrict__ ws,
                   int s_cap, int stages) {
-  constexpr int KSTEPS = D / 16;            // k-steps of QK^T
+  constexpr int NR = D / 16;                // 16-channel register slots per row (r index of the key layout)
+  constexpr int KS32 = D / 32;              // k-steps of an 8-bit MMA
   constexpr int MT = D / 16;                // m-tiles of PV (channels)
   constexpr int KW = D * KB / 128;          // K words per lane per token row
   constexpr int VW = D * VB / 64;           // V words per lane per 16-token tile
-  constexpr int KPPW = Unpack<KB>::PPW;
+  constexpr int FPB = 8 / KB;               // key fields per byte
   constexpr int VPPW = Unpack<VB>::PPW;
   constexpr int K_ROW_BYTES = D * KB / 8;
   constexpr int V_TILE_BYTES = 16 * D * VB / 8;
   constexpr int NCONS = NW * 32;
   constexpr uint32_t FULL = 0xffffffffu;
+  static_assert(KAXIS == 0 || KB != 2, "channel-wise 2-bit keys are not instantiated");
 
   extern __shared__ __align__(128) uint8_t smem[];
   const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D);
@@ -162,8 +168,12 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   }
 
   // =========================================================== consumer warps
-  uint32_t qf[2 * KSTEPS];                   // B fragments of q (fp16), heads >= G are zero
+  // q operands: signed-byte limbs (token-wise keys) or fp16 pairs (channel-wise keys), heads >= G are zero.
+  // Slot r holds channels 16 r + 4 tid + {0..3} of head gid.
+  uint32_t ql[(KAXIS == 0) ? NL : 1][(KAXIS == 0) ? NR : 1];
+  uint32_t qf[(KAXIS == 1) ? 2 * NR : 1];    // fp16 pairs (j = 0, 2) and (j = 1, 3) of slot r
   float qsum[2][NGK];                        // c1 * sum of q over each key group, heads (2 tid, 2 tid + 1)
+  float hs0 = 0.f, hs1 = 0.f;                // c1 / fixed-point scale of heads (2 tid, 2 tid + 1)
   float O[MT][4];
   float zacc[2][NGV];
   float m0, m1, l0, l1;
@@ -176,27 +186,66 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     const int n_tok = c.seq_len[b];
     const int stream = b * Hkv + h;
 
-    // ---- segment start: q fragments and group sums for this stream's heads
+    // ---- segment start: q operands and group sums for this stream's heads
     {
       float part[NGK];
 #pragma unroll
       for (int j = 0; j < NGK; ++j) part[j] = 0.f;
+      float qv[NR][4];
+      float amax = 0.f;
       const uint16_t* qrow = q + ((size_t)b * g.Hq + (size_t)h * G + gid) * D;
 #pragma unroll
-      for (int s = 0; s < KSTEPS; ++s) {
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          uint32_t v = 0;
-          if (gid < G) {
-            uint32_t raw = *reinterpret_cast<const uint32_t*>(qrow + 16 * s + 2 * tid + 8 * hh);
-            float f0 = bits16_to_f32((uint16_t)(raw & 0xFFFF), g.in_dtype);
-            float f1 = bits16_to_f32((uint16_t)(raw >> 16), g.in_dtype);
-            v = pack_h2(f0, f1);
-            __half2 hv = as_h2(v);
-            part[s / (KSTEPS / NGK)] += __low2float(hv) + __high2float(hv);
-          }
-          qf[2 * s + hh] = v;
+      for (int r = 0; r < NR; ++r) {
+        uint2 raw = make_uint2(0u, 0u);
+        if (gid < G) raw = *reinterpret_cast<const uint2*>(qrow + 16 * r + 4 * tid);
+        float f[4];
+        f[0] = bits16_to_f32((uint16_t)(raw.x & 0xFFFF), g.in_dtype);
+        f[1] = bits16_to_f32((uint16_t)(raw.x >> 16), g.in_dtype);
+        f[2] = bits16_to_f32((uint16_t)(raw.y & 0xFFFF), g.in_dtype);
+        f[3] = bits16_to_f32((uint16_t)(raw.y >> 16), g.in_dtype);
+        if constexpr (KAXIS == 1) {
+          // the tensor core sees q rounded to fp16: keep the sums consistent with that
+          qf[2 * r] = pack_h2(f[0], f[2]);
+          qf[2 * r + 1] = pack_h2(f[1], f[3]);
+          const float2 a = __half22float2(as_h2(qf[2 * r])), bb = __half22float2(as_h2(qf[2 * r + 1]));
+          f[0] = a.x; f[2] = a.y; f[1] = bb.x; f[3] = bb.y;
         }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          qv[r][j] = f[j];
+          amax = fmaxf(amax, fabsf(f[j]));
+          part[r / (NR / NGK)] += f[j];
+        }
+      }
+      if constexpr (KAXIS == 0) {
+        // per head: 22-bit fixed point relative to the head's largest entry, Q = rint(q * 2^k) with
+        // |Q| < 2^22, split into three balanced signed bytes  Q = l0 * 65536 + l1 * 256 + l2
+        static_assert(NL == 3, "three signed 8-bit limbs");
+        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 2));
+        int e = (int)((__float_as_uint(amax) >> 23) & 0xFF) - 127;
+        e = max(e, -60);
+        const int k = 21 - e;
+        const float scale = __uint_as_float((uint32_t)(127 + k) << 23);
+        const float hs = c1 * __uint_as_float((uint32_t)(127 - k) << 23);
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+          uint32_t w0 = 0, w1 = 0, w2 = 0;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int Q = __float2int_rn(qv[r][j] * scale);
+            const int b2 = (int)(int8_t)(Q & 0xFF);
+            const int Q1 = (Q - b2) >> 8;
+            const int b1 = (int)(int8_t)(Q1 & 0xFF);
+            const int b0 = (Q1 - b1) >> 8;
+            w0 |= (uint32_t)(b0 & 0xFF) << (8 * j);
+            w1 |= (uint32_t)(b1 & 0xFF) << (8 * j);
+            w2 |= (uint32_t)(b2 & 0xFF) << (8 * j);
+          }
+          ql[0][r] = w0; ql[1][r] = w1; ql[2][r] = w2;
+        }
+        hs0 = __shfl_sync(FULL, hs, (2 * tid) * 4);
+        hs1 = __shfl_sync(FULL, hs, (2 * tid + 1) * 4);
       }
 #pragma unroll
       for (int j = 0; j < NGK; ++j) {
@@ -230,23 +279,20 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         const int ntiles = (nv + 15) >> 4;
 
         // ---- channel-wise keys: per page, fold the channel scales into q and get sum_d q_d z_d by one more mma
-        uint32_t qs[(KAXIS == 1) ? 2 * KSTEPS : 1];
+        uint32_t qs[(KAXIS == 1) ? 2 * NR : 1];
         float zq0 = 0.f, zq1 = 0.f;
         if constexpr (KAXIS == 1) {
           if (!tail_k) {
             const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
             float sz[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int s = 0; s < KSTEPS; ++s) {
-              uint32_t zf[2];
-#pragma unroll
-              for (int hh = 0; hh < 2; ++hh) {
-                uint2 mm = *reinterpret_cast<const uint2*>(km + 16 * s + 2 * tid + 8 * hh);
-                uint32_t sc2 = __byte_perm(mm.x, mm.y, 0x5410);
-                zf[hh] = __byte_perm(mm.x, mm.y, 0x7632);
-                qs[2 * s + hh] = as_u32(__hmul2(as_h2(qf[2 * s + hh]), as_h2(sc2)));
-              }
-              mma16816(sz, zf[0], zf[0], zf[1], zf[1], qf[2 * s], qf[2 * s + 1]);
+            for (int r = 0; r < NR; ++r) {
+              const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);   // (s,z) of 4 channels
+              const uint32_t s02 = __byte_perm(mm.x, mm.z, 0x5410), s13 = __byte_perm(mm.y, mm.w, 0x5410);
+              const uint32_t z02 = __byte_perm(mm.x, mm.z, 0x7632), z13 = __byte_perm(mm.y, mm.w, 0x7632);
+              qs[2 * r] = as_u32(__hmul2(as_h2(qf[2 * r]), as_h2(s02)));
+              qs[2 * r + 1] = as_u32(__hmul2(as_h2(qf[2 * r + 1]), as_h2(s13)));
+              mma16816(sz, z02, z02, z13, z13, qf[2 * r], qf[2 * r + 1]);
             }
             zq0 = c1 * sz[0];
             zq1 = c1 * sz[1];
@@ -261,58 +307,72 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           float L[4];
 
           // ---------------- logits
-          if (KAXIS == 1 && tail_k) {
-            const uint16_t* tl = c.k_tail + ((size_t)stream * kPageTokens + tok0) * D;
-            float S[4] = {0.f, 0.f, 0.f, 0.f};
+          if constexpr (KAXIS == 1) {
+            float S[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // two chains, summed below
+            if (tail_k) {
+              const uint16_t* tl = c.k_tail + ((size_t)stream * kPageTokens + tok0) * D;
 #pragma unroll
-            for (int s = 0; s < KSTEPS; ++s) {
-              const int col = 16 * s + 2 * tid;
-              uint32_t a0 = v0 ? *reinterpret_cast<const uint32_t*>(tl + col) : 0u;
-              uint32_t a1 = v1 ? *reinterpret_cast<const uint32_t*>(tl + 8 * D + col) : 0u;
-              uint32_t a2 = v0 ? *reinterpret_cast<const uint32_t*>(tl + col + 8) : 0u;
-              uint32_t a3 = v1 ? *reinterpret_cast<const uint32_t*>(tl + 8 * D + col + 8) : 0u;
-              mma16816(S, a0, a1, a2, a3, qf[2 * s], qf[2 * s + 1]);
+              for (int r = 0; r < NR; ++r) {
+                uint2 ra = make_uint2(0u, 0u), rb = make_uint2(0u, 0u);
+                if (v0) ra = *reinterpret_cast<const uint2*>(tl + 16 * r + 4 * tid);
+                if (v1) rb = *reinterpret_cast<const uint2*>(tl + 8 * D + 16 * r + 4 * tid);
+                mma16816(S[r & 1], __byte_perm(ra.x, ra.y, 0x5410), __byte_perm(rb.x, rb.y, 0x5410),
+                         __byte_perm(ra.x, ra.y, 0x7632), __byte_perm(rb.x, rb.y, 0x7632), qf[2 * r], qf[2 * r + 1]);
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i) L[i] = c1 * (S[0][i] + S[1][i]);
+            } else {
+              uint32_t ka[KW], kb2[KW];
+              const uint8_t* krow = sp + (size_t)tok0 * K_ROW_BYTES;
+              load_chunk<KW>(krow, tid, 4, ka);
+              load_chunk<KW>(krow + 8 * K_ROW_BYTES, tid, 4, kb2);
+#pragma unroll
+              for (int w = 0; w < KW; ++w) {
+                uint32_t pa[Unpack<KB>::PPW], pb[Unpack<KB>::PPW];
+                Unpack<KB>::run(ka[w], pa);
+                Unpack<KB>::run(kb2[w], pb);
+#pragma unroll
+                for (int i = 0; i < FPB; ++i) {
+                  const int r = w * FPB + i;       // pairs (j = 0, 2) sit in output i, (j = 1, 3) in output FPB + i
+                  mma16816(S[r & 1], pa[i], pb[i], pa[FPB + i], pb[FPB + i], qs[2 * r], qs[2 * r + 1]);
+                }
+              }
+              L[0] = fmaf(c1, S[0][0] + S[1][0], zq0); L[1] = fmaf(c1, S[0][1] + S[1][1], zq1);
+              L[2] = fmaf(c1, S[0][2] + S[1][2], zq0); L[3] = fmaf(c1, S[0][3] + S[1][3], zq1);
             }
-#pragma unroll
-            for (int r = 0; r < 4; ++r) L[r] = c1 * S[r];
           } else {
             uint32_t ka[KW], kb2[KW];
             const uint8_t* krow = sp + (size_t)tok0 * K_ROW_BYTES;
             load_chunk<KW>(krow, tid, 4, ka);
             load_chunk<KW>(krow + 8 * K_ROW_BYTES, tid, 4, kb2);
-            float S[NGK][4];
+            int S[NGK][NL][4];
 #pragma unroll
-            for (int j = 0; j < NGK; ++j) { S[j][0] = S[j][1] = S[j][2] = S[j][3] = 0.f; }
+            for (int j = 0; j < NGK; ++j) {
 #pragma unroll
-            for (int w = 0; w < KW; ++w) {
-              uint32_t pa[KPPW], pb[KPPW];
-              Unpack<KB>::run(ka[w], pa);
-              Unpack<KB>::run(kb2[w], pb);
-#pragma unroll
-              for (int i = 0; i < KPPW; i += 2) {
-                const int s = (w * KPPW + i) / 2;
-                if constexpr (KAXIS == 1)
-                  mma16816(S[0], pa[i], pb[i], pa[i + 1], pb[i + 1], qs[2 * s], qs[2 * s + 1]);
-                else
-                  mma16816(S[s / (KSTEPS / NGK)], pa[i], pb[i], pa[i + 1], pb[i + 1], qf[2 * s], qf[2 * s + 1]);
-              }
+              for (int l = 0; l < NL; ++l) { S[j][l][0] = S[j][l][1] = S[j][l][2] = S[j][l][3] = 0; }
             }
-            if constexpr (KAXIS == 1) {
-              L[0] = fmaf(c1, S[0][0], zq0); L[1] = fmaf(c1, S[0][1], zq1);
-              L[2] = fmaf(c1, S[0][2], zq0); L[3] = fmaf(c1, S[0][3], zq1);
-            } else {
-              const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
-              L[0] = L[1] = L[2] = L[3] = 0.f;
 #pragma unroll
-              for (int j = 0; j < NGK; ++j) {
-                const float2 ma = __half22float2(as_h2(km[tok0 * NGK + j]));          // (scale, zero)
-                const float2 mb = __half22float2(as_h2(km[(tok0 + 8) * NGK + j]));
-                const float sa = c1 * ma.x, sb = c1 * mb.x;
-                L[0] += fmaf(sa, S[j][0], ma.y * qsum[0][j]);
-                L[1] += fmaf(sa, S[j][1], ma.y * qsum[1][j]);
-                L[2] += fmaf(sb, S[j][2], mb.y * qsum[0][j]);
-                L[3] += fmaf(sb, S[j][3], mb.y * qsum[1][j]);
-              }
+            for (int s = 0; s < KS32; ++s) {
+              const int j = s / (KS32 / NGK);
+              const uint32_t a0 = key_slot<KB, KW>(ka, 2 * s), a1 = key_slot<KB, KW>(kb2, 2 * s);
+              const uint32_t a2 = key_slot<KB, KW>(ka, 2 * s + 1), a3 = key_slot<KB, KW>(kb2, 2 * s + 1);
+#pragma unroll
+              for (int l = 0; l < NL; ++l) mma16832_u8s8(S[j][l], a0, a1, a2, a3, ql[l][2 * s], ql[l][2 * s + 1]);
+            }
+            const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
+            L[0] = L[1] = L[2] = L[3] = 0.f;
+#pragma unroll
+            for (int j = 0; j < NGK; ++j) {
+              float t[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i)       // sum_d code_d * Q_d = (S0 * 256 + S1) * 256 + S2, exact up to the last step
+                t[i] = fmaf((float)(S[j][0][i] * 256 + S[j][1][i]), 256.f, (float)S[j][2][i]);
+              const float2 ma = __half22float2(as_h2(km[tok0 * NGK + j]));          // (scale, zero)
+              const float2 mb = __half22float2(as_h2(km[(tok0 + 8) * NGK + j]));
+              L[0] += fmaf(ma.x * hs0, t[0], ma.y * qsum[0][j]);
+              L[1] += fmaf(ma.x * hs1, t[1], ma.y * qsum[1][j]);
+              L[2] += fmaf(mb.x * hs0, t[2], mb.y * qsum[0][j]);
+              L[3] += fmaf(mb.x * hs1, t[3], mb.y * qsum[1][j]);
             }
           }
           if (MASKED) {
@@ -476,7 +536,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 }
 
 // Launches one instantiation; defined per instantiation unit.
-template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NW, int MINB>
+template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NL, int NW, int MINB>
 int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap,
                     cudaStream_t stream) {
   const int budget = (227 * 1024) / MINB - 1024;            // shared memory per CTA for MINB resident CTAs per SM
@@ -484,7 +544,7 @@ int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, 
   if (stages > 8) stages = 8;
   if (stages < 2) return KVQ_ERR_UNSUPPORTED;
   const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D);
-  auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NW, MINB>;
+  auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
     return KVQ_ERR_CUDA_LAUNCH;
   kern<<<148 * MINB, (NW + 1) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap,

@@ -14,7 +14,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libkvq.so")
+LIB_PATH = os.environ.get("KVQ_LIB_PATH") or os.path.join(_HERE, "libkvq.so")   # override: load another build
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2502_15075_b200.build` "

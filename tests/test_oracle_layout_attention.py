@@ -70,19 +70,24 @@ def test_pack_unpack_roundtrip_and_sizes(D, kb, vb, gk, gv, k_axis):
 
 def test_single_field_encoding_is_little_endian_words():
     """Spot values of the index function worked out by hand from its definition."""
-    # K, D=128, 4-bit: d=0 -> chunk 0, P 0, word 0, field 0 -> byte 0 low nibble
+    # K, D=128, 4-bit (2 fields per byte): d=0 -> chunk 0, r 0, word 0, byte 0 low nibble
     assert ol.k_code_pos(0, 0, 128, 4) == (0, 0)
-    # d=1 (odd): field 0 + ppw(4) = 4 -> bit 16 -> byte 2, shift 0
-    assert ol.k_code_pos(0, 1, 128, 4) == (2, 0)
-    # d=8: P=1 -> field 1 -> bit 4 -> byte 0, shift 4
-    assert ol.k_code_pos(0, 8, 128, 4) == (0, 4)
-    # d=2: chunk 1 -> byte 16
-    assert ol.k_code_pos(0, 2, 128, 4) == (16, 0)
-    # d=16: P=2 -> field 2 -> bit 8 -> byte 1 ; d=32: P=4 -> word 1 -> byte 4
-    assert ol.k_code_pos(0, 16, 128, 4) == (1, 0)
+    # d=1..3 are the next bytes of the same word; d=4 starts chunk 1 (16 bytes further)
+    assert ol.k_code_pos(0, 1, 128, 4) == (1, 0)
+    assert ol.k_code_pos(0, 3, 128, 4) == (3, 0)
+    assert ol.k_code_pos(0, 4, 128, 4) == (16, 0)
+    assert ol.k_code_pos(0, 8, 128, 4) == (32, 0)
+    # d=16: r=1 -> same word, high nibble of byte 0 ; d=32: r=2 -> word 1 -> byte 4
+    assert ol.k_code_pos(0, 16, 128, 4) == (0, 4)
+    assert ol.k_code_pos(0, 17, 128, 4) == (1, 4)
     assert ol.k_code_pos(0, 32, 128, 4) == (4, 0)
     # token stride = 64 bytes
     assert ol.k_code_pos(3, 0, 128, 4) == (192, 0)
+    # 2-bit: four fields per byte: d=16,32,48 share byte 0 at shifts 2,4,6; d=64 -> word 1
+    assert ol.k_code_pos(0, 16, 128, 2) == (0, 2)
+    assert ol.k_code_pos(0, 48, 128, 2) == (0, 6)
+    assert ol.k_code_pos(0, 64, 128, 2) == (4, 0)
+    assert ol.k_code_pos(0, 4, 128, 2) == (8, 0)
     # V, D=128, 2-bit: (t=0,d=0) byte 0; t=1 (odd token): field 8 -> bit 16 -> byte 2
     assert ol.v_code_pos(0, 0, 128, 2) == (0, 0)
     assert ol.v_code_pos(1, 0, 128, 2) == (2, 0)
@@ -97,12 +102,13 @@ def test_single_field_encoding_is_little_endian_words():
     # next tile of 16 tokens: 16*128*2/8 = 512 bytes further
     assert ol.v_code_pos(16, 0, 128, 2) == (512, 0)
     # quad-major word placement when a chunk has more than 4 words:
-    # K, D=128, 8-bit (8 words per chunk): d=2 -> chunk 1 -> byte 16; d=64 -> P=8 -> word 4 -> second quad
-    # -> byte 4 chunks * 16 = 64; d=66 -> 64 + 16; d=1 -> field 0 + ppw(2) = 2 -> byte 2
-    assert ol.k_code_pos(0, 2, 128, 8) == (16, 0)
+    # K, D=128, 8-bit (one field per byte, 8 words per chunk): d=2 -> byte 2; d=4 -> chunk 1 -> byte 16;
+    # d=16 -> word 1 -> byte 4; d=64 -> word 4 -> second quad -> byte 4 chunks * 16 = 64; d=68 -> 64 + 16
+    assert ol.k_code_pos(0, 2, 128, 8) == (2, 0)
+    assert ol.k_code_pos(0, 4, 128, 8) == (16, 0)
+    assert ol.k_code_pos(0, 16, 128, 8) == (4, 0)
     assert ol.k_code_pos(0, 64, 128, 8) == (64, 0)
-    assert ol.k_code_pos(0, 66, 128, 8) == (80, 0)
-    assert ol.k_code_pos(0, 1, 128, 8) == (2, 0)
+    assert ol.k_code_pos(0, 68, 128, 8) == (80, 0)
     assert ol.k_code_pos(1, 0, 128, 8) == (128, 0)
     # V, D=128, 4-bit (8 words per chunk): d=64 -> P=16 -> word 4 -> second quad -> byte 32 chunks * 16 = 512
     assert ol.v_code_pos(0, 64, 128, 4) == (512, 0)
