@@ -1,5 +1,11 @@
 // kvq_dequantize kernel: x^ = fmaf(code, scale, zero) rounded to the 16-bit
 // input type (App. B.1: A^ = scale * Q, here with the group minimum as offset).
+//
+// One CTA per (page, stream): the packed page is copied to shared memory, each
+// thread expands whole 32-bit words of codes (no per-element index arithmetic)
+// into a [128][D] 16-bit tile in shared memory, and the tile's valid token rows
+// go out with 16-byte coalesced stores.  The kernel is bound by those stores
+// (it writes 4-8x what it reads).
 #include "kvq_internal.h"
 
 namespace kvq {
@@ -8,10 +14,87 @@ namespace {
 
 constexpr int kThreads = 256;
 
+// All sizes that index arithmetic divides by are powers of two: use shifts.
+__device__ __forceinline__ int ilog2(int x) { return 31 - __clz(x); }
+
+__device__ __forceinline__ float meta_scale(uint32_t m) { return __half2float(__ushort_as_half((uint16_t)(m & 0xFFFF))); }
+__device__ __forceinline__ float meta_zero(uint32_t m) { return __half2float(__ushort_as_half((uint16_t)(m >> 16))); }
+
+// Expand the key codes of a page into tile[t][d] (16-bit patterns of dtype).
+template <int B>
+__device__ __forceinline__ void expand_keys(const uint8_t* spage, const Geom& g, uint16_t* tile, int tid) {
+  const int D = g.D;
+  constexpr int FPB = 8 / B;
+  const int wpr = D * B / 32;          // words per token row
+  const int wpc = wpr / 4;             // words per chunk
+  const uint32_t* meta = reinterpret_cast<const uint32_t*>(spage + g.k_meta_off);
+  const int lgk = ilog2(g.gk), ngk = D >> lgk;
+  const int lwpr = ilog2(wpr), lwpc = ilog2(wpc);
+  for (int idx = tid; idx < kPageTokens * wpr; idx += kThreads) {
+    const int t = idx >> lwpr, wi = idx & (wpr - 1);
+    const int chunk = wi >> lwpc, word = wi & (wpc - 1);
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(spage + (size_t)t * (D * B / 8) +
+                                                           chunk_word_byte(chunk, word, wpc, 4));
+#pragma unroll
+    for (int i = 0; i < FPB; ++i) {
+      const int d0 = 16 * (word * FPB + i) + 4 * chunk;           // bytes j = 0..3 hold channels d0 + j
+      uint16_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float code = (float)((w >> (8 * j + B * i)) & ((1u << B) - 1u));
+        const uint32_t m = meta[g.k_axis == 1 ? d0 + j : t * ngk + ((d0 + j) >> lgk)];
+        o[j] = f32_to_bits16(fmaf(code, meta_scale(m), meta_zero(m)), g.in_dtype);
+      }
+      *reinterpret_cast<uint2*>(tile + t * D + d0) =
+          make_uint2((uint32_t)o[0] | ((uint32_t)o[1] << 16), (uint32_t)o[2] | ((uint32_t)o[3] << 16));
+    }
+  }
+}
+
+// Expand the value codes of a page into tile[t][d].
+template <int B>
+__device__ __forceinline__ void expand_values(const uint8_t* spage, const Geom& g, uint16_t* tile, int tid) {
+  const int D = g.D;
+  constexpr int NF = 32 / B;
+  const int wpt = D * B / 2;           // words per 16-token tile
+  const int wpc = D * B / 64;          // words per chunk
+  const uint8_t* codes = spage + g.v_codes_off;
+  const uint32_t* meta = reinterpret_cast<const uint32_t*>(spage + g.v_meta_off);
+  const int lgv = ilog2(g.gv), ngv = D >> lgv;
+  const int lwpt = ilog2(wpt), lwpc = ilog2(wpc);
+  for (int idx = tid; idx < 8 * wpt; idx += kThreads) {
+    const int vt = idx >> lwpt, wi = idx & (wpt - 1);
+    const int chunk = wi >> lwpc, word = wi & (wpc - 1);
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(codes + (size_t)vt * (16 * D * B / 8) +
+                                                           chunk_word_byte(chunk, word, wpc, 32));
+#pragma unroll
+    for (int f = 0; f < NF; ++f) {
+      int tau, d;
+      v_field_pos(chunk, word, f, B, tau, d);
+      const int t = vt * 16 + tau;
+      const uint32_t m = meta[t * ngv + (d >> lgv)];
+      const float code = (float)((w >> (f * B)) & ((1u << B) - 1u));
+      tile[t * D + d] = f32_to_bits16(fmaf(code, meta_scale(m), meta_zero(m)), g.in_dtype);
+    }
+  }
+}
+
+// Copy token rows [lo, hi) of tile[128][D] to out rows (16-byte vectors).
+__device__ __forceinline__ void store_rows(const uint16_t* tile, uint16_t* out, int D, int lo, int hi, int tid) {
+  const int vpr = D / 8, lv = ilog2(vpr);
+  for (int idx = tid; idx < (hi - lo) * vpr; idx += kThreads) {
+    const int t = lo + (idx >> lv), v = idx & (vpr - 1);
+    reinterpret_cast<uint4*>(out + (size_t)t * D)[v] = reinterpret_cast<const uint4*>(tile + t * D)[v];
+  }
+}
+
 __global__ void __launch_bounds__(kThreads)
 dequant_kernel(Geom g, CachePtrs c, uint16_t* __restrict__ k_out, uint16_t* __restrict__ v_out,
                int t_begin, int t_end, int page0) {
-  extern __shared__ __align__(16) uint8_t spage[];
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int D = g.D, tid = threadIdx.x;
+  uint8_t* spage = smem;
+  uint16_t* tile = reinterpret_cast<uint16_t*>(smem + ((g.page_bytes + 15) & ~15));   // [128][D]
   const int bh = blockIdx.y;
   const int b = bh / g.Hkv;
   const int n = c.seq_len[b];
@@ -20,51 +103,45 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* __restrict__ k_out, uint16_t* __re
   const int lo_t = max(t_begin, page * kPageTokens), hi_t = min(hi, page * kPageTokens + kPageTokens);
   if (lo_t >= hi_t) return;
   const int nv = min(kPageTokens, n - page * kPageTokens);
-  const int D = g.D, tid = threadIdx.x;
   const uint8_t* pg = c.pages + ((size_t)bh * g.n_pages + page) * g.page_bytes;
   for (int i = tid; i < g.page_bytes / 16; i += kThreads)
     reinterpret_cast<uint4*>(spage)[i] = reinterpret_cast<const uint4*>(pg)[i];
   __syncthreads();
-  const bool tail_k = (g.k_axis == 1) && (nv < kPageTokens);
-  const uint16_t* tail = tail_k ? c.k_tail + (size_t)bh * kPageTokens * D : nullptr;
-  const size_t out_base = (size_t)bh * g.capacity * D;
+  const int lo = lo_t - page * kPageTokens, hi_l = hi_t - page * kPageTokens;
+  const size_t out_base = ((size_t)bh * g.capacity + (size_t)page * kPageTokens) * D;
 
-  for (int idx = tid; idx < (hi_t - lo_t) * D; idx += kThreads) {
-    const int t = lo_t + idx / D, d = idx % D;
-    const int tp = t - page * kPageTokens;
-    if (v_out) {
-      uint16_t r;
-      if (g.vb == 16) {
-        r = reinterpret_cast<const uint16_t*>(spage + g.v_codes_off)[tp * D + d];
-      } else {
-        int wb, bit;
-        v_code_pos(tp, d, D, g.vb, wb, bit);
-        float code = (float)load_code(spage + g.v_codes_off, wb, bit, g.vb);
-        uint32_t m = reinterpret_cast<const uint32_t*>(spage + g.v_meta_off)[tp * (D / g.gv) + d / g.gv];
-        float s = __half2float(__ushort_as_half((uint16_t)(m & 0xFFFF)));
-        float z = __half2float(__ushort_as_half((uint16_t)(m >> 16)));
-        r = f32_to_bits16(fmaf(code, s, z), g.in_dtype);
-      }
-      v_out[out_base + (size_t)t * D + d] = r;
+  if (v_out) {
+    if (g.vb == 16) {
+      store_rows(reinterpret_cast<const uint16_t*>(spage + g.v_codes_off), v_out + out_base, D, lo, hi_l, tid);
+    } else {
+      if (g.vb == 2) expand_values<2>(spage, g, tile, tid);
+      else if (g.vb == 4) expand_values<4>(spage, g, tile, tid);
+      else expand_values<8>(spage, g, tile, tid);
+      __syncthreads();
+      store_rows(tile, v_out + out_base, D, lo, hi_l, tid);
     }
-    if (k_out) {
-      uint16_t r;
-      if (tail_k) {
-        uint16_t hbits = tail[tp * D + d];
-        r = (g.in_dtype == KVQ_FP16) ? hbits : f32_to_bits16(bits16_to_f32(hbits, KVQ_FP16), KVQ_BF16);
-      } else if (g.kb == 16) {
-        r = reinterpret_cast<const uint16_t*>(spage)[tp * D + d];
-      } else {
-        int wb, bit;
-        k_code_pos(tp, d, D, g.kb, wb, bit);
-        float code = (float)load_code(spage, wb, bit, g.kb);
-        int mi = (g.k_axis == 1) ? d : tp * (D / g.gk) + d / g.gk;
-        uint32_t m = reinterpret_cast<const uint32_t*>(spage + g.k_meta_off)[mi];
-        float s = __half2float(__ushort_as_half((uint16_t)(m & 0xFFFF)));
-        float z = __half2float(__ushort_as_half((uint16_t)(m >> 16)));
-        r = f32_to_bits16(fmaf(code, s, z), g.in_dtype);
+  }
+  if (k_out) {
+    const bool tail_k = (g.k_axis == 1) && (nv < kPageTokens);
+    if (tail_k) {
+      // keys of an incomplete channel-wise block live in the fp16 tail
+      const uint16_t* tail = c.k_tail + (size_t)bh * kPageTokens * D;
+      const int lD = ilog2(D);
+      for (int idx = tid; idx < (hi_l - lo) * D; idx += kThreads) {
+        const int t = lo + (idx >> lD), d = idx & (D - 1);
+        const uint16_t hbits = tail[t * D + d];
+        k_out[out_base + (size_t)t * D + d] =
+            (g.in_dtype == KVQ_FP16) ? hbits : f32_to_bits16(bits16_to_f32(hbits, KVQ_FP16), KVQ_BF16);
       }
-      k_out[out_base + (size_t)t * D + d] = r;
+    } else if (g.kb == 16) {
+      store_rows(reinterpret_cast<const uint16_t*>(spage), k_out + out_base, D, lo, hi_l, tid);
+    } else {
+      __syncthreads();          // the value tile has been copied out
+      if (g.kb == 2) expand_keys<2>(spage, g, tile, tid);
+      else if (g.kb == 4) expand_keys<4>(spage, g, tile, tid);
+      else expand_keys<8>(spage, g, tile, tid);
+      __syncthreads();
+      store_rows(tile, k_out + out_base, D, lo, hi_l, tid);
     }
   }
 }
@@ -76,10 +153,11 @@ int launch_dequantize(const Geom& g, const CachePtrs& c, void* k_out, void* v_ou
   if (t_end <= t_begin) return KVQ_OK;
   const int page0 = t_begin / kPageTokens;
   const int page1 = (t_end + kPageTokens - 1) / kPageTokens;
-  cudaFuncSetAttribute(dequant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 4);
+  const size_t smem = (size_t)((g.page_bytes + 15) & ~15) + (size_t)kPageTokens * g.D * 2;
+  cudaFuncSetAttribute(dequant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 4 + 128 * 128 * 2);
   dim3 grid(page1 - page0, g.B * g.Hkv);
-  dequant_kernel<<<grid, kThreads, g.page_bytes, stream>>>(g, c, static_cast<uint16_t*>(k_out),
-                                                           static_cast<uint16_t*>(v_out), t_begin, t_end, page0);
+  dequant_kernel<<<grid, kThreads, smem, stream>>>(g, c, static_cast<uint16_t*>(k_out),
+                                                   static_cast<uint16_t*>(v_out), t_begin, t_end, page0);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
 
