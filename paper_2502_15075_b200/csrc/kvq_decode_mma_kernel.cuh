@@ -64,6 +64,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   constexpr int K_ROW_BYTES = D * KB / 8;
   constexpr int V_TILE_BYTES = 16 * D * VB / 8;
   constexpr int NCONS = NW * 32;
+  constexpr int TPW = (kPageTokens / 16) / NW;   // tiles per warp per page
   constexpr uint32_t FULL = 0xffffffffu;
   static_assert(KAXIS == 0 || KB != 2, "channel-wise 2-bit keys are not instantiated");
 
@@ -299,14 +300,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           }
         }
 
-        // One 16-token tile: logits -> online softmax -> PV.  MASKED handles a partially filled page.
-        auto do_tile = [&](const int tile, auto masked_tag) {
-          constexpr bool MASKED = decltype(masked_tag)::value;
-          const int tok0 = tile * 16 + gid;            // page-local tokens of this lane's two rows
-          const bool v0 = !MASKED || tok0 < nv, v1 = !MASKED || tok0 + 8 < nv;
-          float L[4];
-
-          // ---------------- logits
+        // The TPW tiles this warp owns in the page (tile = warp + NW * u) are processed together: logits of all
+        // of them, one joint running-max check, then probabilities and PV.  MASKED handles a partial page.
+        auto logits = [&](const int tok0, const bool v0, const bool v1, float (&L)[4]) {
           if constexpr (KAXIS == 1) {
             float S[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // two chains, summed below
             if (tail_k) {
@@ -375,36 +371,12 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               L[3] += fmaf(mb.x * hs1, t[3], mb.y * qsum[1][j]);
             }
           }
-          if (MASKED) {
-            if (!v0) { L[0] = -INFINITY; L[1] = -INFINITY; }
-            if (!v1) { L[2] = -INFINITY; L[3] = -INFINITY; }
-          }
+          if (!v0) { L[0] = -INFINITY; L[1] = -INFINITY; }
+          if (!v1) { L[2] = -INFINITY; L[3] = -INFINITY; }
+        };
 
-          // ---------------- online softmax (rescale only when some logit exceeds the running max)
-          const float t0 = fmaxf(L[0], L[2]), t1 = fmaxf(L[1], L[3]);
-          if (__any_sync(FULL, (t0 > m0) | (t1 > m1))) {
-            float u0 = t0, u1 = t1;
-#pragma unroll
-            for (int off = 4; off < 32; off <<= 1) {
-              u0 = fmaxf(u0, __shfl_xor_sync(FULL, u0, off));
-              u1 = fmaxf(u1, __shfl_xor_sync(FULL, u1, off));
-            }
-            const float n0 = fmaxf(m0, u0), n1 = fmaxf(m1, u1);
-            const float a0 = (n0 == -INFINITY) ? 1.f : ex2(m0 - n0);
-            const float a1 = (n1 == -INFINITY) ? 1.f : ex2(m1 - n1);
-            m0 = n0; m1 = n1;
-            l0 *= a0; l1 *= a1;
-#pragma unroll
-            for (int j = 0; j < NGV; ++j) { zacc[0][j] *= a0; zacc[1][j] *= a1; }
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) { O[mt][0] *= a0; O[mt][1] *= a1; O[mt][2] *= a0; O[mt][3] *= a1; }
-          }
-          float p[4];
-          p[0] = ex2(L[0] - m0); p[1] = ex2(L[1] - m1); p[2] = ex2(L[2] - m0); p[3] = ex2(L[3] - m1);
-          l0 += p[0] + p[2];
-          l1 += p[1] + p[3];
-
-          // ---------------- values: fold the scale into p, keep the zero-point term as a scalar per group
+        // values of one tile: fold the scale into p, keep the zero-point term as a scalar per group
+        auto values = [&](const int tile, const int tok0, const bool v0, const bool v1, const float (&p)[4]) {
           const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + g.v_meta_off);
           const uint32_t pa01 = pack_h2(p[0], p[1]), pb01 = pack_h2(p[2], p[3]);
           uint32_t bw[NGV][2];
@@ -437,12 +409,57 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           }
         };
 
-        if (nv == kPageTokens) {
-#pragma unroll 1
-          for (int tile = warp; tile < kPageTokens / 16; tile += NW) do_tile(tile, std::false_type{});
-        } else {
-#pragma unroll 1
-          for (int tile = warp; tile < ntiles; tile += NW) do_tile(tile, std::true_type{});
+        auto do_tiles = [&](auto masked_tag) {
+          constexpr bool MASKED = decltype(masked_tag)::value;
+          float L[TPW][4];
+          bool v0[TPW], v1[TPW];
+          float t0 = -INFINITY, t1 = -INFINITY;
+#pragma unroll
+          for (int u = 0; u < TPW; ++u) {
+            const int tok0 = (warp + NW * u) * 16 + gid;        // page-local tokens of this lane's two rows
+            v0[u] = !MASKED || tok0 < nv;
+            v1[u] = !MASKED || tok0 + 8 < nv;
+            if (!MASKED || (warp + NW * u) < ntiles) {
+              logits(tok0, v0[u], v1[u], L[u]);
+            } else {
+              L[u][0] = L[u][1] = L[u][2] = L[u][3] = -INFINITY;
+            }
+            t0 = fmaxf(t0, fmaxf(L[u][0], L[u][2]));
+            t1 = fmaxf(t1, fmaxf(L[u][1], L[u][3]));
+          }
+          // online softmax: rescale only when some logit exceeds the running max
+          if (__any_sync(FULL, (t0 > m0) | (t1 > m1))) {
+            float u0 = t0, u1 = t1;
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+              u0 = fmaxf(u0, __shfl_xor_sync(FULL, u0, off));
+              u1 = fmaxf(u1, __shfl_xor_sync(FULL, u1, off));
+            }
+            const float n0 = fmaxf(m0, u0), n1 = fmaxf(m1, u1);
+            const float a0 = (n0 == -INFINITY) ? 1.f : ex2(m0 - n0);
+            const float a1 = (n1 == -INFINITY) ? 1.f : ex2(m1 - n1);
+            m0 = n0; m1 = n1;
+            l0 *= a0; l1 *= a1;
+#pragma unroll
+            for (int j = 0; j < NGV; ++j) { zacc[0][j] *= a0; zacc[1][j] *= a1; }
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) { O[mt][0] *= a0; O[mt][1] *= a1; O[mt][2] *= a0; O[mt][3] *= a1; }
+          }
+#pragma unroll
+          for (int u = 0; u < TPW; ++u) {
+            if (!MASKED || (warp + NW * u) < ntiles) {
+              float p[4];
+              p[0] = ex2(L[u][0] - m0); p[1] = ex2(L[u][1] - m1); p[2] = ex2(L[u][2] - m0); p[3] = ex2(L[u][3] - m1);
+              l0 += p[0] + p[2];
+              l1 += p[1] + p[3];
+              values(warp + NW * u, (warp + NW * u) * 16 + gid, v0[u], v1[u], p);
+            }
+          }
+        };
+
+        if (ntiles > warp) {                     // a short last page may leave this warp without a tile
+          if (nv == kPageTokens) do_tiles(std::false_type{});
+          else do_tiles(std::true_type{});
         }
       }
       __syncwarp();
