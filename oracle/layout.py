@@ -22,9 +22,10 @@ token lives in
 share the word: masking one field out of every byte yields four consecutive
 channels as four bytes).
 V codes (b = vb in {2,4,8}): 8 tiles of 16 tokens, a tile holds 32 chunks of
-wpc = D*b/64 words.  Channel d of token tau (0..15 inside its tile) lives in
-    chunk  = 4*(d % 8) + (tau % 8) // 2
-    P      = 4*(d // 16) + (d % 16) // 8 + 2*(tau // 8)
+wpc = D*b/64 words.  With k = 8*(d // 64) + d % 8, channel d of token tau
+(0..15 inside its tile) lives in
+    chunk  = 4*((d // 8) % 8) + (tau % 8) // 2
+    P      = 4*(k // 2) + k % 2 + 2*(tau // 8)
     word   = P // ppw,  field = P % ppw + ppw*(tau % 2)
 Placement of (chunk, word) inside its row / tile of `nchunks` chunks: words are
 kept in quads of qw = min(wpc, 4) words, quad-major:
@@ -115,8 +116,9 @@ def v_code_pos(t, d, D, b):
     ppw = 16 // b
     tile = t // 16
     tau = t % 16
-    chunk = 4 * (d % 8) + (tau % 8) // 2
-    P = 4 * (d // 16) + (d % 16) // 8 + 2 * (tau // 8)
+    k = 8 * (d // 64) + d % 8
+    chunk = 4 * ((d // 8) % 8) + (tau % 8) // 2
+    P = 4 * (k // 2) + k % 2 + 2 * (tau // 8)
     word = P // ppw
     field = P % ppw + ppw * (tau % 2)
     bit = field * b

@@ -97,8 +97,9 @@ __host__ __device__ __forceinline__ void k_code_pos(int t, int d, int D, int b, 
 __host__ __device__ __forceinline__ void v_code_pos(int t, int d, int D, int b, int& word_byte, int& bit) {
   int ppw = 16 / b;
   int tile = t >> 4, tau = t & 15;
-  int chunk = 4 * (d & 7) + ((tau & 7) >> 1);
-  int P = 4 * (d >> 4) + ((d & 15) >> 3) + 2 * (tau >> 3);
+  int k = 8 * (d >> 6) + (d & 7);
+  int chunk = 4 * ((d >> 3) & 7) + ((tau & 7) >> 1);
+  int P = 4 * (k >> 1) + (k & 1) + 2 * (tau >> 3);
   word_byte = tile * (16 * D * b / 8) + chunk_word_byte(chunk, P / ppw, D * b / 64, 32);
   bit = (P % ppw + ppw * (tau & 1)) * b;
 }
@@ -110,10 +111,11 @@ __device__ __forceinline__ int k_field_channel(int chunk, int word, int f, int b
   return 16 * r + 4 * chunk + (f / fpb);
 }
 
-__device__ __forceinline__ void v_field_pos(int chunk, int word, int f, int b, int& tau, int& d) {
+__device__ __forceinline__ void v_field_pos(int chunk, int word, int f, int b, int D, int& tau, int& d) {
   int ppw = 16 / b;
   int P = word * ppw + (f % ppw);
-  d = 16 * (P >> 2) + 8 * (P & 1) + (chunk >> 2);
+  int k = 2 * (P >> 2) + (P & 1);
+  d = 64 * (k >> 3) + 8 * (chunk >> 2) + (k & 7);
   tau = 8 * ((P & 3) >> 1) + 2 * (chunk & 3) + (f / ppw);
 }
 

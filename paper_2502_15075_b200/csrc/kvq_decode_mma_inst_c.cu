@@ -6,7 +6,6 @@ namespace mma {
 #define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB)                                          \
   template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB>(const Geom&, const CachePtrs&, const void*, \
                                                                          float, float*, int, cudaStream_t);
-KVQ_MMA_DECL(64, 4, 2, 0, 2, 2, 3, 4, 3)
 KVQ_MMA_DECL(64, 4, 2, 0, 1, 1, 3, 4, 3)
 KVQ_MMA_DECL(128, 4, 2, 0, 4, 1, 3, 4, 3)
 #undef KVQ_MMA_DECL

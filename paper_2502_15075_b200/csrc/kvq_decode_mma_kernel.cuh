@@ -529,8 +529,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               if (gid == 0) { dst[0] = e ? m1 : m0; dst[1] = e ? l1 : l0; }
 #pragma unroll
               for (int mt = 0; mt < MT; ++mt) {
-                dst[2 + 16 * mt + gid] = O[mt][e];
-                dst[2 + 16 * mt + gid + 8] = O[mt][2 + e];
+                // accumulator rows (gid, gid + 8) of m-tile mt are channels 64 (mt/4) + 8 gid + 2 (mt%4) + {0, 1}
+                dst[2 + 64 * (mt >> 2) + 8 * gid + 2 * (mt & 3)] = O[mt][e];
+                dst[2 + 64 * (mt >> 2) + 8 * gid + 2 * (mt & 3) + 1] = O[mt][2 + e];
               }
             }
           }

@@ -70,7 +70,7 @@ __device__ __forceinline__ void expand_values(const uint8_t* spage, const Geom& 
 #pragma unroll
     for (int f = 0; f < NF; ++f) {
       int tau, d;
-      v_field_pos(chunk, word, f, B, tau, d);
+      v_field_pos(chunk, word, f, B, D, tau, d);
       const int t = vt * 16 + tau;
       const uint32_t m = meta[t * ngv + (d >> lgv)];
       const float code = (float)((w >> (f * B)) & ((1u << B) - 1u));

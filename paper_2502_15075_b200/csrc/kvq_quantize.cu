@@ -2,6 +2,13 @@
 // quantization (App. B.1 quantizer per group; Sec. 4.1 grouping: token-wise
 // groups along head_dim, or channel-wise groups over a 128-token block with an
 // fp16 residual tail) and packing into the page layout.
+//
+// Token-wise kernel: one warp per 16-token tile of one stream.  Every lane loads
+// 16 bytes (8 consecutive channels of one token), groups reduce min/max with
+// shuffles, the 8 codes of a lane are merged into at most four partial words and
+// OR-ed into an image of the packed tile in shared memory, and the finished image
+// leaves with 16-byte coalesced stores.  The kernel is bound by reading the 16-bit
+// inputs from HBM.
 #include "kvq_internal.h"
 
 namespace kvq {
@@ -9,42 +16,178 @@ namespace kvq {
 namespace {
 
 constexpr int kThreads = 128;
+constexpr int kWarps = kThreads / 32;
+constexpr uint32_t FULL = 0xffffffffu;
 
-// One warp quantizes one token row of D elements (token-wise axis) and leaves
-// the codes as bytes in `codes` (shared memory) and the (scale, zero) words in
-// `meta` (global).  bits == 16: raw copy of the row to `raw_dst`.
-__device__ __forceinline__ void quantize_row_warp(const uint16_t* __restrict__ row, int D, int bits, int gsz,
-                                                  int dtype, uint8_t* codes, uint32_t* meta,
-                                                  uint16_t* raw_dst, int lane) {
-  const int epl = D >> 5;  // elements per lane: 2 (D=64) or 4 (D=128)
-  uint16_t e[4];
-  if (epl == 4) {
-    uint2 v = *reinterpret_cast<const uint2*>(row + lane * 4);
-    e[0] = v.x & 0xFFFF; e[1] = v.x >> 16; e[2] = v.y & 0xFFFF; e[3] = v.y >> 16;
-  } else {
-    uint32_t v = *reinterpret_cast<const uint32_t*>(row + lane * 2);
-    e[0] = v & 0xFFFF; e[1] = v >> 16; e[2] = e[3] = 0;
+// Quantize one side (keys or values) of a 16-token tile held in global memory as rows of D 16-bit values.
+// `img` is the warp's shared-memory image of the packed codes of the tile: for keys 16 token rows of
+// D*BITS/8 bytes, for values the tile's D*BITS*2 bytes.  Tokens outside [lo, hi) are left alone.
+template <int BITS, bool IS_V>
+__device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ src, int64_t st, int D, int gsz,
+                                                   int dtype, int lo, int hi, uint32_t* img,
+                                                   uint32_t* __restrict__ meta_out, bool clear_first, int lane) {
+  const int lpr = D >> 3;                    // lanes per token row (8 channels each)
+  const int rps = 32 / lpr;                  // rows per step
+  const int l = lane & (lpr - 1);
+  const int d0 = l * 8;
+  const int lpg = gsz >> 3;                  // lanes per group
+  const int ng = D / gsz;
+  const float qmax = (float)((1 << BITS) - 1);
+  for (int step = 0; step < 16 / rps; ++step) {
+    const int tau = step * rps + lane / lpr;
+    const bool valid = tau >= lo && tau < hi;
+    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+    if (valid) raw = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + d0);
+    const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+    float x[8];
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[2 * i] = bits16_to_f32((uint16_t)(rw[i] & 0xFFFF), dtype);
+      x[2 * i + 1] = bits16_to_f32((uint16_t)(rw[i] >> 16), dtype);
+      mn = fminf(mn, fminf(x[2 * i], x[2 * i + 1]));
+      mx = fmaxf(mx, fmaxf(x[2 * i], x[2 * i + 1]));
+    }
+    for (int off = 1; off < lpg; off <<= 1) {
+      mn = fminf(mn, __shfl_xor_sync(FULL, mn, off));
+      mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, off));
+    }
+    const GroupParams p = group_params(mn, mx, qmax);
+    if (!valid) continue;
+    if ((l & (lpg - 1)) == 0) meta_out[tau * ng + d0 / gsz] = p.meta;
+    uint32_t code[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) code[i] = code_of(x[i], p, qmax);
+
+    if constexpr (!IS_V) {
+      // keys: channels d0..d0+3 and d0+4..d0+7 are the four bytes of one word each (chunks 2(l%2), 2(l%2)+1),
+      // register slot r = d0/16, field r % fpb of every byte
+      constexpr int FPB = 8 / BITS;
+      const int wpc = D * BITS / 128;
+      const int r = l >> 1;
+      const int sh = BITS * (r % FPB);
+      const int word = r / FPB;
+      const int row_words = D * BITS / 32;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const uint32_t w = (code[4 * hh] | (code[4 * hh + 1] << 8) | (code[4 * hh + 2] << 16) |
+                            (code[4 * hh + 3] << 24)) << sh;
+        const int chunk = 2 * (l & 1) + hh;
+        atomicOr(&img[tau * row_words + chunk_word_byte(chunk, word, wpc, 4) / 4], w);
+      }
+    } else {
+      // values: the lane's 8 channels d0 + kk belong to one lane-chunk group gidc = (d0/8) % 8, k = 8 (d0/64) + kk
+      constexpr int PPW = 16 / BITS;
+      const int wpc = D * BITS / 64;
+      const int gidc = l & 7, h = l >> 3;            // d0 = 64 h + 8 gidc
+      const int tidT = (tau & 7) >> 1, hiT = tau >> 3, oddT = tau & 1;
+      const int chunk = 4 * gidc + tidT;
+      constexpr int NWORD = (BITS == 2) ? 2 : 4;     // words this lane contributes to
+      uint32_t part[NWORD], mask[NWORD];
+      int widx[NWORD];
+#pragma unroll
+      for (int i = 0; i < NWORD; ++i) { part[i] = 0; mask[i] = 0; widx[i] = 0; }
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        const int k = 8 * h + kk;
+        const int P = 4 * (k >> 1) + (k & 1) + 2 * hiT;
+        const int word = P / PPW;
+        const int field = P % PPW + PPW * oddT;
+        const int wo = (BITS == 2) ? (kk >> 2) : (kk >> 1);
+        widx[wo] = word;
+        part[wo] |= code[kk] << (field * BITS);
+        mask[wo] |= ((1u << BITS) - 1u) << (field * BITS);
+      }
+#pragma unroll
+      for (int i = 0; i < NWORD; ++i) {
+        uint32_t* dst = &img[chunk_word_byte(chunk, widx[i], wpc, 32) / 4];
+        if (clear_first) atomicAnd(dst, ~mask[i]);
+        atomicOr(dst, part[i]);
+      }
+    }
   }
-  if (bits == 16) {
-    for (int i = 0; i < epl; ++i) raw_dst[lane * epl + i] = e[i];
-    return;
+}
+
+// 16-bit passthrough of one side of a tile: rows [lo, hi) copied to the page as they are.
+__device__ __forceinline__ void copy_tile_side(const uint16_t* __restrict__ src, int64_t st, int D, int lo, int hi,
+                                               uint16_t* __restrict__ dst_rows, int lane) {
+  const int lpr = D >> 3, rps = 32 / lpr, l = lane & (lpr - 1);
+  for (int step = 0; step < 16 / rps; ++step) {
+    const int tau = step * rps + lane / lpr;
+    if (tau >= lo && tau < hi)
+      *reinterpret_cast<uint4*>(dst_rows + (size_t)tau * D + l * 8) =
+          *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + l * 8);
   }
-  float x[4];
-  float mn = INFINITY, mx = -INFINITY;
-  for (int i = 0; i < epl; ++i) {
-    x[i] = bits16_to_f32(e[i], dtype);
-    mn = fminf(mn, x[i]);
-    mx = fmaxf(mx, x[i]);
+}
+
+template <bool IS_V>
+__device__ __forceinline__ void quantize_tile_side_bits(int bits, const uint16_t* src, int64_t st, int D, int gsz,
+                                                        int dtype, int lo, int hi, uint32_t* img, uint32_t* meta_out,
+                                                        bool clear_first, int lane) {
+  if (bits == 2) quantize_tile_side<2, IS_V>(src, st, D, gsz, dtype, lo, hi, img, meta_out, clear_first, lane);
+  else if (bits == 4) quantize_tile_side<4, IS_V>(src, st, D, gsz, dtype, lo, hi, img, meta_out, clear_first, lane);
+  else quantize_tile_side<8, IS_V>(src, st, D, gsz, dtype, lo, hi, img, meta_out, clear_first, lane);
+}
+
+// Token-wise quantization of V (always) and of K (when do_k).  grid.y = stream, grid.x strides over the
+// 16-token tiles touched by this append, one warp per tile.
+__global__ void __launch_bounds__(kThreads)
+quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
+                   int64_t sb, int64_t sh, int64_t st, int t_new, int do_k) {
+  __shared__ __align__(16) uint32_t sImg[kWarps][2][512];   // per warp: key image, value image (<= 2 KB each)
+  const int bh = blockIdx.y;
+  const int b = bh / g.Hkv, h = bh % g.Hkv;
+  const int t0 = c.seq_len[b];
+  if (t0 + t_new > g.capacity) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int D = g.D;
+  const int first_tile = t0 >> 4;
+  const int n_tiles = ((t0 + t_new + 15) >> 4) - first_tile;
+  uint32_t* kimg = sImg[warp][0];
+  uint32_t* vimg = sImg[warp][1];
+  const int k_row_words = D * g.kb / 32;          // words per key row (quantized)
+  const int v_tile_words = D * g.vb / 2;          // words per value tile (quantized)
+
+  for (int j = blockIdx.x * kWarps + warp; j < n_tiles; j += gridDim.x * kWarps) {
+    const int tile = first_tile + j;
+    const int tbeg = max(t0, tile * 16), tend = min(t0 + t_new, tile * 16 + 16);
+    const int lo = tbeg & 15, hi = lo + (tend - tbeg);
+    const bool full = (hi - lo) == 16;
+    const int page = tile >> 3, tp0 = (tile & 7) * 16;        // page-local token of the tile's first row
+    uint8_t* pg = c.pages + ((size_t)bh * g.n_pages + page) * g.page_bytes;
+    // row 0 of the tile in the input (may lie before the first new token; never dereferenced there)
+    const int64_t off = (int64_t)b * sb + (int64_t)h * sh + (int64_t)(tile * 16 - t0) * st;
+
+    // ---- values
+    if (g.vb == 16) {
+      copy_tile_side(v_new + off, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg + g.v_codes_off) + (size_t)tp0 * D, lane);
+    } else {
+      uint4* gv = reinterpret_cast<uint4*>(pg + g.v_codes_off + (size_t)(tile & 7) * (v_tile_words * 4));
+      for (int i = lane; i < v_tile_words / 4; i += 32)
+        reinterpret_cast<uint4*>(vimg)[i] = full ? make_uint4(0u, 0u, 0u, 0u) : gv[i];
+      __syncwarp();
+      quantize_tile_side_bits<true>(g.vb, v_new + off, st, D, g.gv, g.in_dtype, lo, hi, vimg,
+                                    reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / g.gv), !full, lane);
+      __syncwarp();
+      for (int i = lane; i < v_tile_words / 4; i += 32) gv[i] = reinterpret_cast<const uint4*>(vimg)[i];
+    }
+    // ---- keys
+    if (do_k) {
+      if (g.kb == 16) {
+        copy_tile_side(k_new + off, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg) + (size_t)tp0 * D, lane);
+      } else {
+        for (int i = lane; i < 16 * k_row_words / 4; i += 32) reinterpret_cast<uint4*>(kimg)[i] = make_uint4(0u, 0u, 0u, 0u);
+        __syncwarp();
+        quantize_tile_side_bits<false>(g.kb, k_new + off, st, D, g.gk, g.in_dtype, lo, hi, kimg,
+                                       reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / g.gk), false, lane);
+        __syncwarp();
+        uint4* gk = reinterpret_cast<uint4*>(pg + (size_t)tp0 * (k_row_words * 4));
+        const int v_lo = lo * k_row_words / 4, v_hi = hi * k_row_words / 4;   // 16-byte vectors of the new rows
+        for (int i = v_lo + lane; i < v_hi; i += 32) gk[i] = reinterpret_cast<const uint4*>(kimg)[i];
+      }
+    }
+    __syncwarp();
   }
-  const int lpg = gsz / epl;  // lanes per group
-  for (int off = 1; off < lpg; off <<= 1) {
-    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, off));
-    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-  }
-  const float qmax = (float)((1 << bits) - 1);
-  GroupParams p = group_params(mn, mx, qmax);
-  if ((lane % lpg) == 0) meta[lane / lpg] = p.meta;
-  for (int i = 0; i < epl; ++i) codes[lane * epl + i] = (uint8_t)code_of(x[i], p, qmax);
 }
 
 // Pack K rows: `codes` holds bytes [ntok rows][D]; row r goes to page-local token slot0 + r.
@@ -62,64 +205,6 @@ __device__ __forceinline__ void pack_k_rows(const uint8_t* codes, int code_strid
       w |= (uint32_t)codes[r * code_stride + d] << (f * b);
     }
     *reinterpret_cast<uint32_t*>(kregion + (size_t)(slot0 + r) * (D * b / 8) + chunk_word_byte(chunk, word, wpc, 4)) = w;
-  }
-}
-
-// Token-wise quantization of V (always) and of K (when do_k): one CTA per
-// (16-token tile touched, stream).
-__global__ void __launch_bounds__(kThreads)
-quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
-                   int64_t sb, int64_t sh, int64_t st, int t_new, int do_k) {
-  __shared__ __align__(16) uint8_t sK[16][128];
-  __shared__ __align__(16) uint8_t sV[16][128];
-  const int bh = blockIdx.y;
-  const int b = bh / g.Hkv, h = bh % g.Hkv;
-  const int t0 = c.seq_len[b];
-  if (t0 + t_new > g.capacity) return;
-  const int tile = (t0 >> 4) + blockIdx.x;
-  const int tbeg = max(t0, tile * 16), tend = min(t0 + t_new, tile * 16 + 16);
-  if (tbeg >= tend) return;
-  const int page = tile >> 3;
-  uint8_t* pg = c.pages + ((size_t)bh * g.n_pages + page) * g.page_bytes;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int D = g.D;
-
-  for (int t = tbeg + warp; t < tend; t += kThreads / 32) {
-    const int tau = t & 15, tp = t & 127;
-    const int64_t off = (int64_t)b * sb + (int64_t)h * sh + (int64_t)(t - t0) * st;
-    quantize_row_warp(v_new + off, D, g.vb, g.gv, g.in_dtype, sV[tau],
-                      reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp * (D / g.gv),
-                      reinterpret_cast<uint16_t*>(pg + g.v_codes_off) + tp * D, lane);
-    if (do_k)
-      quantize_row_warp(k_new + off, D, g.kb, g.gk, g.in_dtype, sK[tau],
-                        reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp * (D / g.gk),
-                        reinterpret_cast<uint16_t*>(pg) + tp * D, lane);
-  }
-  __syncthreads();
-
-  const int ntok = tend - tbeg;
-  if (do_k && g.kb != 16) pack_k_rows(&sK[tbeg & 15][0], 128, ntok, tbeg & 127, pg, D, g.kb, tid);
-
-  if (g.vb != 16) {
-    const int b_ = g.vb;
-    const int wpt = D * b_ / 2;     // words per tile
-    const int wpc = D * b_ / 64;    // words per chunk
-    const int nf = 32 / b_;
-    const int lo = tbeg & 15, hi = lo + ntok;   // tile-local token range [lo, hi)
-    const bool full = (ntok == 16);
-    uint32_t* vt = reinterpret_cast<uint32_t*>(pg + g.v_codes_off + (size_t)(tile & 7) * (16 * D * b_ / 8));
-    const uint32_t fm = (1u << b_) - 1u;
-    for (int wi = tid; wi < wpt; wi += kThreads) {
-      int chunk = wi / wpc, word = wi % wpc;
-      uint32_t* wp = vt + chunk_word_byte(chunk, word, wpc, 32) / 4;
-      uint32_t w = full ? 0u : *wp;
-      for (int f = 0; f < nf; ++f) {
-        int tau, d;
-        v_field_pos(chunk, word, f, b_, tau, d);
-        if (tau >= lo && tau < hi) w = (w & ~(fm << (f * b_))) | ((uint32_t)sV[tau][d] << (f * b_));
-      }
-      *wp = w;
-    }
   }
 }
 
@@ -220,12 +305,18 @@ int launch_quantize_append(const Geom& g, const CachePtrs& c, const void* k_new,
                            int64_t sb, int64_t sh, int64_t st, int t_new, cudaStream_t stream) {
   const uint16_t* k = static_cast<const uint16_t*>(k_new);
   const uint16_t* v = static_cast<const uint16_t*>(v_new);
-  dim3 grid1((t_new + 15) / 16 + 1, g.B * g.Hkv);
+  // tiles touched per stream: at most ceil(t_new / 16) + 1; one warp per tile, CTAs stride over them
+  const int max_tiles = (t_new + 15) / 16 + 1;
+  int gx = (max_tiles + kWarps - 1) / kWarps;
+  const int streams = g.B * g.Hkv;
+  const int want = (148 * 16 + streams - 1) / streams;       // enough CTAs to fill the GPU, not one per tile
+  if (gx > want) gx = want;
+  dim3 grid1(gx, streams);
   quant_token_kernel<<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, g.k_axis == 0 ? 1 : 0);
   if (g.k_axis == 1) {
     size_t smem = (size_t)kPageTokens * g.D * 3;
     cudaFuncSetAttribute(quant_kchan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 3);
-    dim3 grid2((t_new + 127) / 128 + 1, g.B * g.Hkv);
+    dim3 grid2((t_new + 127) / 128 + 1, streams);
     quant_kchan_kernel<<<grid2, kThreads, smem, stream>>>(g, c, k, sb, sh, st, t_new);
   }
   bump_seq_len_kernel<<<(g.B + 127) / 128, 128, 0, stream>>>(g, c, t_new);
