@@ -76,6 +76,15 @@ __device__ __forceinline__ uint32_t code_of(float x, const GroupParams& p, float
   return (uint32_t)r;
 }
 
+// Same result as code_of without the round / convert instructions: after the clamp to [0, qmax], adding
+// 1.5 * 2^23 rounds to nearest-even in the float adder and leaves the integer in the low mantissa bits
+// (rounding and clamping to integer bounds commute).
+__device__ __forceinline__ uint32_t code_of_fast(float x, const GroupParams& p, float qmax) {
+  float u = __fmul_rn(__fsub_rn(x, p.z), p.inv);
+  u = fminf(fmaxf(u, 0.0f), qmax);
+  return __float_as_uint(__fadd_rn(u, 12582912.0f)) & 0xFFu;
+}
+
 // ---------------------------------------------------------------- layout index functions
 // Byte offset (inside the K-code region of a page) of the 32-bit word holding
 // channel d of page-local token t, and the field's bit offset inside that word.

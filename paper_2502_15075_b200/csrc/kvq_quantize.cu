@@ -22,17 +22,18 @@ constexpr uint32_t FULL = 0xffffffffu;
 // Quantize one side (keys or values) of a 16-token tile held in global memory as rows of D 16-bit values.
 // `img` is the warp's shared-memory image of the packed codes of the tile: for keys 16 token rows of
 // D*BITS/8 bytes, for values the tile's D*BITS*2 bytes.  Tokens outside [lo, hi) are left alone.
-template <int BITS, bool IS_V>
-__device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ src, int64_t st, int D, int gsz,
-                                                   int dtype, int lo, int hi, uint32_t* img,
+template <int BITS, bool IS_V, int D, int DTYPE>
+__device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ src, int64_t st, int gsz,
+                                                   int lo, int hi, uint32_t* img,
                                                    uint32_t* __restrict__ meta_out, bool clear_first, int lane) {
-  const int lpr = D >> 3;                    // lanes per token row (8 channels each)
-  const int rps = 32 / lpr;                  // rows per step
+  constexpr int lpr = D >> 3;                // lanes per token row (8 channels each)
+  constexpr int rps = 32 / lpr;              // rows per step
   const int l = lane & (lpr - 1);
   const int d0 = l * 8;
   const int lpg = gsz >> 3;                  // lanes per group
   const int ng = D / gsz;
   const float qmax = (float)((1 << BITS) - 1);
+#pragma unroll 4
   for (int step = 0; step < 16 / rps; ++step) {
     const int tau = step * rps + lane / lpr;
     const bool valid = tau >= lo && tau < hi;
@@ -43,21 +44,30 @@ __device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ 
     float mn = INFINITY, mx = -INFINITY;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      x[2 * i] = bits16_to_f32((uint16_t)(rw[i] & 0xFFFF), dtype);
-      x[2 * i + 1] = bits16_to_f32((uint16_t)(rw[i] >> 16), dtype);
+      if constexpr (DTYPE == KVQ_BF16) {
+        x[2 * i] = __uint_as_float(rw[i] << 16);
+        x[2 * i + 1] = __uint_as_float(rw[i] & 0xFFFF0000u);
+      } else {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&rw[i]));
+        x[2 * i] = f.x;
+        x[2 * i + 1] = f.y;
+      }
       mn = fminf(mn, fminf(x[2 * i], x[2 * i + 1]));
       mx = fmaxf(mx, fmaxf(x[2 * i], x[2 * i + 1]));
     }
-    for (int off = 1; off < lpg; off <<= 1) {
-      mn = fminf(mn, __shfl_xor_sync(FULL, mn, off));
-      mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, off));
+#pragma unroll
+    for (int off = 1; off < 16; off <<= 1) {
+      if (off < lpg) {
+        mn = fminf(mn, __shfl_xor_sync(FULL, mn, off));
+        mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, off));
+      }
     }
     const GroupParams p = group_params(mn, mx, qmax);
     if (!valid) continue;
     if ((l & (lpg - 1)) == 0) meta_out[tau * ng + d0 / gsz] = p.meta;
     uint32_t code[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) code[i] = code_of(x[i], p, qmax);
+    for (int i = 0; i < 8; ++i) code[i] = code_of_fast(x[i], p, qmax);
 
     if constexpr (!IS_V) {
       // keys: channels d0..d0+3 and d0+4..d0+7 are the four bytes of one word each (chunks 2(l%2), 2(l%2)+1),
@@ -120,17 +130,18 @@ __device__ __forceinline__ void copy_tile_side(const uint16_t* __restrict__ src,
   }
 }
 
-template <bool IS_V>
-__device__ __forceinline__ void quantize_tile_side_bits(int bits, const uint16_t* src, int64_t st, int D, int gsz,
-                                                        int dtype, int lo, int hi, uint32_t* img, uint32_t* meta_out,
+template <bool IS_V, int D, int DTYPE>
+__device__ __forceinline__ void quantize_tile_side_bits(int bits, const uint16_t* src, int64_t st, int gsz,
+                                                        int lo, int hi, uint32_t* img, uint32_t* meta_out,
                                                         bool clear_first, int lane) {
-  if (bits == 2) quantize_tile_side<2, IS_V>(src, st, D, gsz, dtype, lo, hi, img, meta_out, clear_first, lane);
-  else if (bits == 4) quantize_tile_side<4, IS_V>(src, st, D, gsz, dtype, lo, hi, img, meta_out, clear_first, lane);
-  else quantize_tile_side<8, IS_V>(src, st, D, gsz, dtype, lo, hi, img, meta_out, clear_first, lane);
+  if (bits == 2) quantize_tile_side<2, IS_V, D, DTYPE>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane);
+  else if (bits == 4) quantize_tile_side<4, IS_V, D, DTYPE>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane);
+  else quantize_tile_side<8, IS_V, D, DTYPE>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane);
 }
 
 // Token-wise quantization of V (always) and of K (when do_k).  grid.y = stream, grid.x strides over the
 // 16-token tiles touched by this append, one warp per tile.
+template <int D, int DTYPE>
 __global__ void __launch_bounds__(kThreads)
 quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
                    int64_t sb, int64_t sh, int64_t st, int t_new, int do_k) {
@@ -140,7 +151,6 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
   const int t0 = c.seq_len[b];
   if (t0 + t_new > g.capacity) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int D = g.D;
   const int first_tile = t0 >> 4;
   const int n_tiles = ((t0 + t_new + 15) >> 4) - first_tile;
   uint32_t* kimg = sImg[warp][0];
@@ -166,7 +176,7 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
       for (int i = lane; i < v_tile_words / 4; i += 32)
         reinterpret_cast<uint4*>(vimg)[i] = full ? make_uint4(0u, 0u, 0u, 0u) : gv[i];
       __syncwarp();
-      quantize_tile_side_bits<true>(g.vb, v_new + off, st, D, g.gv, g.in_dtype, lo, hi, vimg,
+      quantize_tile_side_bits<true, D, DTYPE>(g.vb, v_new + off, st, g.gv, lo, hi, vimg,
                                     reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / g.gv), !full, lane);
       __syncwarp();
       for (int i = lane; i < v_tile_words / 4; i += 32) gv[i] = reinterpret_cast<const uint4*>(vimg)[i];
@@ -178,7 +188,7 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
       } else {
         for (int i = lane; i < 16 * k_row_words / 4; i += 32) reinterpret_cast<uint4*>(kimg)[i] = make_uint4(0u, 0u, 0u, 0u);
         __syncwarp();
-        quantize_tile_side_bits<false>(g.kb, k_new + off, st, D, g.gk, g.in_dtype, lo, hi, kimg,
+        quantize_tile_side_bits<false, D, DTYPE>(g.kb, k_new + off, st, g.gk, lo, hi, kimg,
                                        reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / g.gk), false, lane);
         __syncwarp();
         uint4* gk = reinterpret_cast<uint4*>(pg + (size_t)tp0 * (k_row_words * 4));
@@ -312,7 +322,15 @@ int launch_quantize_append(const Geom& g, const CachePtrs& c, const void* k_new,
   const int want = (148 * 16 + streams - 1) / streams;       // enough CTAs to fill the GPU, not one per tile
   if (gx > want) gx = want;
   dim3 grid1(gx, streams);
-  quant_token_kernel<<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, g.k_axis == 0 ? 1 : 0);
+  const int do_k = g.k_axis == 0 ? 1 : 0;
+  if (g.D == 128 && g.in_dtype == KVQ_BF16)
+    quant_token_kernel<128, KVQ_BF16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, do_k);
+  else if (g.D == 128)
+    quant_token_kernel<128, KVQ_FP16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, do_k);
+  else if (g.in_dtype == KVQ_BF16)
+    quant_token_kernel<64, KVQ_BF16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, do_k);
+  else
+    quant_token_kernel<64, KVQ_FP16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, do_k);
   if (g.k_axis == 1) {
     size_t smem = (size_t)kPageTokens * g.D * 3;
     cudaFuncSetAttribute(quant_kchan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 3);
