@@ -62,6 +62,22 @@ def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
 
+# ----------------------------------------------------------------------------- multi-rank bookkeeping
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Every rank times its own replica; the job's time is the slowest rank's."""
+    if world <= 1:
+        return ms
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_rank_step: float, ms_per_step: float, world: int) -> float:
+    """Weak scaling: every rank streams the same number of bytes per step; aggregate over the job."""
+    return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -260,12 +276,7 @@ def main_gpu(args):
             fn(events) if events is not None else fn()
         e.record()
         barrier()
-        ms = s.elapsed_time(e)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(s.elapsed_time(e), world, dev)
 
     for _ in range(args.warmup):
         step_device()
@@ -285,8 +296,8 @@ def main_gpu(args):
 
     bytes_layer = decode_bytes_per_layer(w)
     bytes_step = bytes_layer * L
-    value = world * bytes_step / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * bytes_step / (e2e_ms * 1e-3) / 1e9
+    value = whole_job_gbs(bytes_step, ms_per_step, world)
+    e2e_value = whole_job_gbs(bytes_step, e2e_ms, world)
 
     if rank != 0:
         return
