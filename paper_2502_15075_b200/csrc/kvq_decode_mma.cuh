@@ -202,6 +202,23 @@ __device__ __forceinline__ void load_chunk(const uint8_t* base, int chunk, int n
   }
 }
 
+// Same, from a pointer that already addresses the lane's chunk; quads of words lie `quad_stride` bytes apart.
+template <int NWORDS>
+__device__ __forceinline__ void load_words(const uint8_t* p, int quad_stride, uint32_t (&w)[NWORDS]) {
+  if constexpr (NWORDS >= 4) {
+#pragma unroll
+    for (int qd = 0; qd < NWORDS / 4; ++qd) {
+      uint4 v = *reinterpret_cast<const uint4*>(p + qd * quad_stride);
+      w[4 * qd + 0] = v.x; w[4 * qd + 1] = v.y; w[4 * qd + 2] = v.z; w[4 * qd + 3] = v.w;
+    }
+  } else if constexpr (NWORDS == 2) {
+    uint2 v = *reinterpret_cast<const uint2*>(p);
+    w[0] = v.x; w[1] = v.y;
+  } else {
+    w[0] = *reinterpret_cast<const uint32_t*>(p);
+  }
+}
+
 __device__ __forceinline__ float meta_s(uint32_t m) { return __half2float(__ushort_as_half((uint16_t)(m & 0xFFFF))); }
 __device__ __forceinline__ float meta_z(uint32_t m) { return __half2float(__ushort_as_half((uint16_t)(m >> 16))); }
 

@@ -181,6 +181,12 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   int stage = 0;
   uint32_t phase = 0;
   bool aborted = false;
+  // byte offsets inside a page of this lane's operands for the warp's first tile (rows warp*16 + gid, +8)
+  constexpr int KCB = (KW < 4 ? KW : 4) * 4, VCB = (VW < 4 ? VW : 4) * 4;     // bytes of a lane chunk's first quad
+  const int lane_k = (warp * 16 + gid) * K_ROW_BYTES + tid * KCB;
+  const int lane_km = g.k_meta_off + (warp * 16 + gid) * 4 * NGK;
+  const int lane_v = g.v_codes_off + warp * V_TILE_BYTES + lane * VCB;
+  const int lane_vm = g.v_meta_off + (warp * 16 + gid) * 4 * NGV;
 
   for (long long x = x_lo; x < x_hi;) {
     const int seg_pages = (int)min((long long)(pages_b - page), x_hi - x);
@@ -276,6 +282,11 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       }
       if (!aborted) {
         const uint8_t* sp = smem + stage * sl.page_stride;
+        // this lane's first byte in each region for the warp's tile 0 (tile u adds a constant)
+        const uint8_t* sp_k = sp + lane_k;
+        const uint8_t* sp_km = sp + lane_km;
+        const uint8_t* sp_v = sp + lane_v;
+        const uint8_t* sp_vm = sp + lane_vm;
         const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
         const int ntiles = (nv + 15) >> 4;
 
@@ -302,7 +313,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
         // The TPW tiles this warp owns in the page (tile = warp + NW * u) are processed together: logits of all
         // of them, one joint running-max check, then probabilities and PV.  MASKED handles a partial page.
-        auto logits = [&](const int tok0, const bool v0, const bool v1, float (&L)[4]) {
+        auto logits = [&](const int u, const int tok0, const bool v0, const bool v1, float (&L)[4]) {
           if constexpr (KAXIS == 1) {
             float S[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // two chains, summed below
             if (tail_k) {
@@ -319,9 +330,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               for (int i = 0; i < 4; ++i) L[i] = c1 * (S[0][i] + S[1][i]);
             } else {
               uint32_t ka[KW], kb2[KW];
-              const uint8_t* krow = sp + (size_t)tok0 * K_ROW_BYTES;
-              load_chunk<KW>(krow, tid, 4, ka);
-              load_chunk<KW>(krow + 8 * K_ROW_BYTES, tid, 4, kb2);
+              const uint8_t* krow = sp_k + u * (NW * 16 * K_ROW_BYTES);      // this lane's chunk of row tok0
+              load_words<KW>(krow, 64, ka);
+              load_words<KW>(krow + 8 * K_ROW_BYTES, 64, kb2);
 #pragma unroll
               for (int w = 0; w < KW; ++w) {
                 uint32_t pa[Unpack<KB>::PPW], pb[Unpack<KB>::PPW];
@@ -338,9 +349,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             }
           } else {
             uint32_t ka[KW], kb2[KW];
-            const uint8_t* krow = sp + (size_t)tok0 * K_ROW_BYTES;
-            load_chunk<KW>(krow, tid, 4, ka);
-            load_chunk<KW>(krow + 8 * K_ROW_BYTES, tid, 4, kb2);
+            const uint8_t* krow = sp_k + u * (NW * 16 * K_ROW_BYTES);      // this lane's chunk of row tok0
+            load_words<KW>(krow, 64, ka);
+            load_words<KW>(krow + 8 * K_ROW_BYTES, 64, kb2);
             int S[NGK][NL][4];
 #pragma unroll
             for (int j = 0; j < NGK; ++j) {
@@ -355,7 +366,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
               for (int l = 0; l < NL; ++l) mma16832_u8s8(S[j][l], a0, a1, a2, a3, ql[l][2 * s], ql[l][2 * s + 1]);
             }
-            const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
+            const uint32_t* km = reinterpret_cast<const uint32_t*>(sp_km + u * (NW * 16 * 4 * NGK));   // row tok0
             L[0] = L[1] = L[2] = L[3] = 0.f;
 #pragma unroll
             for (int j = 0; j < NGK; ++j) {
@@ -363,8 +374,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
               for (int i = 0; i < 4; ++i)       // sum_d code_d * Q_d = (S0 * 256 + S1) * 256 + S2, exact up to the last step
                 t[i] = fmaf((float)(S[j][0][i] * 256 + S[j][1][i]), 256.f, (float)S[j][2][i]);
-              const float2 ma = __half22float2(as_h2(km[tok0 * NGK + j]));          // (scale, zero)
-              const float2 mb = __half22float2(as_h2(km[(tok0 + 8) * NGK + j]));
+              const float2 ma = __half22float2(as_h2(km[j]));                       // (scale, zero)
+              const float2 mb = __half22float2(as_h2(km[8 * NGK + j]));
               L[0] += fmaf(ma.x * hs0, t[0], ma.y * qsum[0][j]);
               L[1] += fmaf(ma.x * hs1, t[1], ma.y * qsum[1][j]);
               L[2] += fmaf(mb.x * hs0, t[2], mb.y * qsum[0][j]);
@@ -376,14 +387,14 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         };
 
         // values of one tile: fold the scale into p, keep the zero-point term as a scalar per group
-        auto values = [&](const int tile, const int tok0, const bool v0, const bool v1, const float (&p)[4]) {
-          const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp + g.v_meta_off);
+        auto values = [&](const int u, const bool v0, const bool v1, const float (&p)[4]) {
+          const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp_vm + u * (NW * 16 * 4 * NGV));   // row tok0
           const uint32_t pa01 = pack_h2(p[0], p[1]), pb01 = pack_h2(p[2], p[3]);
           uint32_t bw[NGV][2];
 #pragma unroll
           for (int j = 0; j < NGV; ++j) {
-            const uint32_t ma = v0 ? vm[tok0 * NGV + j] : 0u;
-            const uint32_t mb = v1 ? vm[(tok0 + 8) * NGV + j] : 0u;
+            const uint32_t ma = v0 ? vm[j] : 0u;
+            const uint32_t mb = v1 ? vm[8 * NGV + j] : 0u;
             const float za = meta_z(ma), zb = meta_z(mb);
             zacc[0][j] += p[0] * za + p[2] * zb;
             zacc[1][j] += p[1] * za + p[3] * zb;
@@ -393,7 +404,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             bw[j][1] = movmatrix_trans(as_u32(__hmul2(as_h2(pb01), as_h2(sb2))));
           }
           uint32_t vw[VW];
-          load_chunk<VW>(sp + g.v_codes_off + (size_t)tile * V_TILE_BYTES, lane, 32, vw);
+          load_words<VW>(sp_v + u * (NW * V_TILE_BYTES), 512, vw);
           uint32_t pv[4 * MT];
 #pragma unroll
           for (int w = 0; w < VW; ++w) {
@@ -420,7 +431,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             v0[u] = !MASKED || tok0 < nv;
             v1[u] = !MASKED || tok0 + 8 < nv;
             if (!MASKED || (warp + NW * u) < ntiles) {
-              logits(tok0, v0[u], v1[u], L[u]);
+              logits(u, tok0, v0[u], v1[u], L[u]);
             } else {
               L[u][0] = L[u][1] = L[u][2] = L[u][3] = -INFINITY;
             }
@@ -452,7 +463,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               p[0] = ex2(L[u][0] - m0); p[1] = ex2(L[u][1] - m1); p[2] = ex2(L[u][2] - m0); p[3] = ex2(L[u][3] - m1);
               l0 += p[0] + p[2];
               l1 += p[1] + p[3];
-              values(warp + NW * u, (warp + NW * u) * 16 + gid, v0[u], v1[u], p);
+              values(u, v0[u], v1[u], p);
             }
           }
         };

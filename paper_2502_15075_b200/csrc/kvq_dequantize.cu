@@ -89,7 +89,7 @@ __device__ __forceinline__ void store_rows(const uint16_t* tile, uint16_t* out, 
 }
 
 __global__ void __launch_bounds__(kThreads)
-dequant_kernel(Geom g, CachePtrs c, uint16_t* __restrict__ k_out, uint16_t* __restrict__ v_out,
+dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
                int t_begin, int t_end, int page0) {
   extern __shared__ __align__(16) uint8_t smem[];
   const int D = g.D, tid = threadIdx.x;
@@ -104,12 +104,17 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* __restrict__ k_out, uint16_t* __re
   if (lo_t >= hi_t) return;
   const int nv = min(kPageTokens, n - page * kPageTokens);
   const uint8_t* pg = c.pages + ((size_t)bh * g.n_pages + page) * g.page_bytes;
-  for (int i = tid; i < g.page_bytes / 16; i += kThreads)
+  // only this CTA's side of the page: keys [0, v_codes_off), values [v_codes_off, page_bytes)
+  const int v16_lo = (blockIdx.z == 0 ? g.v_codes_off : 0) / 16;
+  const int v16_hi = (blockIdx.z == 0 ? g.page_bytes : g.v_codes_off) / 16;
+  for (int i = v16_lo + tid; i < v16_hi; i += kThreads)
     reinterpret_cast<uint4*>(spage)[i] = reinterpret_cast<const uint4*>(pg)[i];
   __syncthreads();
   const int lo = lo_t - page * kPageTokens, hi_l = hi_t - page * kPageTokens;
   const size_t out_base = ((size_t)bh * g.capacity + (size_t)page * kPageTokens) * D;
 
+  // blockIdx.z picks the side: 0 values, 1 keys (two CTAs share a page so that short ranges still fill the GPU)
+  if (blockIdx.z == 0) k_out = nullptr; else v_out = nullptr;
   if (v_out) {
     if (g.vb == 16) {
       store_rows(reinterpret_cast<const uint16_t*>(spage + g.v_codes_off), v_out + out_base, D, lo, hi_l, tid);
@@ -155,7 +160,7 @@ int launch_dequantize(const Geom& g, const CachePtrs& c, void* k_out, void* v_ou
   const int page1 = (t_end + kPageTokens - 1) / kPageTokens;
   const size_t smem = (size_t)((g.page_bytes + 15) & ~15) + (size_t)kPageTokens * g.D * 2;
   cudaFuncSetAttribute(dequant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 4 + 128 * 128 * 2);
-  dim3 grid(page1 - page0, g.B * g.Hkv);
+  dim3 grid(page1 - page0, g.B * g.Hkv, 2);
   dequant_kernel<<<grid, kThreads, smem, stream>>>(g, c, static_cast<uint16_t*>(k_out),
                                                    static_cast<uint16_t*>(v_out), t_begin, t_end, page0);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
