@@ -2,14 +2,19 @@
 // (App. A.1) over the packed cache, with K^ = z + s*code and V^ likewise
 // reconstructed inside the contraction.
 //
-// Structure (one CTA = NW consumer warps + 1 producer warp):
+// Structure (one CTA = NW consumer warps + 1 producer warp, several CTAs per SM):
 //  * the producer streams whole 128-token pages into a shared-memory ring with
 //    cp.async.bulk (one bulk copy per page, completion on an mbarrier);
 //  * each consumer warp owns 16-token tiles of every page: it loads its operand
-//    fragments with 16-byte shared loads (the page layout already is fragment
-//    order), turns the codes into integer-valued fp16 with LOP3/PRMT + one HFMA2
-//    per pair, and runs QK^T and PV on the tensor cores (mma.m16n8k16, fp32
-//    accumulate) for the <= 8 query heads that share the KV head;
+//    fragments with 16-byte shared loads (the page layout already is fragment order);
+//  * token-wise keys: the code bytes go straight into integer tensor-core MMAs
+//    (mma.m16n8k32 u8 x s8 -> s32; one mask or shift+mask per register), with q held as
+//    22-bit fixed point split into three signed bytes per head, so q.c_t is exact;
+//    channel-wise keys: fp16 MMAs on codes converted with LOP3 + HFMA2, channel scales
+//    folded into q once per page;
+//  * values: codes become integer-valued fp16 with one LOP3 + one HFMA2 per pair and
+//    PV runs on fp16 MMAs (mma.m16n8k16, fp32 accumulate) for the <= 8 query heads
+//    that share the KV head;
 //  * scale and zero-point never touch the codes:  q.K^_t = s_t (q.c_t) + z_t sum(q)
 //    and  o = sum_t (p_t s_t) c_t + sum_t p_t z_t ;
 //  * the sequence is split flat over the grid: CTA i takes the i-th equal share of
