@@ -33,6 +33,11 @@ struct CachePtrs {
   uint32_t* status;
 };
 
+// Sequence length as the kernels use it: a corrupt value can never index outside the cache.
+__device__ __forceinline__ int clamped_len(const int32_t* seq_len, int b, int capacity) {
+  return min(max(seq_len[b], 0), capacity);
+}
+
 // ---------------------------------------------------------------- conversions
 __device__ __forceinline__ float bits16_to_f32(uint16_t u, int dtype) {
   if (dtype == KVQ_FP16) return __half2float(__ushort_as_half(u));

@@ -32,7 +32,7 @@ decode_generic_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float
   const int bh = blockIdx.y, split = blockIdx.x;
   const int b = bh / g.Hkv, h = bh % g.Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int n = c.seq_len[b];
+  const int n = clamped_len(c.seq_len, b, g.capacity);
   const int n_pages = (n + kPageTokens - 1) / kPageTokens;
   const int chunk = (n_pages + n_split - 1) / n_split;
   const int p0 = split * chunk, p1 = min(n_pages, p0 + chunk);

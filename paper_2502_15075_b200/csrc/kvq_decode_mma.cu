@@ -22,7 +22,7 @@ __global__ void merge_flat_kernel(Geom g, const int32_t* __restrict__ seq_len, c
   long long N = 0, before = 0;
   int pages_max = 0, pages_b = 0;
   for (int i = 0; i < g.B; ++i) {
-    int p = (seq_len[i] + kPageTokens - 1) >> 7;
+    int p = (clamped_len(seq_len, i, g.capacity) + kPageTokens - 1) >> 7;
     if (i < b) before += p;
     if (i == b) pages_b = p;
     N += p;

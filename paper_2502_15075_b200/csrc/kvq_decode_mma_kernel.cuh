@@ -83,7 +83,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   if (tid_ == 0) { sPref[0] = 0; sMisc[0] = 0; sMisc[1] = 0; }
   __syncthreads();
   for (int b = tid_; b < B; b += blockDim.x) {
-    int pages = (c.seq_len[b] + kPageTokens - 1) >> 7;
+    int pages = (clamped_len(c.seq_len, b, g.capacity) + kPageTokens - 1) >> 7;
     sPref[b + 1] = pages * Hkv;
     atomicMax(&sMisc[0], pages);
   }
@@ -190,7 +190,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
   for (long long x = x_lo; x < x_hi;) {
     const int seg_pages = (int)min((long long)(pages_b - page), x_hi - x);
-    const int n_tok = c.seq_len[b];
+    const int n_tok = clamped_len(c.seq_len, b, g.capacity);
     const int stream = b * Hkv + h;
 
     // ---- segment start: q operands and group sums for this stream's heads

@@ -97,7 +97,7 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
   uint16_t* tile = reinterpret_cast<uint16_t*>(smem + ((g.page_bytes + 15) & ~15));   // [128][D]
   const int bh = blockIdx.y;
   const int b = bh / g.Hkv;
-  const int n = c.seq_len[b];
+  const int n = clamped_len(c.seq_len, b, g.capacity);
   const int hi = min(t_end, n);
   const int page = page0 + blockIdx.x;
   const int lo_t = max(t_begin, page * kPageTokens), hi_t = min(hi, page * kPageTokens + kPageTokens);

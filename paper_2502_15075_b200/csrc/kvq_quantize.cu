@@ -149,7 +149,7 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
   const int bh = blockIdx.y;
   const int b = bh / g.Hkv, h = bh % g.Hkv;
   const int t0 = c.seq_len[b];
-  if (t0 + t_new > g.capacity) return;
+  if (t0 < 0 || t0 + t_new > g.capacity) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int first_tile = t0 >> 4;
   const int n_tiles = ((t0 + t_new + 15) >> 4) - first_tile;
@@ -232,7 +232,7 @@ quant_kchan_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new,
   const int bh = blockIdx.y;
   const int b = bh / g.Hkv, h = bh % g.Hkv;
   const int t0 = c.seq_len[b];
-  if (t0 + t_new > g.capacity) return;
+  if (t0 < 0 || t0 + t_new > g.capacity) return;
   const int end = t0 + t_new;
   const int first_page = t0 >> 7;
   const int nblk = ((end + 127) >> 7) - first_page;
@@ -302,7 +302,7 @@ __global__ void bump_seq_len_kernel(Geom g, CachePtrs c, int t_new) {
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= g.B) return;
   int t0 = c.seq_len[b];
-  if (t0 + t_new > g.capacity) {
+  if (t0 < 0 || t0 + t_new > g.capacity) {
     atomicOr(c.status, KVQ_STATUS_CAPACITY);
   } else {
     c.seq_len[b] = t0 + t_new;

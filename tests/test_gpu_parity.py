@@ -213,3 +213,28 @@ def test_k4v2_beats_k2v4_on_gpu(kvq):
             got = tl.gpu_decode(kvq, cfg, gc, q)
             e[(kb, vb)].append(np.linalg.norm(got - exact) / np.linalg.norm(exact))
     assert np.mean(e[(4, 2)]) < np.mean(e[(2, 4)])
+
+
+def test_corrupt_sequence_lengths_are_clamped(kvq):
+    """A seq_len outside [0, capacity] never indexes outside the cache: decode and dequantize treat it as
+    clamped, append refuses it and sets the capacity status."""
+    w = wl.LLAMA_8B.with_(n_kv_heads=2, n_q_heads=8)
+    B, cap = 3, 256
+    k, v = wl.make_kv(w, tokens=cap, batch=B)
+    cfg = tl.gpu_config_for(kvq, w, B, cap)
+    gc = kvq.Cache(cfg)
+    oc = tl.oracle_cache_for(w, B, cap)
+    kvq.kvq_quantize_append(cfg, gc, k.cuda(), v.cuda())
+    oc.append(tl.bits_of(k), tl.bits_of(v))
+    gc.seq_len.copy_(torch.tensor([-5, 10 ** 6, 200], dtype=torch.int32))
+    oc.seq_len[:] = [0, cap, 200]
+    q = wl.make_q(w, batch=B)
+    got = tl.gpu_decode(kvq, cfg, gc, q)
+    tl.assert_attention_close(got, oc.decode(tl.bits_of(q)))
+    assert not got[0].any()
+    ko = torch.zeros((B, 2, cap, 128), dtype=torch.bfloat16, device="cuda")
+    kvq.kvq_dequantize(cfg, gc, ko, None, 0, cap)
+    assert not ko[0].any() and ko[1].abs().sum() > 0 and not ko[2, :, 200:].any()
+    kvq.kvq_quantize_append(cfg, gc, k.cuda()[:, :, :8], v.cuda()[:, :, :8])
+    assert kvq.kvq_check_status(gc) == -5
+    assert gc.seq_len.tolist() == [-5, 10 ** 6, 208]
