@@ -36,9 +36,9 @@
  *     r = d/16, word r/fpb, bit 8*(d%4) + b*(r%fpb)  (byte j of a word holds channels
  *     16r + 4*chunk + j: one mask per field gives four consecutive channels as four bytes).
  *   V codes, b in {2,4,8}: 8 tiles of 16 tokens, each holding 32 chunks of
- *     wpc = D*b/64 words; with k = 8*(d/64) + d%8, channel d of tile-local token tau:
- *     chunk 4*((d/8)%8) + (tau%8)/2, P = 4*(k/2) + k%2 + 2*(tau/8), word P/ppw,
- *     field P%ppw + ppw*(tau%2).
+ *     wpc = D*b/64 words; with k = 8*(d/64) + d%8 and npos = 8/b, channel d of tile-local
+ *     token tau: chunk 4*((d/8)%8) + (tau%8)/2, word k/npos,
+ *     field k%npos + npos*(tau/8) + ppw*(tau%2).
  *   (chunk, word) inside a row / tile of nchunks chunks, with qw = min(wpc, 4):
  *     byte = (word/4)*(nchunks*4*qw) + chunk*(4*qw) + (word%4)*4   (quads of words, quad-major).
  *   b = 16: rows [token][D] of the input's 16-bit patterns, no meta.

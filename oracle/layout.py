@@ -22,11 +22,13 @@ token lives in
 share the word: masking one field out of every byte yields four consecutive
 channels as four bytes).
 V codes (b = vb in {2,4,8}): 8 tiles of 16 tokens, a tile holds 32 chunks of
-wpc = D*b/64 words.  With k = 8*(d // 64) + d % 8, channel d of token tau
-(0..15 inside its tile) lives in
+wpc = D*b/64 words.  With k = 8*(d // 64) + d % 8 and npos = 8/b, channel d of
+token tau (0..15 inside its tile) lives in
     chunk  = 4*((d // 8) % 8) + (tau % 8) // 2
-    P      = 4*(k // 2) + k % 2 + 2*(tau // 8)
-    word   = P // ppw,  field = P % ppw + ppw*(tau % 2)
+    word   = k // npos
+    field  = k % npos + npos*(tau // 8) + ppw*(tau % 2)
+(a 16-bit half of a word holds, in its low byte, the codes of tokens 0..7 of the
+tile and, in its high byte, those of tokens 8..15, at the same bit position).
 Placement of (chunk, word) inside its row / tile of `nchunks` chunks: words are
 kept in quads of qw = min(wpc, 4) words, quad-major:
     byte   = (word // 4)*(nchunks*4*qw) + chunk*(4*qw) + (word % 4)*4
@@ -116,11 +118,11 @@ def v_code_pos(t, d, D, b):
     ppw = 16 // b
     tile = t // 16
     tau = t % 16
+    npos = 8 // b                     # code positions inside the low byte of a 16-bit half
     k = 8 * (d // 64) + d % 8
     chunk = 4 * ((d // 8) % 8) + (tau % 8) // 2
-    P = 4 * (k // 2) + k % 2 + 2 * (tau // 8)
-    word = P // ppw
-    field = P % ppw + ppw * (tau % 2)
+    word = k // npos
+    field = k % npos + npos * (tau // 8) + ppw * (tau % 2)
     bit = field * b
     byte = tile * (16 * D * b // 8) + _chunk_word_byte(chunk, word, D * b // 64, 32) + bit // 8
     return byte, bit % 8

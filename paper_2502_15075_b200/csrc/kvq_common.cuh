@@ -111,11 +111,11 @@ __host__ __device__ __forceinline__ void k_code_pos(int t, int d, int D, int b, 
 __host__ __device__ __forceinline__ void v_code_pos(int t, int d, int D, int b, int& word_byte, int& bit) {
   int ppw = 16 / b;
   int tile = t >> 4, tau = t & 15;
+  int npos = 8 / b;             // code positions inside the low byte of a 16-bit half
   int k = 8 * (d >> 6) + (d & 7);
   int chunk = 4 * ((d >> 3) & 7) + ((tau & 7) >> 1);
-  int P = 4 * (k >> 1) + (k & 1) + 2 * (tau >> 3);
-  word_byte = tile * (16 * D * b / 8) + chunk_word_byte(chunk, P / ppw, D * b / 64, 32);
-  bit = (P % ppw + ppw * (tau & 1)) * b;
+  word_byte = tile * (16 * D * b / 8) + chunk_word_byte(chunk, k / npos, D * b / 64, 32);
+  bit = (k % npos + npos * (tau >> 3) + ppw * (tau & 1)) * b;
 }
 
 // Inverse maps: which channel (and tile-local token) sits in field f of a word.
@@ -127,10 +127,11 @@ __device__ __forceinline__ int k_field_channel(int chunk, int word, int f, int b
 
 __device__ __forceinline__ void v_field_pos(int chunk, int word, int f, int b, int D, int& tau, int& d) {
   int ppw = 16 / b;
-  int P = word * ppw + (f % ppw);
-  int k = 2 * (P >> 2) + (P & 1);
+  int npos = 8 / b;
+  int fh = f % ppw;             // field inside its 16-bit half
+  int k = word * npos + fh % npos;
   d = 64 * (k >> 3) + 8 * (chunk >> 2) + (k & 7);
-  tau = 8 * ((P & 3) >> 1) + 2 * (chunk & 3) + (f / ppw);
+  tau = 8 * (fh / npos) + 2 * (chunk & 3) + (f / ppw);
 }
 
 __device__ __forceinline__ uint32_t load_code(const uint8_t* region, int word_byte, int bit, int b) {

@@ -153,6 +153,17 @@ __device__ __forceinline__ uint32_t key_slot(const uint32_t (&kw)[KW], int r) {
   }
 }
 
+// Value codes as fp16 MMA operands without arithmetic: (x & mask) | 0x64006400 puts the B-bit field at
+// position `pos` of the low byte of each 16-bit half into the mantissa of 1024.0, giving the two halves the
+// values 1024 + code * 2^(B * pos) of two consecutive tokens.
+template <int B>
+__device__ __forceinline__ uint32_t biased_pair(uint32_t x, int pos) {
+  const uint32_t mask = (((1u << B) - 1u) << (B * pos)) * 0x00010001u;
+  uint32_t d;
+  asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "r"(mask), "r"(kMagic));
+  return d;
+}
+
 template <int B> struct Unpack;
 
 template <> struct Unpack<4> {

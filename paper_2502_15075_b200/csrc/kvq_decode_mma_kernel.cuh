@@ -60,7 +60,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   constexpr int KW = D * KB / 128;          // K words per lane per token row
   constexpr int VW = D * VB / 64;           // V words per lane per 16-token tile
   constexpr int FPB = 8 / KB;               // key fields per byte
-  constexpr int VPPW = Unpack<VB>::PPW;
+  constexpr int NPOS = 8 / VB;              // value code positions inside a byte
   constexpr int K_ROW_BYTES = D * KB / 8;
   constexpr int V_TILE_BYTES = 16 * D * VB / 8;
   constexpr int NCONS = NW * 32;
@@ -313,6 +313,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
         // The TPW tiles this warp owns in the page (tile = warp + NW * u) are processed together: logits of all
         // of them, one joint running-max check, then probabilities and PV.  MASKED handles a partial page.
+        float wbias[NGV][4];                   // sum of p * s over the tokens of one do_tiles call, per head
         auto logits = [&](const int u, const int tok0, const bool v0, const bool v1, float (&L)[4]) {
           if constexpr (KAXIS == 1) {
             float S[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // two chains, summed below
@@ -403,21 +404,27 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             bw[j][0] = movmatrix_trans(as_u32(__hmul2(as_h2(pa01), as_h2(sa2))));
             bw[j][1] = movmatrix_trans(as_u32(__hmul2(as_h2(pb01), as_h2(sb2))));
           }
+          // The codes enter the MMA as 1024 + code * 2^(VB * pos) (field bits OR-ed into the mantissa of 1024.0,
+          // one LOP3 per register): the 2^(VB * pos) factor is the same for every token of a channel and is
+          // divided out once per stream; the 1024 adds 1024 * sum_t w_t to every row, which an MMA against
+          // all-ones rows accumulates in wbias and do_tiles subtracts again before it can cost precision.
           uint32_t vw[VW];
           load_words<VW>(sp_v + u * (NW * V_TILE_BYTES), 512, vw);
-          uint32_t pv[4 * MT];
+          uint32_t vh[VW];
 #pragma unroll
-          for (int w = 0; w < VW; ++w) {
-            uint32_t t[VPPW];
-            Unpack<VB>::run(vw[w], t);
-#pragma unroll
-            for (int i = 0; i < VPPW; ++i) pv[w * VPPW + i] = t[i];
-          }
+          for (int w = 0; w < VW; ++w) vh[w] = vw[w] >> 8;        // tokens 8..15 of the tile
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             const int j = mt / (MT / NGV);
-            mma16816(O[mt], pv[4 * mt], pv[4 * mt + 1], pv[4 * mt + 2], pv[4 * mt + 3], bw[j][0], bw[j][1]);
+            const uint32_t a0 = biased_pair<VB>(vw[(2 * mt) / NPOS], (2 * mt) % NPOS);
+            const uint32_t a1 = biased_pair<VB>(vw[(2 * mt + 1) / NPOS], (2 * mt + 1) % NPOS);
+            const uint32_t a2 = biased_pair<VB>(vh[(2 * mt) / NPOS], (2 * mt) % NPOS);
+            const uint32_t a3 = biased_pair<VB>(vh[(2 * mt + 1) / NPOS], (2 * mt + 1) % NPOS);
+            mma16816(O[mt], a0, a1, a2, a3, bw[j][0], bw[j][1]);
           }
+#pragma unroll
+          for (int j = 0; j < NGV; ++j)
+            mma16816(wbias[j], 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, bw[j][0], bw[j][1]);
         };
 
         auto do_tiles = [&](auto masked_tag) {
@@ -425,6 +432,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           float L[TPW][4];
           bool v0[TPW], v1[TPW];
           float t0 = -INFINITY, t1 = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < NGV; ++j) { wbias[j][0] = wbias[j][1] = wbias[j][2] = wbias[j][3] = 0.f; }
 #pragma unroll
           for (int u = 0; u < TPW; ++u) {
             const int tok0 = (warp + NW * u) * 16 + gid;        // page-local tokens of this lane's two rows
@@ -466,6 +475,13 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               values(u, v0[u], v1[u], p);
             }
           }
+          // take the 1024 * sum(w) of these tiles out of the accumulators again
+#pragma unroll
+          for (int mt = 0; mt < MT; ++mt) {
+            const int j = mt / (MT / NGV);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) O[mt][r] = fmaf(-1024.f, wbias[j][r], O[mt][r]);
+          }
         };
 
         if (ntiles > warp) {                     // a short last page may leave this warp without a tile
@@ -493,7 +509,10 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
         const int j = mt / (MT / NGV);
-        O[mt][0] += zacc[0][j]; O[mt][1] += zacc[1][j]; O[mt][2] += zacc[0][j]; O[mt][3] += zacc[1][j];
+        // rows (gid, gid + 8) of m-tile mt hold channel slots k = 2 mt, 2 mt + 1: undo their 2^(VB * (k % NPOS))
+        const float f0 = 1.f / (float)(1 << (VB * ((2 * mt) % NPOS))), f1 = 1.f / (float)(1 << (VB * ((2 * mt + 1) % NPOS)));
+        O[mt][0] = fmaf(O[mt][0], f0, zacc[0][j]); O[mt][1] = fmaf(O[mt][1], f0, zacc[1][j]);
+        O[mt][2] = fmaf(O[mt][2], f1, zacc[0][j]); O[mt][3] = fmaf(O[mt][3], f1, zacc[1][j]);
       }
       constexpr int PER_LANE = MT * 4 + 4;
 #pragma unroll

@@ -92,18 +92,18 @@ __device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ 
       const int gidc = l & 7, h = l >> 3;            // d0 = 64 h + 8 gidc
       const int tidT = (tau & 7) >> 1, hiT = tau >> 3, oddT = tau & 1;
       const int chunk = 4 * gidc + tidT;
-      constexpr int NWORD = (BITS == 2) ? 2 : 4;     // words this lane contributes to
+      constexpr int NWORD = BITS;                    // words this lane contributes to (8 codes, 8/BITS per word)
       uint32_t part[NWORD], mask[NWORD];
       int widx[NWORD];
 #pragma unroll
       for (int i = 0; i < NWORD; ++i) { part[i] = 0; mask[i] = 0; widx[i] = 0; }
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
+        constexpr int NPOS = 8 / BITS;
         const int k = 8 * h + kk;
-        const int P = 4 * (k >> 1) + (k & 1) + 2 * hiT;
-        const int word = P / PPW;
-        const int field = P % PPW + PPW * oddT;
-        const int wo = (BITS == 2) ? (kk >> 2) : (kk >> 1);
+        const int word = k / NPOS;
+        const int field = k % NPOS + NPOS * hiT + PPW * oddT;
+        const int wo = kk / NPOS;
         widx[wo] = word;
         part[wo] |= code[kk] << (field * BITS);
         mask[wo] |= ((1u << BITS) - 1u) << (field * BITS);

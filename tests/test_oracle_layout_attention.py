@@ -88,18 +88,19 @@ def test_single_field_encoding_is_little_endian_words():
     assert ol.k_code_pos(0, 48, 128, 2) == (0, 6)
     assert ol.k_code_pos(0, 64, 128, 2) == (4, 0)
     assert ol.k_code_pos(0, 4, 128, 2) == (8, 0)
-    # V, D=128, 2-bit: (t=0,d=0) byte 0; t=1 (odd token): field 8 -> byte 2
+    # V, D=128, 2-bit (4 positions per byte): (t=0,d=0) byte 0; t=1 (odd token): field 8 -> byte 2
     assert ol.v_code_pos(0, 0, 128, 2) == (0, 0)
     assert ol.v_code_pos(1, 0, 128, 2) == (2, 0)
-    # t=2 -> chunk 1 -> byte 16 ; d=8 -> next chunk group -> chunk 4 -> byte 64 ; t=8 -> P=2 -> field 2 -> bit 4
+    # t=2 -> chunk 1 -> byte 16 ; d=8 -> next chunk group -> chunk 4 -> byte 64 ; t=8 -> high byte of the half
     assert ol.v_code_pos(2, 0, 128, 2) == (16, 0)
     assert ol.v_code_pos(0, 8, 128, 2) == (64, 0)
-    assert ol.v_code_pos(8, 0, 128, 2) == (0, 4)
-    # d=1 -> k=1 -> P=1 -> bit 2 ; d=2 -> k=2 -> P=4 -> bit 8 -> byte 1 ; d=4 -> P=8 -> word 1 -> byte 4
+    assert ol.v_code_pos(8, 0, 128, 2) == (1, 0)
+    assert ol.v_code_pos(9, 0, 128, 2) == (3, 0)
+    # d=1..3 -> positions 1..3 of the same byte ; d=4 -> k=4 -> word 1 -> byte 4
     assert ol.v_code_pos(0, 1, 128, 2) == (0, 2)
-    assert ol.v_code_pos(0, 2, 128, 2) == (1, 0)
+    assert ol.v_code_pos(0, 3, 128, 2) == (0, 6)
     assert ol.v_code_pos(0, 4, 128, 2) == (4, 0)
-    # d=64 -> k=8 -> P=16 -> word 2 -> byte 8 (same chunk as d=0)
+    # d=64 -> k=8 -> word 2 -> byte 8 (same chunk as d=0)
     assert ol.v_code_pos(0, 64, 128, 2) == (8, 0)
     # next tile of 16 tokens: 16*128*2/8 = 512 bytes further
     assert ol.v_code_pos(16, 0, 128, 2) == (512, 0)
@@ -112,10 +113,17 @@ def test_single_field_encoding_is_little_endian_words():
     assert ol.k_code_pos(0, 64, 128, 8) == (64, 0)
     assert ol.k_code_pos(0, 68, 128, 8) == (80, 0)
     assert ol.k_code_pos(1, 0, 128, 8) == (128, 0)
-    # V, D=128, 4-bit (8 words per chunk): d=64 -> k=8 -> P=16 -> word 4 -> second quad -> byte 32 chunks * 16 = 512
+    # V, D=128, 4-bit (2 positions per byte, 8 words per chunk): d=1 -> high nibble of byte 0; d=2 -> word 1;
+    # d=64 -> k=8 -> word 4 -> second quad -> byte 32 chunks * 16 = 512
+    assert ol.v_code_pos(0, 1, 128, 4) == (0, 4)
+    assert ol.v_code_pos(0, 2, 128, 4) == (4, 0)
     assert ol.v_code_pos(0, 64, 128, 4) == (512, 0)
     assert ol.v_code_pos(2, 64, 128, 4) == (528, 0)
-    assert ol.v_code_pos(0, 2, 128, 4) == (4, 0)
+    # 8-bit: one word per channel slot k: tokens (0, 8, 1, 9) of the lane's token pair in bytes 0..3
+    assert ol.v_code_pos(0, 0, 128, 8) == (0, 0)
+    assert ol.v_code_pos(8, 0, 128, 8) == (1, 0)
+    assert ol.v_code_pos(1, 0, 128, 8) == (2, 0)
+    assert ol.v_code_pos(0, 1, 128, 8) == (4, 0)
 
 
 def test_memory_ratio_k4v2_vs_k4v4():
