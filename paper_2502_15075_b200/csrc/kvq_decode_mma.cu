@@ -38,18 +38,32 @@ __global__ void merge_flat_kernel(Geom g, const int32_t* __restrict__ seq_len, c
     const int n = min(c_last - c_first + 1, s_cap);
     const float* base = ws + (((size_t)(b * g.Hkv + h) * s_cap) * g.G + gh) * (D + 2);
     const size_t slot_stride = (size_t)g.G * (D + 2);
-    float mstar = -INFINITY;
-    for (int j = 0; j < n; ++j) mstar = fmaxf(mstar, base[j * slot_stride]);
-    float num = 0.f, den = 0.f;
-    if (mstar != -INFINITY) {
-      for (int j = 0; j < n; ++j) {
-        const float* pj = base + j * slot_stride;
-        const float mj = pj[0];
-        if (mj == -INFINITY) continue;
-        const float w = exp2f(mj - mstar);
-        num = fmaf(w, pj[2 + d], num);
-        den = fmaf(w, pj[1], den);
+    // slots are few: issue all loads of a batch of 8 before using any (the merge is latency-bound)
+    float mstar = -INFINITY, num = 0.f, den = 0.f;
+    for (int j0 = 0; j0 < n; j0 += 8) {
+      float mj[8], lj[8], oj[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const bool on = j0 + u < n;
+        const float* pj = base + (size_t)(on ? j0 + u : 0) * slot_stride;
+        mj[u] = on ? pj[0] : -INFINITY;
+        lj[u] = on ? pj[1] : 0.f;
+        oj[u] = on ? pj[2 + d] : 0.f;
       }
+      float mb = mstar;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) mb = fmaxf(mb, mj[u]);
+      if (mb == -INFINITY) continue;
+      const float keep = (mstar == -INFINITY) ? 0.f : exp2f(mstar - mb);
+      num *= keep;
+      den *= keep;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const float w = (mj[u] == -INFINITY) ? 0.f : exp2f(mj[u] - mb);
+        num = fmaf(w, oj[u], num);
+        den = fmaf(w, lj[u], den);
+      }
+      mstar = mb;
     }
     r = den > 0.f ? num / den : 0.f;
   }

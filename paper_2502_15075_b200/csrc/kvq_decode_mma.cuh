@@ -164,6 +164,19 @@ __device__ __forceinline__ uint32_t biased_pair(uint32_t x, int pos) {
   return d;
 }
 
+// Codes are centred on the middle of their range before the PV contraction.
+template <int B> constexpr float kCodeMid = (float)(1 << (B - 1));
+
+// biased_pair, then one HFMA2: (1024 + code * 2^(B pos)) * 2^-(B pos) - (1024 * 2^-(B pos) + MID) = code - MID,
+// exact in fp16 (all constants and the result are representable).
+template <int B>
+__device__ __forceinline__ uint32_t centered_pair(uint32_t x, int pos) {
+  const float inv = 1.f / (float)(1 << (B * pos));
+  const __half2 scale = __float2half2_rn(inv);
+  const __half2 off = __float2half2_rn(-(1024.f * inv + kCodeMid<B>));
+  return as_u32(__hfma2(as_h2(biased_pair<B>(x, pos)), scale, off));
+}
+
 template <int B> struct Unpack;
 
 template <> struct Unpack<4> {

@@ -313,7 +313,6 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
         // The TPW tiles this warp owns in the page (tile = warp + NW * u) are processed together: logits of all
         // of them, one joint running-max check, then probabilities and PV.  MASKED handles a partial page.
-        float wbias[NGV][4];                   // sum of p * s over the tokens of one do_tiles call, per head
         auto logits = [&](const int u, const int tok0, const bool v0, const bool v1, float (&L)[4]) {
           if constexpr (KAXIS == 1) {
             float S[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // two chains, summed below
@@ -396,7 +395,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           for (int j = 0; j < NGV; ++j) {
             const uint32_t ma = v0 ? vm[j] : 0u;
             const uint32_t mb = v1 ? vm[8 * NGV + j] : 0u;
-            const float za = meta_z(ma), zb = meta_z(mb);
+            // zero-point of the centred codes: z + s * MID
+            const float za = fmaf(meta_s(ma), kCodeMid<VB>, meta_z(ma)), zb = fmaf(meta_s(mb), kCodeMid<VB>, meta_z(mb));
             zacc[0][j] += p[0] * za + p[2] * zb;
             zacc[1][j] += p[1] * za + p[3] * zb;
             // (p * s) in fp16: both heads of a row share the row's scale
@@ -404,10 +404,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             bw[j][0] = movmatrix_trans(as_u32(__hmul2(as_h2(pa01), as_h2(sa2))));
             bw[j][1] = movmatrix_trans(as_u32(__hmul2(as_h2(pb01), as_h2(sb2))));
           }
-          // The codes enter the MMA as 1024 + code * 2^(VB * pos) (field bits OR-ed into the mantissa of 1024.0,
-          // one LOP3 per register): the 2^(VB * pos) factor is the same for every token of a channel and is
-          // divided out once per stream; the 1024 adds 1024 * sum_t w_t to every row, which an MMA against
-          // all-ones rows accumulates in wbias and do_tiles subtracts again before it can cost precision.
+          // Codes become fp16 with one LOP3 (field bits into the mantissa of 1024.0) and one HFMA2 that strips the
+          // 1024, undoes the field's bit position and centres the code on MID: the MMA then sums p*s*(code - MID),
+          // which is small where sum p*s*code and sum p*z would cancel, and MID moves into the zero-point above.
           uint32_t vw[VW];
           load_words<VW>(sp_v + u * (NW * V_TILE_BYTES), 512, vw);
           uint32_t vh[VW];
@@ -416,15 +415,12 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
           for (int mt = 0; mt < MT; ++mt) {
             const int j = mt / (MT / NGV);
-            const uint32_t a0 = biased_pair<VB>(vw[(2 * mt) / NPOS], (2 * mt) % NPOS);
-            const uint32_t a1 = biased_pair<VB>(vw[(2 * mt + 1) / NPOS], (2 * mt + 1) % NPOS);
-            const uint32_t a2 = biased_pair<VB>(vh[(2 * mt) / NPOS], (2 * mt) % NPOS);
-            const uint32_t a3 = biased_pair<VB>(vh[(2 * mt + 1) / NPOS], (2 * mt + 1) % NPOS);
+            const uint32_t a0 = centered_pair<VB>(vw[(2 * mt) / NPOS], (2 * mt) % NPOS);
+            const uint32_t a1 = centered_pair<VB>(vw[(2 * mt + 1) / NPOS], (2 * mt + 1) % NPOS);
+            const uint32_t a2 = centered_pair<VB>(vh[(2 * mt) / NPOS], (2 * mt) % NPOS);
+            const uint32_t a3 = centered_pair<VB>(vh[(2 * mt + 1) / NPOS], (2 * mt + 1) % NPOS);
             mma16816(O[mt], a0, a1, a2, a3, bw[j][0], bw[j][1]);
           }
-#pragma unroll
-          for (int j = 0; j < NGV; ++j)
-            mma16816(wbias[j], 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, bw[j][0], bw[j][1]);
         };
 
         auto do_tiles = [&](auto masked_tag) {
@@ -432,8 +428,6 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           float L[TPW][4];
           bool v0[TPW], v1[TPW];
           float t0 = -INFINITY, t1 = -INFINITY;
-#pragma unroll
-          for (int j = 0; j < NGV; ++j) { wbias[j][0] = wbias[j][1] = wbias[j][2] = wbias[j][3] = 0.f; }
 #pragma unroll
           for (int u = 0; u < TPW; ++u) {
             const int tok0 = (warp + NW * u) * 16 + gid;        // page-local tokens of this lane's two rows
@@ -475,13 +469,6 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               values(u, v0[u], v1[u], p);
             }
           }
-          // take the 1024 * sum(w) of these tiles out of the accumulators again
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-            const int j = mt / (MT / NGV);
-#pragma unroll
-            for (int r = 0; r < 4; ++r) O[mt][r] = fmaf(-1024.f, wbias[j][r], O[mt][r]);
-          }
         };
 
         if (ntiles > warp) {                     // a short last page may leave this warp without a tile
@@ -509,10 +496,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
         const int j = mt / (MT / NGV);
-        // rows (gid, gid + 8) of m-tile mt hold channel slots k = 2 mt, 2 mt + 1: undo their 2^(VB * (k % NPOS))
-        const float f0 = 1.f / (float)(1 << (VB * ((2 * mt) % NPOS))), f1 = 1.f / (float)(1 << (VB * ((2 * mt + 1) % NPOS)));
-        O[mt][0] = fmaf(O[mt][0], f0, zacc[0][j]); O[mt][1] = fmaf(O[mt][1], f0, zacc[1][j]);
-        O[mt][2] = fmaf(O[mt][2], f1, zacc[0][j]); O[mt][3] = fmaf(O[mt][3], f1, zacc[1][j]);
+        O[mt][0] += zacc[0][j]; O[mt][1] += zacc[1][j]; O[mt][2] += zacc[0][j]; O[mt][3] += zacc[1][j];
       }
       constexpr int PER_LANE = MT * 4 + 4;
 #pragma unroll

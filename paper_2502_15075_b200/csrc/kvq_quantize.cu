@@ -35,6 +35,7 @@ __device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ 
   const float qmax = (float)((1 << BITS) - 1);
 #pragma unroll 4
   for (int step = 0; step < 16 / rps; ++step) {
+    if (step * rps + rps <= lo || step * rps >= hi) continue;      // no new token in this step's rows (warp-uniform)
     const int tau = step * rps + lane / lpr;
     const bool valid = tau >= lo && tau < hi;
     uint4 raw = make_uint4(0u, 0u, 0u, 0u);
@@ -123,6 +124,7 @@ __device__ __forceinline__ void copy_tile_side(const uint16_t* __restrict__ src,
                                                uint16_t* __restrict__ dst_rows, int lane) {
   const int lpr = D >> 3, rps = 32 / lpr, l = lane & (lpr - 1);
   for (int step = 0; step < 16 / rps; ++step) {
+    if (step * rps + rps <= lo || step * rps >= hi) continue;
     const int tau = step * rps + lane / lpr;
     if (tau >= lo && tau < hi)
       *reinterpret_cast<uint4*>(dst_rows + (size_t)tau * D + l * 8) =
