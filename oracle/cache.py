@@ -22,9 +22,14 @@ ERR_CAPACITY_BIT = 1
 
 
 class OracleCache:
-    def __init__(self, batch, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, dtype, capacity_tokens):
+    def __init__(self, batch, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, dtype, capacity_tokens, k_signs=None):
+        """k_signs: None, or +-1 per channel: keys are rotated by the randomized Hadamard transform
+        y = H (signs * x) / sqrt(D) before quantization (Sec. 4.3, key-only rotation); queries get the same
+        rotation at decode time and dequantize rotates back."""
         assert capacity_tokens % PAGE_TOKENS == 0
         assert not (k_axis == 1 and kb == 16)
+        assert k_signs is None or kb != 16
+        self.k_signs = None if k_signs is None else np.asarray(k_signs, np.int8)
         self.B, self.H, self.D = batch, n_kv_heads, head_dim
         self.dtype = dtype
         self.capacity = capacity_tokens
@@ -62,15 +67,24 @@ class OracleCache:
                         layout.put_v_codes(page, L, slots, c)
                         layout.put_v_meta_tokens(page, L, slots, s, z)
                     # keys
+                    if self.k_signs is not None:
+                        k32 = quantizer.rotate_f32(quantizer.bits_to_f32(kx, self.dtype), self.k_signs)
                     if L.k_axis == 0:
                         if L.kb == 16:
                             layout.put_k_codes(page, L, slots, kx)
                         else:
-                            c, s, z = quantizer.quantize_per_token(kx, self.dtype, L.kb, L.gk)
+                            if self.k_signs is None:
+                                c, s, z = quantizer.quantize_per_token(kx, self.dtype, L.kb, L.gk)
+                            else:
+                                c, s, z = quantizer.quantize_groups(k32.reshape(n, self.D // L.gk, L.gk), L.kb)
+                                c = c.reshape(n, self.D)
                             layout.put_k_codes(page, L, slots, c)
                             layout.put_k_meta_tokens(page, L, slots, s, z)
                     else:
-                        self.k_tail[b, h, slot:slot + n] = quantizer.to_tail_fp16_bits(kx, self.dtype)
+                        if self.k_signs is None:
+                            self.k_tail[b, h, slot:slot + n] = quantizer.to_tail_fp16_bits(kx, self.dtype)
+                        else:
+                            self.k_tail[b, h, slot:slot + n] = quantizer.f32_to_fp16_bits(k32, saturate=True)
                         if slot + n == PAGE_TOKENS:      # block complete: flush the tail
                             c, s, z = quantizer.quantize_per_channel_block(self.k_tail[b, h], L.kb)
                             layout.put_k_codes(page, L, np.arange(PAGE_TOKENS), c)
@@ -140,13 +154,16 @@ class OracleCache:
                     lo_t = max(t_begin, p * PAGE_TOKENS)
                     hi_t = min(hi, p * PAGE_TOKENS + nv)
                     sl = slice(lo_t - p * PAGE_TOKENS, hi_t - p * PAGE_TOKENS)
-                    k_out[b, h, lo_t:hi_t] = quantizer.f32_to_bits(k[sl], self.dtype)
+                    ks = k[sl] if self.k_signs is None else quantizer.unrotate_f32(k[sl], self.k_signs)
+                    k_out[b, h, lo_t:hi_t] = quantizer.f32_to_bits(ks, self.dtype)
                     v_out[b, h, lo_t:hi_t] = quantizer.f32_to_bits(v[sl], self.dtype)
 
     # ------------------------------------------------------------------ decode
     def decode(self, q_bits: np.ndarray, scale=None) -> np.ndarray:
         """q_bits uint16 [B, Hq, D] of the input dtype -> fp64 [B, Hq, D]."""
         q = quantizer.bits_to_f32(q_bits, self.dtype).astype(np.float64)
+        if self.k_signs is not None:
+            q = quantizer.hadamard_rotate_f64(q, self.k_signs)      # (H k) . (H q) = k . q
         K, V = self.values_f64()
         return attention.decode_attention(q, K, V, self.seq_len, scale)
 
@@ -155,6 +172,8 @@ class OracleCache:
         {(b, kv_head): fp64 (G, D)} (used to sample full-size workloads)."""
         import math
         q = quantizer.bits_to_f32(q_bits, self.dtype).astype(np.float64)
+        if self.k_signs is not None:
+            q = quantizer.hadamard_rotate_f64(q, self.k_signs)
         G = q.shape[1] // self.H
         sc = scale if scale and scale > 0 else 1.0 / math.sqrt(self.D)
         res = {}

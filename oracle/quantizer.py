@@ -169,3 +169,54 @@ def mse(A: np.ndarray, Ahat: np.ndarray) -> float:
     """MSE = ||A - Ahat||_F^2 / number of entries (App. B.3)."""
     d = np.asarray(A, np.float64) - np.asarray(Ahat, np.float64)
     return float(np.sum(d * d) / d.size)
+
+
+# ----------------------------------------------------------------------------
+# Randomized Hadamard rotation of keys (Sec. 4.3: rotate the keys before quantization)
+# ----------------------------------------------------------------------------
+def fwht_f32(x: np.ndarray) -> np.ndarray:
+    """Unnormalised fast Walsh-Hadamard transform along the last axis in fp32, butterfly stages
+    h = 1, 2, 4, ... in this order, (a, b) -> (a + b, a - b) with a the element whose index has bit h clear.
+    Every addition is an individually rounded fp32 operation, so the result is reproducible bit for bit."""
+    y = np.array(x, dtype=np.float32, copy=True)
+    n = y.shape[-1]
+    assert n & (n - 1) == 0
+    h = 1
+    while h < n:
+        v = y.reshape(y.shape[:-1] + (n // (2 * h), 2, h))
+        a = v[..., 0, :].copy()
+        b = v[..., 1, :].copy()
+        v[..., 0, :] = a + b
+        v[..., 1, :] = a - b
+        h *= 2
+    return y
+
+
+def rotate_f32(x32: np.ndarray, signs: np.ndarray) -> np.ndarray:
+    """y = H (signs * x) / sqrt(D) in fp32: sign flip (exact), fwht_f32, one fp32 multiplication by
+    float32(1/sqrt(D)).  `signs` is +-1 per channel.  The same map is its own inverse up to the signs:
+    x = signs * H y / sqrt(D)."""
+    D = x32.shape[-1]
+    inv = np.float32(1.0 / np.sqrt(np.float64(D)))
+    return fwht_f32(np.asarray(x32, np.float32) * signs.astype(np.float32)) * inv
+
+
+def unrotate_f32(y32: np.ndarray, signs: np.ndarray) -> np.ndarray:
+    D = y32.shape[-1]
+    inv = np.float32(1.0 / np.sqrt(np.float64(D)))
+    return (fwht_f32(np.asarray(y32, np.float32)) * inv) * signs.astype(np.float32)
+
+
+def hadamard_rotate_f64(x: np.ndarray, signs: np.ndarray) -> np.ndarray:
+    """The same rotation in exact-ish fp64 (used for queries in the fp64 attention)."""
+    y = np.array(x, dtype=np.float64, copy=True) * signs.astype(np.float64)
+    n = y.shape[-1]
+    h = 1
+    while h < n:
+        v = y.reshape(y.shape[:-1] + (n // (2 * h), 2, h))
+        a = v[..., 0, :].copy()
+        b = v[..., 1, :].copy()
+        v[..., 0, :] = a + b
+        v[..., 1, :] = a - b
+        h *= 2
+    return y / np.sqrt(np.float64(n))
