@@ -100,6 +100,12 @@ typedef struct {
   void* k_tail;     /* device fp16 tail, 16-byte aligned; NULL when k_axis == 0 */
   int32_t* seq_len; /* device [batch]: tokens stored per sequence (quantized + tail) */
   int32_t* status;  /* device, one word of KVQ_STATUS_* bits */
+  const int8_t* k_signs; /* device [head_dim] of +1 / -1, or NULL.  Not NULL: keys are rotated before
+                            quantization by y = H (signs * x) / sqrt(head_dim), H the Sylvester Hadamard matrix
+                            (Sec. 4.3, key-only rotation, which the paper finds sufficient); decode applies the
+                            same rotation to q, dequantize rotates back.  Needs kb != 16.  The transform is
+                            computed in fp32 with butterfly stages h = 1, 2, 4, ... in this order, (a, b) ->
+                            (a + b, a - b), then one multiplication by (float)(1/sqrt(head_dim)). */
 } kvq_cache;        /* one per layer.  The caller zeroes seq_len and status for a fresh cache;
                        pages must be zero-filled once before the first append. */
 

@@ -31,6 +31,7 @@ struct CachePtrs {
   uint16_t* k_tail;
   int32_t* seq_len;
   uint32_t* status;
+  const int8_t* k_signs;   // NULL: keys are not rotated
 };
 
 // Sequence length as the kernels use it: a corrupt value can never index outside the cache.
@@ -88,6 +89,54 @@ __device__ __forceinline__ uint32_t code_of_fast(float x, const GroupParams& p, 
   float u = __fmul_rn(__fsub_rn(x, p.z), p.inv);
   u = fminf(fmaxf(u, 0.0f), qmax);
   return __float_as_uint(__fadd_rn(u, 12582912.0f)) & 0xFFu;
+}
+
+// ---------------------------------------------------------------- key rotation (Sec. 4.3)
+// A token row of D channels is spread over D/8 lanes, lane l holding channels 8l..8l+7.  Unnormalised
+// Walsh-Hadamard transform with the butterfly stages in the order h = 1, 2, 4, ..., (a, b) -> (a + b, a - b)
+// where a is the element whose index has bit h clear; every addition individually rounded.
+template <int D>
+__device__ __forceinline__ void fwht_row8(float (&x)[8], int l) {
+#pragma unroll
+  for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if ((i & h) == 0) {
+        const float a = x[i], b = x[i + h];
+        x[i] = __fadd_rn(a, b);
+        x[i + h] = __fsub_rn(a, b);
+      }
+    }
+  }
+#pragma unroll
+  for (int m = 1; m < D / 8; m <<= 1) {
+    const bool upper = (l & m) != 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float o = __shfl_xor_sync(0xffffffffu, x[i], m);
+      x[i] = upper ? __fsub_rn(o, x[i]) : __fadd_rn(x[i], o);
+    }
+  }
+}
+
+template <int D> __device__ __forceinline__ constexpr float inv_sqrt_dim() { return D == 128 ? 0.08838834764831845f : 0.125f; }
+
+// y = H (signs * x) / sqrt(D)
+template <int D>
+__device__ __forceinline__ void rotate_row8(float (&x)[8], const int8_t* signs, int l) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) x[i] = __fmul_rn(x[i], (float)signs[8 * l + i]);
+  fwht_row8<D>(x, l);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) x[i] = __fmul_rn(x[i], inv_sqrt_dim<D>());
+}
+
+// x = signs * (H y / sqrt(D))
+template <int D>
+__device__ __forceinline__ void unrotate_row8(float (&x)[8], const int8_t* signs, int l) {
+  fwht_row8<D>(x, l);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) x[i] = __fmul_rn(__fmul_rn(x[i], inv_sqrt_dim<D>()), (float)signs[8 * l + i]);
 }
 
 // ---------------------------------------------------------------- layout index functions

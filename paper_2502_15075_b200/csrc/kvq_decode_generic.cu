@@ -39,7 +39,25 @@ decode_generic_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float
 
   for (int i = tid; i < G * D; i += kThreads) {
     int gh = i / D, d = i % D;
-    sq[i] = bits16_to_f32(q[((size_t)b * g.Hq + h * G + gh) * D + d], g.in_dtype) * scale_log2e;
+    float v = bits16_to_f32(q[((size_t)b * g.Hq + h * G + gh) * D + d], g.in_dtype) * scale_log2e;
+    if (c.k_signs) v *= (float)c.k_signs[d];
+    sq[i] = v;
+  }
+  if (c.k_signs) {
+    // rotated keys: q' = H (signs * q) / sqrt(D), butterflies in shared memory
+    for (int hh = 1; hh < D; hh <<= 1) {
+      __syncthreads();
+      for (int i = tid; i < G * D / 2; i += kThreads) {
+        const int gh = i / (D / 2), p = i % (D / 2);
+        const int d0 = (p / hh) * 2 * hh + (p % hh);
+        const float a = sq[gh * D + d0], bq = sq[gh * D + d0 + hh];
+        sq[gh * D + d0] = a + bq;
+        sq[gh * D + d0 + hh] = a - bq;
+      }
+    }
+    __syncthreads();
+    const float inv = rsqrtf((float)D);
+    for (int i = tid; i < G * D; i += kThreads) sq[i] *= inv;
   }
   float m[kMaxGroupHeads], l[kMaxGroupHeads], o[kMaxGroupHeads];
   for (int gh = 0; gh < kMaxGroupHeads; ++gh) { m[gh] = -INFINITY; l[gh] = 0.f; o[gh] = 0.f; }

@@ -124,6 +124,14 @@ __device__ __forceinline__ uint32_t h2fma(uint32_t a, uint32_t b, uint32_t c) {
 }
 __device__ __forceinline__ uint32_t pack_h2(float lo, float hi) { return as_u32(__floats2half2_rn(lo, hi)); }
 
+// (a, b) in fp32 -> fp16 pairs hi and lo with hi + lo = (a, b) to 22 bits: hi = fp16(x), lo = fp16(x - hi).
+__device__ __forceinline__ void split_h2(float a, float b, uint32_t& hi, uint32_t& lo) {
+  const __half2 h = __floats2half2_rn(a, b);
+  const float2 hf = __half22float2(h);
+  hi = as_u32(h);
+  lo = as_u32(__floats2half2_rn(a - hf.x, b - hf.y));
+}
+
 // ------------------------------------------------------------------ code -> fp16 conversion
 // A word holds 32/B fields; pair i = (field i, field i + 16/B) becomes one half2 register holding the two
 // codes as exact fp16 integers: the field bits are OR-ed into the mantissa of 1024.0 (0x6400), which yields

@@ -172,7 +172,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   // q operands: signed-byte limbs (token-wise keys) or fp16 pairs (channel-wise keys), heads >= G are zero.
   // Slot r holds channels 16 r + 4 tid + {0..3} of head gid.
   uint32_t ql[(KAXIS == 0) ? NL : 1][(KAXIS == 0) ? NR : 1];
-  uint32_t qf[(KAXIS == 1) ? 2 * NR : 1];    // fp16 pairs (j = 0, 2) and (j = 1, 3) of slot r
+  float qk[(KAXIS == 1) ? NR : 1][4];        // channel-wise keys: q (rotated if asked) in fp32, kept for the stream
   float qsum[2][NGK];                        // c1 * sum of q over each key group, heads (2 tid, 2 tid + 1)
   float hs0 = 0.f, hs1 = 0.f;                // c1 / fixed-point scale of heads (2 tid, 2 tid + 1)
   float O[MT][4];
@@ -205,21 +205,56 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       for (int r = 0; r < NR; ++r) {
         uint2 raw = make_uint2(0u, 0u);
         if (gid < G) raw = *reinterpret_cast<const uint2*>(qrow + 16 * r + 4 * tid);
-        float f[4];
-        f[0] = bits16_to_f32((uint16_t)(raw.x & 0xFFFF), g.in_dtype);
-        f[1] = bits16_to_f32((uint16_t)(raw.x >> 16), g.in_dtype);
-        f[2] = bits16_to_f32((uint16_t)(raw.y & 0xFFFF), g.in_dtype);
-        f[3] = bits16_to_f32((uint16_t)(raw.y >> 16), g.in_dtype);
-        if constexpr (KAXIS == 1) {
-          // the tensor core sees q rounded to fp16: keep the sums consistent with that
-          qf[2 * r] = pack_h2(f[0], f[2]);
-          qf[2 * r + 1] = pack_h2(f[1], f[3]);
-          const float2 a = __half22float2(as_h2(qf[2 * r])), bb = __half22float2(as_h2(qf[2 * r + 1]));
-          f[0] = a.x; f[2] = a.y; f[1] = bb.x; f[3] = bb.y;
+        qv[r][0] = bits16_to_f32((uint16_t)(raw.x & 0xFFFF), g.in_dtype);
+        qv[r][1] = bits16_to_f32((uint16_t)(raw.x >> 16), g.in_dtype);
+        qv[r][2] = bits16_to_f32((uint16_t)(raw.y & 0xFFFF), g.in_dtype);
+        qv[r][3] = bits16_to_f32((uint16_t)(raw.y >> 16), g.in_dtype);
+      }
+      if (c.k_signs != nullptr) {
+        // rotated keys: give q the same rotation, q' = H (signs * q) / sqrt(D); channel 16 r + 4 tid + j,
+        // so the butterflies run over j inside the lane, over tid across lanes, over r inside the lane
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) qv[r][j] *= (float)c.k_signs[16 * r + 4 * tid + j];
+          float a = qv[r][0], bq = qv[r][1], cq = qv[r][2], dq = qv[r][3];
+          qv[r][0] = (a + bq) + (cq + dq); qv[r][1] = (a - bq) + (cq - dq);
+          qv[r][2] = (a + bq) - (cq + dq); qv[r][3] = (a - bq) - (cq - dq);
+#pragma unroll
+          for (int m = 1; m < 4; m <<= 1) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float o = __shfl_xor_sync(FULL, qv[r][j], m);
+              qv[r][j] = (tid & m) ? o - qv[r][j] : qv[r][j] + o;
+            }
+          }
         }
 #pragma unroll
+        for (int hh = 1; hh < NR; hh <<= 1) {
+#pragma unroll
+          for (int r = 0; r < NR; ++r) {
+            if ((r & hh) == 0) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float a = qv[r][j], bq = qv[r + hh][j];
+                qv[r][j] = a + bq;
+                qv[r + hh][j] = a - bq;
+              }
+            }
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) qv[r][j] *= inv_sqrt_dim<D>();
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < NR; ++r) {
+        float f[4] = {qv[r][0], qv[r][1], qv[r][2], qv[r][3]};
+#pragma unroll
         for (int j = 0; j < 4; ++j) {
-          qv[r][j] = f[j];
+          if constexpr (KAXIS == 1) qk[r][j] = f[j];
           amax = fmaxf(amax, fabsf(f[j]));
           part[r / (NR / NGK)] += f[j];
         }
@@ -290,24 +325,32 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
         const int ntiles = (nv + 15) >> 4;
 
-        // ---- channel-wise keys: per page, fold the channel scales into q and get sum_d q_d z_d by one more mma
-        uint32_t qs[(KAXIS == 1) ? 2 * NR : 1];
+        // ---- channel-wise keys: per page, q_d * s_d in fp32 split into an fp16 high and low part (the product
+        // has 22 significant bits; one fp16 alone would cost 2^-12 of every logit term), and sum_d q_d z_d in fp32
+        uint32_t qs_hi[(KAXIS == 1) ? 2 * NR : 1], qs_lo[(KAXIS == 1) ? 2 * NR : 1];
         float zq0 = 0.f, zq1 = 0.f;
         if constexpr (KAXIS == 1) {
           if (!tail_k) {
             const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
-            float sz[4] = {0.f, 0.f, 0.f, 0.f};
+            float zsum = 0.f;
 #pragma unroll
             for (int r = 0; r < NR; ++r) {
               const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);   // (s,z) of 4 channels
-              const uint32_t s02 = __byte_perm(mm.x, mm.z, 0x5410), s13 = __byte_perm(mm.y, mm.w, 0x5410);
-              const uint32_t z02 = __byte_perm(mm.x, mm.z, 0x7632), z13 = __byte_perm(mm.y, mm.w, 0x7632);
-              qs[2 * r] = as_u32(__hmul2(as_h2(qf[2 * r]), as_h2(s02)));
-              qs[2 * r + 1] = as_u32(__hmul2(as_h2(qf[2 * r + 1]), as_h2(s13)));
-              mma16816(sz, z02, z02, z13, z13, qf[2 * r], qf[2 * r + 1]);
+              const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
+              float t[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 sz = __half22float2(as_h2(mw[j]));
+                t[j] = qk[r][j] * sz.x;
+                zsum = fmaf(qk[r][j], sz.y, zsum);
+              }
+              split_h2(t[0], t[2], qs_hi[2 * r], qs_lo[2 * r]);
+              split_h2(t[1], t[3], qs_hi[2 * r + 1], qs_lo[2 * r + 1]);
             }
-            zq0 = c1 * sz[0];
-            zq1 = c1 * sz[1];
+            zsum += __shfl_xor_sync(FULL, zsum, 1);
+            zsum += __shfl_xor_sync(FULL, zsum, 2);
+            zq0 = c1 * __shfl_sync(FULL, zsum, (2 * tid) * 4);
+            zq1 = c1 * __shfl_sync(FULL, zsum, (2 * tid + 1) * 4);
           }
         }
 
@@ -323,8 +366,13 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
                 uint2 ra = make_uint2(0u, 0u), rb = make_uint2(0u, 0u);
                 if (v0) ra = *reinterpret_cast<const uint2*>(tl + 16 * r + 4 * tid);
                 if (v1) rb = *reinterpret_cast<const uint2*>(tl + 8 * D + 16 * r + 4 * tid);
-                mma16816(S[r & 1], __byte_perm(ra.x, ra.y, 0x5410), __byte_perm(rb.x, rb.y, 0x5410),
-                         __byte_perm(ra.x, ra.y, 0x7632), __byte_perm(rb.x, rb.y, 0x7632), qf[2 * r], qf[2 * r + 1]);
+                uint32_t h0, l0_, h1, l1_;       // q as fp16 high + low parts
+                split_h2(qk[r][0], qk[r][2], h0, l0_);
+                split_h2(qk[r][1], qk[r][3], h1, l1_);
+                const uint32_t a0 = __byte_perm(ra.x, ra.y, 0x5410), a1 = __byte_perm(rb.x, rb.y, 0x5410);
+                const uint32_t a2 = __byte_perm(ra.x, ra.y, 0x7632), a3 = __byte_perm(rb.x, rb.y, 0x7632);
+                mma16816(S[r & 1], a0, a1, a2, a3, h0, h1);
+                mma16816(S[r & 1], a0, a1, a2, a3, l0_, l1_);
               }
 #pragma unroll
               for (int i = 0; i < 4; ++i) L[i] = c1 * (S[0][i] + S[1][i]);
@@ -341,7 +389,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
                 for (int i = 0; i < FPB; ++i) {
                   const int r = w * FPB + i;       // pairs (j = 0, 2) sit in output i, (j = 1, 3) in output FPB + i
-                  mma16816(S[r & 1], pa[i], pb[i], pa[FPB + i], pb[FPB + i], qs[2 * r], qs[2 * r + 1]);
+                  mma16816(S[r & 1], pa[i], pb[i], pa[FPB + i], pb[FPB + i], qs_hi[2 * r], qs_hi[2 * r + 1]);
+                  mma16816(S[r & 1], pa[i], pb[i], pa[FPB + i], pb[FPB + i], qs_lo[2 * r], qs_lo[2 * r + 1]);
                 }
               }
               L[0] = fmaf(c1, S[0][0] + S[1][0], zq0); L[1] = fmaf(c1, S[0][1] + S[1][1], zq1);

@@ -79,6 +79,66 @@ __device__ __forceinline__ void expand_values(const uint8_t* spage, const Geom& 
   }
 }
 
+// Rotated keys: reconstruct rows [lo, hi) in fp32, rotate back (x = signs * H y / sqrt(D)) and store 16-bit rows.
+// A row is handled by D/8 consecutive lanes, lane l owning channels 8l..8l+7 (two code words of 4 channels each).
+template <int B, int D>
+__device__ __forceinline__ void dequant_keys_rotated(const uint8_t* spage, const Geom& g, const uint16_t* tail,
+                                                     const int8_t* signs, uint16_t* out, int lo, int hi, int tid) {
+  constexpr int FPB = 8 / B, LPR = D / 8, RPI = kThreads / LPR;     // rows per iteration of the CTA
+  constexpr int wpc = D * B / 128;
+  const uint32_t* meta = reinterpret_cast<const uint32_t*>(spage + g.k_meta_off);
+  const int lgk = ilog2(g.gk), ngk = D >> lgk;
+  const int l = tid % LPR;
+  for (int t0 = lo; t0 < hi; t0 += RPI) {
+    const int t = t0 + tid / LPR;
+    const bool active = t < hi;
+    float x[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = 0.f;
+    if (active) {
+      if (tail) {
+        const uint4 raw = *reinterpret_cast<const uint4*>(tail + (size_t)t * D + 8 * l);
+        const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&rw[i]));
+          x[2 * i] = f.x;
+          x[2 * i + 1] = f.y;
+        }
+      } else {
+        const int r = l >> 1, word = r / FPB, sh = B * (r % FPB);
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          const int chunk = 2 * (l & 1) + hh;
+          const uint32_t w = *reinterpret_cast<const uint32_t*>(spage + (size_t)t * (D * B / 8) +
+                                                                 chunk_word_byte(chunk, word, wpc, 4));
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int d = 8 * l + 4 * hh + j;
+            const uint32_t m = meta[g.k_axis == 1 ? d : t * ngk + (d >> lgk)];
+            x[4 * hh + j] = fmaf((float)((w >> (8 * j + sh)) & ((1u << B) - 1u)), meta_scale(m), meta_zero(m));
+          }
+        }
+      }
+    }
+    unrotate_row8<D>(x, signs, l);
+    if (active) {
+      uint32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        o[i] = (uint32_t)f32_to_bits16(x[2 * i], g.in_dtype) | ((uint32_t)f32_to_bits16(x[2 * i + 1], g.in_dtype) << 16);
+      *reinterpret_cast<uint4*>(out + (size_t)t * D + 8 * l) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  }
+}
+
+template <int B>
+__device__ __forceinline__ void dequant_keys_rotated_d(const uint8_t* spage, const Geom& g, const uint16_t* tail,
+                                                       const int8_t* signs, uint16_t* out, int lo, int hi, int tid) {
+  if (g.D == 128) dequant_keys_rotated<B, 128>(spage, g, tail, signs, out, lo, hi, tid);
+  else dequant_keys_rotated<B, 64>(spage, g, tail, signs, out, lo, hi, tid);
+}
+
 // Copy token rows [lo, hi) of tile[128][D] to out rows (16-byte vectors).
 __device__ __forceinline__ void store_rows(const uint16_t* tile, uint16_t* out, int D, int lo, int hi, int tid) {
   const int vpr = D / 8, lv = ilog2(vpr);
@@ -128,7 +188,12 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
   }
   if (k_out) {
     const bool tail_k = (g.k_axis == 1) && (nv < kPageTokens);
-    if (tail_k) {
+    if (c.k_signs) {
+      const uint16_t* tail = tail_k ? c.k_tail + (size_t)bh * kPageTokens * D : nullptr;
+      if (g.kb == 2) dequant_keys_rotated_d<2>(spage, g, tail, c.k_signs, k_out + out_base, lo, hi_l, tid);
+      else if (g.kb == 4) dequant_keys_rotated_d<4>(spage, g, tail, c.k_signs, k_out + out_base, lo, hi_l, tid);
+      else dequant_keys_rotated_d<8>(spage, g, tail, c.k_signs, k_out + out_base, lo, hi_l, tid);
+    } else if (tail_k) {
       // keys of an incomplete channel-wise block live in the fp16 tail
       const uint16_t* tail = c.k_tail + (size_t)bh * kPageTokens * D;
       const int lD = ilog2(D);

@@ -55,6 +55,8 @@ int make_cache(const Geom& g, const kvq_cache* cache, CachePtrs* out) {
   out->k_tail = static_cast<uint16_t*>(cache->k_tail);
   out->seq_len = cache->seq_len;
   out->status = reinterpret_cast<uint32_t*>(cache->status);
+  out->k_signs = cache->k_signs;
+  if (cache->k_signs && g.kb == 16) return KVQ_ERR_UNSUPPORTED;   // rotation applies to quantized keys only
   return KVQ_OK;
 }
 

@@ -22,10 +22,11 @@ constexpr uint32_t FULL = 0xffffffffu;
 // Quantize one side (keys or values) of a 16-token tile held in global memory as rows of D 16-bit values.
 // `img` is the warp's shared-memory image of the packed codes of the tile: for keys 16 token rows of
 // D*BITS/8 bytes, for values the tile's D*BITS*2 bytes.  Tokens outside [lo, hi) are left alone.
-template <int BITS, bool IS_V, int D, int DTYPE>
+template <int BITS, bool IS_V, int D, int DTYPE, bool ROT>
 __device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ src, int64_t st, int gsz,
                                                    int lo, int hi, uint32_t* img,
-                                                   uint32_t* __restrict__ meta_out, bool clear_first, int lane) {
+                                                   uint32_t* __restrict__ meta_out, bool clear_first, int lane,
+                                                   const int8_t* __restrict__ signs) {
   constexpr int lpr = D >> 3;                // lanes per token row (8 channels each)
   constexpr int rps = 32 / lpr;              // rows per step
   const int l = lane & (lpr - 1);
@@ -42,7 +43,6 @@ __device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ 
     if (valid) raw = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + d0);
     const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
     float x[8];
-    float mn = INFINITY, mx = -INFINITY;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       if constexpr (DTYPE == KVQ_BF16) {
@@ -53,8 +53,13 @@ __device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ 
         x[2 * i] = f.x;
         x[2 * i + 1] = f.y;
       }
-      mn = fminf(mn, fminf(x[2 * i], x[2 * i + 1]));
-      mx = fmaxf(mx, fmaxf(x[2 * i], x[2 * i + 1]));
+    }
+    if constexpr (ROT) rotate_row8<D>(x, signs, l);      // keys only: y = H (signs * x) / sqrt(D)
+    float mn = INFINITY, mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      mn = fminf(mn, x[i]);
+      mx = fmaxf(mx, x[i]);
     }
 #pragma unroll
     for (int off = 1; off < 16; off <<= 1) {
@@ -132,13 +137,16 @@ __device__ __forceinline__ void copy_tile_side(const uint16_t* __restrict__ src,
   }
 }
 
-template <bool IS_V, int D, int DTYPE>
+template <bool IS_V, int D, int DTYPE, bool ROT>
 __device__ __forceinline__ void quantize_tile_side_bits(int bits, const uint16_t* src, int64_t st, int gsz,
                                                         int lo, int hi, uint32_t* img, uint32_t* meta_out,
-                                                        bool clear_first, int lane) {
-  if (bits == 2) quantize_tile_side<2, IS_V, D, DTYPE>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane);
-  else if (bits == 4) quantize_tile_side<4, IS_V, D, DTYPE>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane);
-  else quantize_tile_side<8, IS_V, D, DTYPE>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane);
+                                                        bool clear_first, int lane, const int8_t* signs) {
+  if (bits == 2)
+    quantize_tile_side<2, IS_V, D, DTYPE, ROT>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane, signs);
+  else if (bits == 4)
+    quantize_tile_side<4, IS_V, D, DTYPE, ROT>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane, signs);
+  else
+    quantize_tile_side<8, IS_V, D, DTYPE, ROT>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane, signs);
 }
 
 // Token-wise quantization of V (always) and of K (when do_k).  grid.y = stream, grid.x strides over the
@@ -178,8 +186,9 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
       for (int i = lane; i < v_tile_words / 4; i += 32)
         reinterpret_cast<uint4*>(vimg)[i] = full ? make_uint4(0u, 0u, 0u, 0u) : gv[i];
       __syncwarp();
-      quantize_tile_side_bits<true, D, DTYPE>(g.vb, v_new + off, st, g.gv, lo, hi, vimg,
-                                    reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / g.gv), !full, lane);
+      quantize_tile_side_bits<true, D, DTYPE, false>(g.vb, v_new + off, st, g.gv, lo, hi, vimg,
+                                    reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / g.gv), !full, lane,
+                                    nullptr);
       __syncwarp();
       for (int i = lane; i < v_tile_words / 4; i += 32) gv[i] = reinterpret_cast<const uint4*>(vimg)[i];
     }
@@ -190,8 +199,13 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
       } else {
         for (int i = lane; i < 16 * k_row_words / 4; i += 32) reinterpret_cast<uint4*>(kimg)[i] = make_uint4(0u, 0u, 0u, 0u);
         __syncwarp();
-        quantize_tile_side_bits<false, D, DTYPE>(g.kb, k_new + off, st, g.gk, lo, hi, kimg,
-                                       reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / g.gk), false, lane);
+        uint32_t* kmeta = reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / g.gk);
+        if (c.k_signs)
+          quantize_tile_side_bits<false, D, DTYPE, true>(g.kb, k_new + off, st, g.gk, lo, hi, kimg, kmeta, false,
+                                                         lane, c.k_signs);
+        else
+          quantize_tile_side_bits<false, D, DTYPE, false>(g.kb, k_new + off, st, g.gk, lo, hi, kimg, kmeta, false,
+                                                          lane, nullptr);
         __syncwarp();
         uint4* gk = reinterpret_cast<uint4*>(pg + (size_t)tp0 * (k_row_words * 4));
         const int v_lo = lo * k_row_words / 4, v_hi = hi * k_row_words / 4;   // 16-byte vectors of the new rows
@@ -259,26 +273,39 @@ quant_kchan_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new,
     const int lo = max(t0, tb) - tb, hi = min(end, tb + 128) - tb;   // new tokens occupy slots [lo, hi)
     const bool complete = (hi == 128);
     // gather the block: slots [0, lo) from the tail, [lo, hi) from the input (as saturated fp16)
+    // (a row is handled by D/8 consecutive lanes, which is what the rotation's shuffles expect; every lane of a
+    // warp runs the loop body, rows past the end are inactive)
     const int vec_per_row = D / 8;   // 16-byte vectors
-    for (int idx = tid; idx < hi * vec_per_row; idx += kThreads) {
-      int slot = idx / vec_per_row, v = idx % vec_per_row;
-      uint4 val;
-      if (slot < lo) {
-        val = *reinterpret_cast<const uint4*>(tail + (size_t)slot * D + v * 8);
-      } else {
-        const uint16_t* src = k_new + (int64_t)b * sb + (int64_t)h * sh + (int64_t)(tb + slot - t0) * st + v * 8;
-        val = *reinterpret_cast<const uint4*>(src);
-        if (g.in_dtype == KVQ_BF16) {
-          uint32_t* w = reinterpret_cast<uint32_t*>(&val);
-          for (int i = 0; i < 4; ++i) {
-            uint16_t a = f32_to_fp16_sat_bits(bits16_to_f32(w[i] & 0xFFFF, KVQ_BF16));
-            uint16_t bb = f32_to_fp16_sat_bits(bits16_to_f32(w[i] >> 16, KVQ_BF16));
-            w[i] = (uint32_t)a | ((uint32_t)bb << 16);
-          }
+    for (int base = 0; base < hi * vec_per_row; base += kThreads) {
+      const int idx = base + tid;
+      const bool active = idx < hi * vec_per_row;
+      const int slot = idx / vec_per_row, v = idx % vec_per_row;
+      uint4 val = make_uint4(0u, 0u, 0u, 0u);
+      const bool is_new = active && slot >= lo;
+      if (active && !is_new) val = *reinterpret_cast<const uint4*>(tail + (size_t)slot * D + v * 8);
+      if (is_new)
+        val = *reinterpret_cast<const uint4*>(k_new + (int64_t)b * sb + (int64_t)h * sh +
+                                              (int64_t)(tb + slot - t0) * st + v * 8);
+      if (c.k_signs != nullptr || g.in_dtype == KVQ_BF16) {
+        // new tokens: to fp32, rotate if asked, store as saturated fp16
+        uint32_t* w = reinterpret_cast<uint32_t*>(&val);
+        float x[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          x[2 * i] = bits16_to_f32((uint16_t)(w[i] & 0xFFFF), g.in_dtype);
+          x[2 * i + 1] = bits16_to_f32((uint16_t)(w[i] >> 16), g.in_dtype);
         }
-        if (!complete) *reinterpret_cast<uint4*>(tail + (size_t)slot * D + v * 8) = val;
+        if (c.k_signs != nullptr) {
+          if (D == 128) rotate_row8<128>(x, c.k_signs, v); else rotate_row8<64>(x, c.k_signs, v);
+        }
+        if (is_new) {
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            w[i] = (uint32_t)f32_to_fp16_sat_bits(x[2 * i]) | ((uint32_t)f32_to_fp16_sat_bits(x[2 * i + 1]) << 16);
+        }
       }
-      *reinterpret_cast<uint4*>(sX + (size_t)slot * D + v * 8) = val;
+      if (is_new && !complete) *reinterpret_cast<uint4*>(tail + (size_t)slot * D + v * 8) = val;
+      if (active) *reinterpret_cast<uint4*>(sX + (size_t)slot * D + v * 8) = val;
     }
     if (!complete) continue;
     __syncthreads();

@@ -34,7 +34,7 @@ class kvq_config(ctypes.Structure):
 
 class kvq_cache(ctypes.Structure):
     _fields_ = [("pages", ctypes.c_void_p), ("k_tail", ctypes.c_void_p),
-                ("seq_len", ctypes.c_void_p), ("status", ctypes.c_void_p)]
+                ("seq_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("k_signs", ctypes.c_void_p)]
 
 
 _P = ctypes.POINTER
@@ -118,15 +118,19 @@ def kvq_workspace_bytes(cfg: kvq_config) -> int:
 class Cache:
     """Caller-owned buffers of one layer's packed cache (torch tensors) plus the POD handed to the library."""
 
-    def __init__(self, cfg: kvq_config, device="cuda"):
+    def __init__(self, cfg: kvq_config, device="cuda", k_signs: Optional[torch.Tensor] = None):
+        """k_signs: optional int8 tensor [head_dim] of +1 / -1: rotate the keys (randomized Hadamard)."""
         self.cfg = cfg
+        self.k_signs = None if k_signs is None else k_signs.to(device=device, dtype=torch.int8).contiguous()
+        assert self.k_signs is None or self.k_signs.numel() == cfg.head_dim
         pages_bytes, tail_bytes = kvq_cache_bytes(cfg)
         self.pages = torch.zeros(pages_bytes, dtype=torch.uint8, device=device)
         self.k_tail = torch.zeros(tail_bytes // 2, dtype=torch.float16, device=device) if tail_bytes else None
         self.seq_len = torch.zeros(cfg.batch, dtype=torch.int32, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.c = kvq_cache(self.pages.data_ptr(), self.k_tail.data_ptr() if self.k_tail is not None else None,
-                           self.seq_len.data_ptr(), self.status.data_ptr())
+                           self.seq_len.data_ptr(), self.status.data_ptr(),
+                           self.k_signs.data_ptr() if self.k_signs is not None else None)
 
     def pages_view(self) -> torch.Tensor:
         c = self.cfg

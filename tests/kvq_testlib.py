@@ -16,8 +16,9 @@ def bits_of(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-def oracle_cache_for(w: wl.Workload, batch: int, capacity: int) -> OracleCache:
-    return OracleCache(batch, w.n_kv_heads, w.head_dim, w.kb, w.vb, w.gk, w.gv, w.k_axis, w.dtype, capacity)
+def oracle_cache_for(w: wl.Workload, batch: int, capacity: int, k_signs=None) -> OracleCache:
+    return OracleCache(batch, w.n_kv_heads, w.head_dim, w.kb, w.vb, w.gk, w.gv, w.k_axis, w.dtype, capacity,
+                       k_signs=k_signs)
 
 
 def gpu_config_for(kvq, w: wl.Workload, batch: int, capacity: int):
@@ -25,12 +26,13 @@ def gpu_config_for(kvq, w: wl.Workload, batch: int, capacity: int):
                            w.torch_dtype, capacity)
 
 
-def build_both(kvq, w: wl.Workload, k: torch.Tensor, v: torch.Tensor, chunks, capacity: int):
-    """Append k, v ([B,Hkv,T,D] CPU tensors) in the given chunk sizes through both paths."""
+def build_both(kvq, w: wl.Workload, k: torch.Tensor, v: torch.Tensor, chunks, capacity: int, k_signs=None):
+    """Append k, v ([B,Hkv,T,D] CPU tensors) in the given chunk sizes through both paths.
+    k_signs: optional +-1 per channel (numpy int8): rotate the keys on both sides."""
     B = k.shape[0]
     cfg = gpu_config_for(kvq, w, B, capacity)
-    gc = kvq.Cache(cfg)
-    oc = oracle_cache_for(w, B, capacity)
+    gc = kvq.Cache(cfg, k_signs=None if k_signs is None else torch.from_numpy(k_signs))
+    oc = oracle_cache_for(w, B, capacity, k_signs)
     kd, vd = k.cuda(), v.cuda()
     kb_, vb_ = bits_of(k), bits_of(v)
     t = 0
@@ -61,7 +63,8 @@ def oracle_on_gpu_codes(gc, w: wl.Workload) -> OracleCache:
     """An oracle cache that holds exactly the bytes the GPU produced (attention parity is measured on the
     same codes)."""
     cfg = gc.cfg
-    oc = oracle_cache_for(w, cfg.batch, cfg.capacity_tokens)
+    oc = oracle_cache_for(w, cfg.batch, cfg.capacity_tokens,
+                          None if gc.k_signs is None else gc.k_signs.cpu().numpy())
     oc.pages = gc.pages_view().cpu().numpy().copy()
     if oc.k_tail is not None:
         oc.k_tail = gc.tail_view().cpu().view(torch.int16).numpy().view(np.uint16).copy()
