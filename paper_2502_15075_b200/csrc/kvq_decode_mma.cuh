@@ -132,6 +132,24 @@ __device__ __forceinline__ void split_h2(float a, float b, uint32_t& hi, uint32_
   lo = as_u32(__floats2half2_rn(a - hf.x, b - hf.y));
 }
 
+// Four values times `scale` rounded to integers |Q| < 2^22 and split into three balanced signed bytes,
+// Q = b0 * 65536 + b1 * 256 + b2; byte j of w0 / w1 / w2 is b0 / b1 / b2 of t[j] (an s8 MMA operand each).
+__device__ __forceinline__ void fixed_point_limbs(const float (&t)[4], float scale, uint32_t& w0, uint32_t& w1,
+                                                  uint32_t& w2) {
+  w0 = w1 = w2 = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int Q = __float2int_rn(t[j] * scale);
+    const int b2 = (int)(int8_t)(Q & 0xFF);
+    const int Q1 = (Q - b2) >> 8;
+    const int b1 = (int)(int8_t)(Q1 & 0xFF);
+    const int b0 = (Q1 - b1) >> 8;
+    w0 |= (uint32_t)(b0 & 0xFF) << (8 * j);
+    w1 |= (uint32_t)(b1 & 0xFF) << (8 * j);
+    w2 |= (uint32_t)(b2 & 0xFF) << (8 * j);
+  }
+}
+
 // ------------------------------------------------------------------ code -> fp16 conversion
 // A word holds 32/B fields; pair i = (field i, field i + 16/B) becomes one half2 register holding the two
 // codes as exact fp16 integers: the field bits are OR-ed into the mantissa of 1024.0 (0x6400), which yields

@@ -31,9 +31,11 @@ __device__ __forceinline__ FlatPlan make_plan(long long N, int pages_max, int gr
 
 // Shared-memory carve-up (dynamic): ring | barriers | prefix | combine buffer
 struct SmemLayout {
-  int page_stride, ring_bytes, bar_off, pref_off, misc_off, comb_off, total;
+  int page_stride, ring_bytes, bar_off, pref_off, misc_off, comb_off, chan_off, total;
 };
-__host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, int nw, int D) {
+// chan: channel-wise keys need, per CTA, two buffers of per-page q limbs (3 x D/16 x 32 words), the partial
+// zero-point sums (64 floats) and the stream's q in fp32 (D/16 x 32 x 4 floats).
+__host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, int nw, int D, bool chan) {
   SmemLayout s;
   s.page_stride = (page_bytes + 127) & ~127;
   s.ring_bytes = s.page_stride * stages;
@@ -42,7 +44,8 @@ __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, in
   s.misc_off = s.pref_off + (kMaxBatchFlat + 1) * 4;
   s.comb_off = (s.misc_off + 64 + 127) & ~127;
   int per_warp = (D / 16 * 4 + 4) * 32 * 4;                 // O fragments + m, l per lane
-  s.total = s.comb_off + (nw / 2 > 0 ? nw / 2 : 1) * per_warp;
+  s.chan_off = s.comb_off + (nw / 2 > 0 ? nw / 2 : 1) * per_warp;
+  s.total = s.chan_off + (chan ? (2 * 3 * (D / 16) * 32 * 4 + 2 * 64 * 4 + (D / 16) * 32 * 16) : 0);
   return s;
 }
 
@@ -69,7 +72,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   static_assert(KAXIS == 0 || KB != 2, "channel-wise 2-bit keys are not instantiated");
 
   extern __shared__ __align__(128) uint8_t smem[];
-  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D);
+  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D, KAXIS == 1);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sl.bar_off);   // full[0..stages), empty[0..stages)
   int* sPref = reinterpret_cast<int*>(smem + sl.pref_off);
   int* sMisc = reinterpret_cast<int*>(smem + sl.misc_off);           // [0] pages_max, [1] abort flag
@@ -171,8 +174,14 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   // =========================================================== consumer warps
   // q operands: signed-byte limbs (token-wise keys) or fp16 pairs (channel-wise keys), heads >= G are zero.
   // Slot r holds channels 16 r + 4 tid + {0..3} of head gid.
-  uint32_t ql[(KAXIS == 0) ? NL : 1][(KAXIS == 0) ? NR : 1];
-  float qk[(KAXIS == 1) ? NR : 1][4];        // channel-wise keys: q (rotated if asked) in fp32, kept for the stream
+  uint32_t ql[NL][NR];
+  constexpr int OWN = (NR / NW > 0) ? NR / NW : 1;     // channel-wise keys: slots whose per-page limbs this warp makes
+  float qk[(KAXIS == 1) ? OWN : 1][4];       // ... and the stream's q (rotated if asked) on those slots, fp32
+  float amax_h = 0.f;                        // ... and max |q| of head gid
+  uint32_t* sB = reinterpret_cast<uint32_t*>(smem + sl.chan_off);          // [2][NL][NR][32] per-page q limbs
+  float* sZ = reinterpret_cast<float*>(smem + sl.chan_off + 2 * NL * NR * 32 * 4);   // [2][8 heads][8] partial sums
+  float4* sQ = reinterpret_cast<float4*>(smem + sl.chan_off + 2 * NL * NR * 32 * 4 + 2 * 64 * 4);   // [NR][32]
+  int page_no = 0;
   float qsum[2][NGK];                        // c1 * sum of q over each key group, heads (2 tid, 2 tid + 1)
   float hs0 = 0.f, hs1 = 0.f;                // c1 / fixed-point scale of heads (2 tid, 2 tid + 1)
   float O[MT][4];
@@ -254,17 +263,36 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         float f[4] = {qv[r][0], qv[r][1], qv[r][2], qv[r][3]};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          if constexpr (KAXIS == 1) qk[r][j] = f[j];
           amax = fmaxf(amax, fabsf(f[j]));
           part[r / (NR / NGK)] += f[j];
         }
       }
+      static_assert(NL == 3, "three signed 8-bit limbs");
+      amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 1));
+      amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 2));
+      if constexpr (KAXIS == 1) {
+        // channel-wise keys: the limbs depend on the page's scales and are made per page; keep what that needs
+        amax_h = amax;
+#pragma unroll
+        for (int i = 0; i < OWN; ++i) {
+#pragma unroll
+          for (int r = 0; r < NR; ++r) {       // (compile-time indices keep qv in registers)
+            if (r == warp * OWN + i) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) qk[i][j] = qv[r][j];
+            }
+          }
+        }
+        named_bar_sync(2, NCONS);                       // nobody still reads the previous stream's copy
+        if (warp == 0) {
+#pragma unroll
+          for (int r = 0; r < NR; ++r) sQ[r * 32 + lane] = make_float4(qv[r][0], qv[r][1], qv[r][2], qv[r][3]);
+        }
+        named_bar_sync(2, NCONS);
+      }
       if constexpr (KAXIS == 0) {
         // per head: 22-bit fixed point relative to the head's largest entry, Q = rint(q * 2^k) with
         // |Q| < 2^22, split into three balanced signed bytes  Q = l0 * 65536 + l1 * 256 + l2
-        static_assert(NL == 3, "three signed 8-bit limbs");
-        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 1));
-        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 2));
         int e = (int)((__float_as_uint(amax) >> 23) & 0xFF) - 127;
         e = max(e, -60);
         const int k = 21 - e;
@@ -272,19 +300,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         const float hs = c1 * __uint_as_float((uint32_t)(127 - k) << 23);
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
-          uint32_t w0 = 0, w1 = 0, w2 = 0;
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int Q = __float2int_rn(qv[r][j] * scale);
-            const int b2 = (int)(int8_t)(Q & 0xFF);
-            const int Q1 = (Q - b2) >> 8;
-            const int b1 = (int)(int8_t)(Q1 & 0xFF);
-            const int b0 = (Q1 - b1) >> 8;
-            w0 |= (uint32_t)(b0 & 0xFF) << (8 * j);
-            w1 |= (uint32_t)(b1 & 0xFF) << (8 * j);
-            w2 |= (uint32_t)(b2 & 0xFF) << (8 * j);
-          }
-          ql[0][r] = w0; ql[1][r] = w1; ql[2][r] = w2;
+          fixed_point_limbs(qv[r], scale, ql[0][r], ql[1][r], ql[2][r]);
         }
         hs0 = __shfl_sync(FULL, hs, (2 * tid) * 4);
         hs1 = __shfl_sync(FULL, hs, (2 * tid + 1) * 4);
@@ -325,77 +341,111 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
         const int ntiles = (nv + 15) >> 4;
 
-        // ---- channel-wise keys: per page, q_d * s_d in fp32 split into an fp16 high and low part (the product
-        // has 22 significant bits; one fp16 alone would cost 2^-12 of every logit term), and sum_d q_d z_d in fp32
-        uint32_t qs_hi[(KAXIS == 1) ? 2 * NR : 1], qs_lo[(KAXIS == 1) ? 2 * NR : 1];
+        // ---- channel-wise keys: per page, the operand of the integer MMAs is q_d * s_d in 22-bit fixed point
+        // (scale from max|q| of the head times the page's largest channel scale).  Each warp makes the limbs of its
+        // own slots, all warps exchange them through shared memory; sum_d q_d z_d is summed in fp32 the same way.
         float zq0 = 0.f, zq1 = 0.f;
         if constexpr (KAXIS == 1) {
           if (!tail_k) {
+            const int buf = page_no & 1;
             const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
+            float smax = 0.f;
+            if (4 * lane < D) {
+              const uint4 mm = *reinterpret_cast<const uint4*>(km + 4 * lane);
+              smax = fmaxf(fmaxf(meta_s(mm.x), meta_s(mm.y)), fmaxf(meta_s(mm.z), meta_s(mm.w)));
+            }
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) smax = fmaxf(smax, __shfl_xor_sync(FULL, smax, off));
+            int e = (int)((__float_as_uint(amax_h * smax) >> 23) & 0xFF) - 127;
+            e = max(e, -60);
+            const int k = 21 - e;
+            const float scale = __uint_as_float((uint32_t)(127 + k) << 23);
+            const float hs = c1 * __uint_as_float((uint32_t)(127 - k) << 23);
+            hs0 = __shfl_sync(FULL, hs, (2 * tid) * 4);
+            hs1 = __shfl_sync(FULL, hs, (2 * tid + 1) * 4);
             float zsum = 0.f;
 #pragma unroll
-            for (int r = 0; r < NR; ++r) {
-              const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);   // (s,z) of 4 channels
-              const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
-              float t[4];
+            for (int i = 0; i < OWN; ++i) {
+              const int r = warp * OWN + i;
+              if (r < NR) {
+                const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);   // (s,z) of 4 channels
+                const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
+                float t[4];
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float2 sz = __half22float2(as_h2(mw[j]));
-                t[j] = qk[r][j] * sz.x;
-                zsum = fmaf(qk[r][j], sz.y, zsum);
+                for (int j = 0; j < 4; ++j) {
+                  const float2 sz = __half22float2(as_h2(mw[j]));
+                  t[j] = qk[i][j] * sz.x;
+                  zsum = fmaf(qk[i][j], sz.y, zsum);
+                }
+                uint32_t w0, w1, w2;
+                fixed_point_limbs(t, scale, w0, w1, w2);
+                sB[((buf * NL + 0) * NR + r) * 32 + lane] = w0;
+                sB[((buf * NL + 1) * NR + r) * 32 + lane] = w1;
+                sB[((buf * NL + 2) * NR + r) * 32 + lane] = w2;
               }
-              split_h2(t[0], t[2], qs_hi[2 * r], qs_lo[2 * r]);
-              split_h2(t[1], t[3], qs_hi[2 * r + 1], qs_lo[2 * r + 1]);
             }
             zsum += __shfl_xor_sync(FULL, zsum, 1);
             zsum += __shfl_xor_sync(FULL, zsum, 2);
-            zq0 = c1 * __shfl_sync(FULL, zsum, (2 * tid) * 4);
-            zq1 = c1 * __shfl_sync(FULL, zsum, (2 * tid + 1) * 4);
+            if (tid == 0 && warp * OWN < NR) sZ[(buf * 8 + gid) * 8 + warp] = zsum;
+          }
+        }
+      }
+      if constexpr (KAXIS == 1) {
+        // every warp takes part in the exchange barrier of a full page, also after a timeout
+        const int nv_b = min(kPageTokens, n_tok - (page + pp) * kPageTokens);
+        if (nv_b == kPageTokens) named_bar_sync(2, NCONS);
+      }
+      if (!aborted) {
+        const uint8_t* sp = smem + stage * sl.page_stride;
+        const uint8_t* sp_k = sp + lane_k;
+        const uint8_t* sp_km = sp + lane_km;
+        const uint8_t* sp_v = sp + lane_v;
+        const uint8_t* sp_vm = sp + lane_vm;
+        const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
+        const int ntiles = (nv + 15) >> 4;
+        float zq0 = 0.f, zq1 = 0.f;
+        if constexpr (KAXIS == 1) {
+          if (!tail_k) {
+            const int buf = page_no & 1;
+#pragma unroll
+            for (int l = 0; l < NL; ++l) {
+#pragma unroll
+              for (int r = 0; r < NR; ++r) ql[l][r] = sB[((buf * NL + l) * NR + r) * 32 + lane];
+            }
+            constexpr int NWR = (NR / OWN < NW) ? NR / OWN : NW;      // warps that contributed
+#pragma unroll
+            for (int w = 0; w < NWR; ++w) {
+              zq0 += sZ[(buf * 8 + 2 * tid) * 8 + w];
+              zq1 += sZ[(buf * 8 + 2 * tid + 1) * 8 + w];
+            }
+            zq0 *= c1;
+            zq1 *= c1;
           }
         }
 
         // The TPW tiles this warp owns in the page (tile = warp + NW * u) are processed together: logits of all
         // of them, one joint running-max check, then probabilities and PV.  MASKED handles a partial page.
         auto logits = [&](const int u, const int tok0, const bool v0, const bool v1, float (&L)[4]) {
-          if constexpr (KAXIS == 1) {
+          if (KAXIS == 1 && tail_k) {
+            // tokens of the incomplete block: fp16 keys from the tail against q as fp16 high + low parts
             float S[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // two chains, summed below
-            if (tail_k) {
-              const uint16_t* tl = c.k_tail + ((size_t)stream * kPageTokens + tok0) * D;
+            const uint16_t* tl = c.k_tail + ((size_t)stream * kPageTokens + tok0) * D;
 #pragma unroll
-              for (int r = 0; r < NR; ++r) {
-                uint2 ra = make_uint2(0u, 0u), rb = make_uint2(0u, 0u);
-                if (v0) ra = *reinterpret_cast<const uint2*>(tl + 16 * r + 4 * tid);
-                if (v1) rb = *reinterpret_cast<const uint2*>(tl + 8 * D + 16 * r + 4 * tid);
-                uint32_t h0, l0_, h1, l1_;       // q as fp16 high + low parts
-                split_h2(qk[r][0], qk[r][2], h0, l0_);
-                split_h2(qk[r][1], qk[r][3], h1, l1_);
-                const uint32_t a0 = __byte_perm(ra.x, ra.y, 0x5410), a1 = __byte_perm(rb.x, rb.y, 0x5410);
-                const uint32_t a2 = __byte_perm(ra.x, ra.y, 0x7632), a3 = __byte_perm(rb.x, rb.y, 0x7632);
-                mma16816(S[r & 1], a0, a1, a2, a3, h0, h1);
-                mma16816(S[r & 1], a0, a1, a2, a3, l0_, l1_);
-              }
-#pragma unroll
-              for (int i = 0; i < 4; ++i) L[i] = c1 * (S[0][i] + S[1][i]);
-            } else {
-              uint32_t ka[KW], kb2[KW];
-              const uint8_t* krow = sp_k + u * (NW * 16 * K_ROW_BYTES);      // this lane's chunk of row tok0
-              load_words<KW>(krow, 64, ka);
-              load_words<KW>(krow + 8 * K_ROW_BYTES, 64, kb2);
-#pragma unroll
-              for (int w = 0; w < KW; ++w) {
-                uint32_t pa[Unpack<KB>::PPW], pb[Unpack<KB>::PPW];
-                Unpack<KB>::run(ka[w], pa);
-                Unpack<KB>::run(kb2[w], pb);
-#pragma unroll
-                for (int i = 0; i < FPB; ++i) {
-                  const int r = w * FPB + i;       // pairs (j = 0, 2) sit in output i, (j = 1, 3) in output FPB + i
-                  mma16816(S[r & 1], pa[i], pb[i], pa[FPB + i], pb[FPB + i], qs_hi[2 * r], qs_hi[2 * r + 1]);
-                  mma16816(S[r & 1], pa[i], pb[i], pa[FPB + i], pb[FPB + i], qs_lo[2 * r], qs_lo[2 * r + 1]);
-                }
-              }
-              L[0] = fmaf(c1, S[0][0] + S[1][0], zq0); L[1] = fmaf(c1, S[0][1] + S[1][1], zq1);
-              L[2] = fmaf(c1, S[0][2] + S[1][2], zq0); L[3] = fmaf(c1, S[0][3] + S[1][3], zq1);
+            for (int r = 0; r < NR; ++r) {
+              uint2 ra = make_uint2(0u, 0u), rb = make_uint2(0u, 0u);
+              if (v0) ra = *reinterpret_cast<const uint2*>(tl + 16 * r + 4 * tid);
+              if (v1) rb = *reinterpret_cast<const uint2*>(tl + 8 * D + 16 * r + 4 * tid);
+              const float4 qq = sQ[r * 32 + lane];
+              uint32_t h0, l0_, h1, l1_;
+              split_h2(qq.x, qq.z, h0, l0_);
+              split_h2(qq.y, qq.w, h1, l1_);
+              const uint32_t a0 = __byte_perm(ra.x, ra.y, 0x5410), a1 = __byte_perm(rb.x, rb.y, 0x5410);
+              const uint32_t a2 = __byte_perm(ra.x, ra.y, 0x7632), a3 = __byte_perm(rb.x, rb.y, 0x7632);
+              mma16816(S[r & 1], a0, a1, a2, a3, h0, h1);
+              mma16816(S[r & 1], a0, a1, a2, a3, l0_, l1_);
             }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) L[i] = c1 * (S[0][i] + S[1][i]);
           } else {
             uint32_t ka[KW], kb2[KW];
             const uint8_t* krow = sp_k + u * (NW * 16 * K_ROW_BYTES);      // this lane's chunk of row tok0
@@ -423,6 +473,11 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
               for (int i = 0; i < 4; ++i)       // sum_d code_d * Q_d = (S0 * 256 + S1) * 256 + S2, exact up to the last step
                 t[i] = fmaf((float)(S[j][0][i] * 256 + S[j][1][i]), 256.f, (float)S[j][2][i]);
+              if constexpr (KAXIS == 1) {       // scales are already inside Q; the zero-points are one sum per page
+                L[0] = fmaf(t[0], hs0, zq0); L[1] = fmaf(t[1], hs1, zq1);
+                L[2] = fmaf(t[2], hs0, zq0); L[3] = fmaf(t[3], hs1, zq1);
+                continue;
+              }
               const float2 ma = __half22float2(as_h2(km[j]));                       // (scale, zero)
               const float2 mb = __half22float2(as_h2(km[8 * NGK + j]));
               L[0] += fmaf(ma.x * hs0, t[0], ma.y * qsum[0][j]);
@@ -528,6 +583,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       __syncwarp();
       if (lane == 0) mbar_arrive(bar0 + 8 * (stages + stage));
       if (++stage == stages) { stage = 0; phase ^= 1; }
+      ++page_no;
     }
 
     // ---- segment end: finish this warp's state, combine the NW warps, write the partial
@@ -621,10 +677,10 @@ template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NL, int NW, in
 int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap,
                     cudaStream_t stream) {
   const int budget = (227 * 1024) / MINB - 1024;            // shared memory per CTA for MINB resident CTAs per SM
-  int stages = (budget - smem_layout(0, 0, NW, D).total) / ((g.page_bytes + 127) & ~127);
+  int stages = (budget - smem_layout(0, 0, NW, D, KAXIS == 1).total) / ((g.page_bytes + 127) & ~127);
   if (stages > 8) stages = 8;
   if (stages < 2) return KVQ_ERR_UNSUPPORTED;
-  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D);
+  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D, KAXIS == 1);
   auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
     return KVQ_ERR_CUDA_LAUNCH;
