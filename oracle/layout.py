@@ -2,7 +2,7 @@
 
 Written from the layout's published index function, independently of the CUDA
 code.  The paper describes no packed layout; this one is the library's own
-(layout version 1):
+(layout version 2):
 
 A page holds 128 consecutive tokens of one (batch, kv-head) stream as four
 regions, in this order, each a multiple of 16 bytes:
@@ -10,7 +10,7 @@ regions, in this order, each a multiple of 16 bytes:
     [K codes | K meta | V codes | V meta]
 
 All multi-byte quantities are little-endian.  A b-bit code field number f of a
-32-bit word occupies bits [f*b, f*b+b).  With ppw = 16/b ("pairs per word"):
+32-bit word occupies bits [f*b, f*b+b).
 
 K codes (b = kb in {2,4,8}): token-major rows of D*b/8 bytes; a row holds 4
 chunks of wpc = D*b/128 words.  With fpb = 8/b fields per byte, channel d of a
@@ -21,15 +21,18 @@ token lives in
 (byte j of a word holds channels 16r + 4*chunk + j for the fpb values of r that
 share the word: masking one field out of every byte yields four consecutive
 channels as four bytes).
-V codes (b = vb in {2,4,8}): 8 tiles of 16 tokens, a tile holds 32 chunks of
-wpc = D*b/64 words.  With k = 8*(d // 64) + d % 8 and npos = 8/b, channel d of
-token tau (0..15 inside its tile) lives in
-    chunk  = 4*((d // 8) % 8) + (tau % 8) // 2
-    word   = k // npos
-    field  = k % npos + npos*(tau // 8) + ppw*(tau % 2)
-(a 16-bit half of a word holds, in its low byte, the codes of tokens 0..7 of the
-tile and, in its high byte, those of tokens 8..15, at the same bit position).
-Placement of (chunk, word) inside its row / tile of `nchunks` chunks: words are
+V codes (b = vb in {2,4,8}): 4 blocks of 32 tokens, a block holds 4*D*b bytes.
+A byte holds the codes of ONE token for the fpb = 8/b channels d, d+16, ...
+that differ only in f below (field f at bit b*f).  With
+    m  = d // 16,  f = m % fpb,  mw = m // fpb,  rh = (d % 16) // 8,  g = d % 8
+    kh = tau // 16,  u = tau % 16,  t = (u % 8) // 2,  j = 2*(u % 2) + u // 8
+channel d of token tau (0..31 inside its block) lives in
+    byte = block*(4*D*b) + mw*512 + (4*g + t)*16 + 4*(2*rh + kh) + j,  bit = b*f
+(the four bytes of a 32-bit word are tokens 2t, 2t+8, 2t+1, 2t+9 of one half
+of the block for one channel; masking one field out of every byte yields four
+tokens of one channel as four bytes, and a token's codes are whole bytes, so an
+append never has to merge with bytes of other tokens).
+Placement of (chunk, word) inside a K row of `nchunks` = 4 chunks: words are
 kept in quads of qw = min(wpc, 4) words, quad-major:
     byte   = (word // 4)*(nchunks*4*qw) + chunk*(4*qw) + (word % 4)*4
 (for wpc <= 4 this is simply chunk-major).
@@ -115,17 +118,20 @@ def k_code_pos(t, d, D, b):
 def v_code_pos(t, d, D, b):
     t = np.asarray(t)
     d = np.asarray(d)
-    ppw = 16 // b
-    tile = t // 16
-    tau = t % 16
-    npos = 8 // b                     # code positions inside the low byte of a 16-bit half
-    k = 8 * (d // 64) + d % 8
-    chunk = 4 * ((d // 8) % 8) + (tau % 8) // 2
-    word = k // npos
-    field = k % npos + npos * (tau // 8) + ppw * (tau % 2)
-    bit = field * b
-    byte = tile * (16 * D * b // 8) + _chunk_word_byte(chunk, word, D * b // 64, 32) + bit // 8
-    return byte, bit % 8
+    fpb = 8 // b                      # codes per byte (channels 16 apart)
+    block = t // 32
+    tau = t % 32
+    kh = tau // 16
+    u = tau % 16
+    tq = (u % 8) // 2
+    j = 2 * (u % 2) + u // 8
+    m = d // 16
+    f = m % fpb
+    mw = m // fpb
+    rh = (d % 16) // 8
+    g = d % 8
+    byte = block * (4 * D * b) + mw * 512 + (4 * g + tq) * 16 + 4 * (2 * rh + kh) + j
+    return byte, b * f + 0 * byte
 
 
 def _put_codes(region: np.ndarray, pos_fn, tokens: np.ndarray, codes: np.ndarray, D, b):

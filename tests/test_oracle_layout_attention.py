@@ -88,22 +88,28 @@ def test_single_field_encoding_is_little_endian_words():
     assert ol.k_code_pos(0, 48, 128, 2) == (0, 6)
     assert ol.k_code_pos(0, 64, 128, 2) == (4, 0)
     assert ol.k_code_pos(0, 4, 128, 2) == (8, 0)
-    # V, D=128, 2-bit (4 positions per byte): (t=0,d=0) byte 0; t=1 (odd token): field 8 -> byte 2
+    # V, D=128, 2-bit (4 codes per byte, blocks of 32 tokens = 1024 bytes).  A word holds tokens
+    # (2t, 2t+8, 2t+1, 2t+9) of one channel: token 0 -> byte 0, token 8 -> byte 1, token 1 -> byte 2, token 9 -> byte 3
     assert ol.v_code_pos(0, 0, 128, 2) == (0, 0)
-    assert ol.v_code_pos(1, 0, 128, 2) == (2, 0)
-    # t=2 -> chunk 1 -> byte 16 ; d=8 -> next chunk group -> chunk 4 -> byte 64 ; t=8 -> high byte of the half
-    assert ol.v_code_pos(2, 0, 128, 2) == (16, 0)
-    assert ol.v_code_pos(0, 8, 128, 2) == (64, 0)
     assert ol.v_code_pos(8, 0, 128, 2) == (1, 0)
+    assert ol.v_code_pos(1, 0, 128, 2) == (2, 0)
     assert ol.v_code_pos(9, 0, 128, 2) == (3, 0)
-    # d=1..3 -> positions 1..3 of the same byte ; d=4 -> k=4 -> word 1 -> byte 4
-    assert ol.v_code_pos(0, 1, 128, 2) == (0, 2)
-    assert ol.v_code_pos(0, 3, 128, 2) == (0, 6)
-    assert ol.v_code_pos(0, 4, 128, 2) == (4, 0)
-    # d=64 -> k=8 -> word 2 -> byte 8 (same chunk as d=0)
-    assert ol.v_code_pos(0, 64, 128, 2) == (8, 0)
-    # next tile of 16 tokens: 16*128*2/8 = 512 bytes further
-    assert ol.v_code_pos(16, 0, 128, 2) == (512, 0)
+    # tokens 2, 3 -> t = 1 -> the next 16-byte lane chunk; tokens 16..31 -> the word one further (kh = 1)
+    assert ol.v_code_pos(2, 0, 128, 2) == (16, 0)
+    assert ol.v_code_pos(16, 0, 128, 2) == (4, 0)
+    # channel d+1 -> g = 1 -> four lane chunks further; d = 8 -> rh = 1 -> two words further
+    assert ol.v_code_pos(0, 1, 128, 2) == (64, 0)
+    assert ol.v_code_pos(0, 8, 128, 2) == (8, 0)
+    # channels 16 apart share the byte: d = 16, 32, 48 at bits 2, 4, 6; d = 64 -> next group of 512 bytes
+    assert ol.v_code_pos(0, 16, 128, 2) == (0, 2)
+    assert ol.v_code_pos(0, 48, 128, 2) == (0, 6)
+    assert ol.v_code_pos(0, 64, 128, 2) == (512, 0)
+    # next block of 32 tokens: 4*128*2 = 1024 bytes further; the very last code of the page
+    assert ol.v_code_pos(32, 0, 128, 2) == (1024, 0)
+    assert ol.v_code_pos(127, 127, 128, 2) == (4095, 6)
+    # head_dim 64: all four 16-channel slices share one group, a block is 512 bytes
+    assert ol.v_code_pos(0, 48, 64, 2) == (0, 6)
+    assert ol.v_code_pos(32, 0, 64, 2) == (512, 0)
     # quad-major word placement when a chunk has more than 4 words:
     # K, D=128, 8-bit (one field per byte, 8 words per chunk): d=2 -> byte 2; d=4 -> chunk 1 -> byte 16;
     # d=16 -> word 1 -> byte 4; d=64 -> word 4 -> second quad -> byte 4 chunks * 16 = 64; d=68 -> 64 + 16
@@ -113,17 +119,17 @@ def test_single_field_encoding_is_little_endian_words():
     assert ol.k_code_pos(0, 64, 128, 8) == (64, 0)
     assert ol.k_code_pos(0, 68, 128, 8) == (80, 0)
     assert ol.k_code_pos(1, 0, 128, 8) == (128, 0)
-    # V, D=128, 4-bit (2 positions per byte, 8 words per chunk): d=1 -> high nibble of byte 0; d=2 -> word 1;
-    # d=64 -> k=8 -> word 4 -> second quad -> byte 32 chunks * 16 = 512
-    assert ol.v_code_pos(0, 1, 128, 4) == (0, 4)
-    assert ol.v_code_pos(0, 2, 128, 4) == (4, 0)
-    assert ol.v_code_pos(0, 64, 128, 4) == (512, 0)
-    assert ol.v_code_pos(2, 64, 128, 4) == (528, 0)
-    # 8-bit: one word per channel slot k: tokens (0, 8, 1, 9) of the lane's token pair in bytes 0..3
+    # V, D=128, 4-bit (2 codes per byte: d and d+16; a block is 2048 bytes): d = 32 -> next group of 512 bytes
+    assert ol.v_code_pos(0, 16, 128, 4) == (0, 4)
+    assert ol.v_code_pos(0, 32, 128, 4) == (512, 0)
+    assert ol.v_code_pos(2, 64, 128, 4) == (1040, 0)
+    assert ol.v_code_pos(32, 0, 128, 4) == (2048, 0)
+    # 8-bit: one code per byte, every 16-channel slice has its own group of 512 bytes
     assert ol.v_code_pos(0, 0, 128, 8) == (0, 0)
     assert ol.v_code_pos(8, 0, 128, 8) == (1, 0)
     assert ol.v_code_pos(1, 0, 128, 8) == (2, 0)
-    assert ol.v_code_pos(0, 1, 128, 8) == (4, 0)
+    assert ol.v_code_pos(0, 16, 128, 8) == (512, 0)
+    assert ol.v_code_pos(0, 9, 128, 8) == (72, 0)
 
 
 def test_memory_ratio_k4v2_vs_k4v4():
