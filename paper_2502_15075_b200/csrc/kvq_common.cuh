@@ -91,7 +91,7 @@ __device__ __forceinline__ uint32_t code_of_fast(float x, const GroupParams& p, 
   return __float_as_uint(__fadd_rn(u, 12582912.0f)) & 0xFFu;
 }
 
-// ---------------------------------------------------------------- key rotation (Sec. 4.3)
+// ---------------------------------------------------------------- key rotation (Sec. 4.4)
 // A token row of D channels is spread over D/8 lanes, lane l holding channels 8l..8l+7.  Unnormalised
 // Walsh-Hadamard transform with the butterfly stages in the order h = 1, 2, 4, ..., (a, b) -> (a + b, a - b)
 // where a is the element whose index has bit h clear; every addition individually rounded.
@@ -142,8 +142,8 @@ __device__ __forceinline__ void unrotate_row8(float (&x)[8], const int8_t* signs
 // ---------------------------------------------------------------- layout index functions
 // Byte offset (inside the K-code region of a page) of the 32-bit word holding
 // channel d of page-local token t, and the field's bit offset inside that word.
-// Byte offset of (chunk, word) inside a K row (nchunks = 4) or a V tile (nchunks = 32): words are kept
-// in quads of min(wpc, 4) words, quad-major, so that a lane's 16-byte load never conflicts with its neighbours'.
+// Byte offset of (chunk, word) inside a K row (nchunks = 4): words are kept in quads of min(wpc, 4) words,
+// quad-major, so that a lane's 16-byte load never conflicts with its neighbours'.
 __host__ __device__ __forceinline__ int chunk_word_byte(int chunk, int word, int wpc, int nchunks) {
   int qw = wpc < 4 ? wpc : 4;
   return (word >> 2) * (nchunks * 4 * qw) + chunk * (4 * qw) + (word & 3) * 4;
@@ -157,14 +157,16 @@ __host__ __device__ __forceinline__ void k_code_pos(int t, int d, int D, int b, 
   bit = 8 * (d & 3) + b * (r % fpb);
 }
 
+// Value codes: 4 blocks of 32 tokens per page, 4*D*b bytes each.  A byte holds the codes of one token for the
+// 8/b channels that lie 16 apart (field f at bit b*f); the four bytes of a word are tokens 2t, 2t+8, 2t+1, 2t+9
+// of one 16-token half of the block.  Returns the word's byte offset and the field's bit offset inside the word.
 __host__ __device__ __forceinline__ void v_code_pos(int t, int d, int D, int b, int& word_byte, int& bit) {
-  int ppw = 16 / b;
-  int tile = t >> 4, tau = t & 15;
-  int npos = 8 / b;             // code positions inside the low byte of a 16-bit half
-  int k = 8 * (d >> 6) + (d & 7);
-  int chunk = 4 * ((d >> 3) & 7) + ((tau & 7) >> 1);
-  word_byte = tile * (16 * D * b / 8) + chunk_word_byte(chunk, k / npos, D * b / 64, 32);
-  bit = (k % npos + npos * (tau >> 3) + ppw * (tau & 1)) * b;
+  const int fpb = 8 / b;
+  const int blk = t >> 5, tau = t & 31, kh = tau >> 4, u = tau & 15;
+  const int tq = (u & 7) >> 1, j = 2 * (u & 1) + (u >> 3);
+  const int m = d >> 4, f = m % fpb, mw = m / fpb, rh = (d >> 3) & 1, gq = d & 7;
+  word_byte = blk * (4 * D * b) + mw * 512 + (4 * gq + tq) * 16 + 4 * (2 * rh + kh);
+  bit = 8 * j + b * f;
 }
 
 // Inverse maps: which channel (and tile-local token) sits in field f of a word.
@@ -174,13 +176,13 @@ __device__ __forceinline__ int k_field_channel(int chunk, int word, int f, int b
   return 16 * r + 4 * chunk + (f / fpb);
 }
 
-__device__ __forceinline__ void v_field_pos(int chunk, int word, int f, int b, int D, int& tau, int& d) {
-  int ppw = 16 / b;
-  int npos = 8 / b;
-  int fh = f % ppw;             // field inside its 16-bit half
-  int k = word * npos + fh % npos;
-  d = 64 * (k >> 3) + 8 * (chunk >> 2) + (k & 7);
-  tau = 8 * (fh / npos) + 2 * (chunk & 3) + (f / ppw);
+// Word number w (0 .. D*b-1) of a value block: which block-local token and channel sit in byte j, field f.
+__device__ __forceinline__ void v_field_pos(int w, int j, int f, int b, int& tau, int& d) {
+  const int fpb = 8 / b;
+  const int mw = w >> 7, lane = (w >> 2) & 31, sub = w & 3;
+  const int gq = lane >> 2, tq = lane & 3, rh = sub >> 1, kh = sub & 1;
+  tau = 16 * kh + 2 * tq + (j >> 1) + 8 * (j & 1);
+  d = 16 * (fpb * mw + f) + 8 * rh + gq;
 }
 
 __device__ __forceinline__ uint32_t load_code(const uint8_t* region, int word_byte, int bit, int b) {

@@ -5,8 +5,8 @@ namespace kvq {
 namespace mma {
 
 // Instantiation units (kvq_decode_mma_inst_*.cu).
-#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB)                                                  \
-  extern template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB>(const Geom&, const CachePtrs&,     \
+#define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB)                                                  \
+  extern template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB>(const Geom&, const CachePtrs&,     \
                                                                                  const void*, float, float*, int, \
                                                                                  cudaStream_t);
 #include "kvq_decode_mma_list.inc"
@@ -92,13 +92,13 @@ static int pick(const Geom& g, const CachePtrs& c, const void* q, float c1, floa
                 cudaStream_t stream, bool probe, int* grid) {
   const int ngk = (g.k_axis == 1 || g.kb == 16) ? 1 : g.D / g.gk;
   const int ngv = (g.vb == 16) ? 1 : g.D / g.gv;
-  const int nl_min = (g.k_axis == 1 || g.in_dtype == KVQ_BF16) ? 2 : 3;   // limbs needed to hold q exactly
-#define KVQ_MMA_DECL(D_, KB_, VB_, KAXIS_, NGK_, NGV_, NL_, NW_, MINB_)                                      \
+  const int nh = g.G <= 4 ? 1 : 2;                                         // query heads per lane
+#define KVQ_MMA_DECL(D_, KB_, VB_, KAXIS_, NGK_, NGV_, NH_, NW_, MINB_)                                      \
   if (g.D == D_ && g.kb == KB_ && g.vb == VB_ && g.k_axis == KAXIS_ && ngk == NGK_ && ngv == NGV_ &&          \
-      NL_ >= nl_min) {                                                                                        \
+      NH_ == nh) {                                                                                            \
     *grid = 148 * MINB_;                                                                                      \
     if (probe) return KVQ_OK;                                                                                 \
-    return mma::launch_mma_inst<D_, KB_, VB_, KAXIS_, NGK_, NGV_, NL_, NW_, MINB_>(g, c, q, c1, ws, s_cap,    \
+    return mma::launch_mma_inst<D_, KB_, VB_, KAXIS_, NGK_, NGV_, NH_, NW_, MINB_>(g, c, q, c1, ws, s_cap,    \
                                                                                    stream);                  \
   }
 #include "kvq_decode_mma_list.inc"

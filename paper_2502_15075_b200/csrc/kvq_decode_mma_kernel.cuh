@@ -29,54 +29,104 @@ __device__ __forceinline__ FlatPlan make_plan(long long N, int pages_max, int gr
   return p;
 }
 
-// Shared-memory carve-up (dynamic): ring | barriers | prefix | combine buffer
+// Shared-memory carve-up (dynamic): ring | barriers | prefix | misc | per-warp fp32 masters | (m, l) | channel-wise scratch
 struct SmemLayout {
-  int page_stride, ring_bytes, bar_off, pref_off, misc_off, comb_off, chan_off, total;
+  int page_stride, ring_bytes, bar_off, pref_off, misc_off, master_off, ml_off, chan_off, total;
 };
-// chan: channel-wise keys need, per CTA, two buffers of per-page q limbs (3 x D/16 x 32 words), the partial
-// zero-point sums (64 floats) and the stream's q in fp32 (D/16 x 32 x 4 floats).
-__host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, int nw, int D, bool chan) {
+// master: per consumer warp, 4 NH heads x (D + 8) floats (the row padding keeps a warp's accesses conflict-free).
+// chan: channel-wise keys need two buffers of per-page q operands (NH x D/16 x 32 words), the partial zero-point
+// sums (2 x 8 heads x 8 floats), the page's fixed-point scale per head (2 x 8) and the stream's q in fp32 (8 x D).
+__host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, int nw, int batch, int D, int nh,
+                                                  bool chan) {
   SmemLayout s;
   s.page_stride = (page_bytes + 127) & ~127;
   s.ring_bytes = s.page_stride * stages;
   s.bar_off = s.ring_bytes;
   s.pref_off = s.bar_off + 16 * 8 * 2;                      // up to 16 stages x (full, empty)
-  s.misc_off = s.pref_off + (kMaxBatchFlat + 1) * 4;
-  s.comb_off = (s.misc_off + 64 + 127) & ~127;
-  int per_warp = (D / 16 * 4 + 4) * 32 * 4;                 // O fragments + m, l per lane
-  s.chan_off = s.comb_off + (nw / 2 > 0 ? nw / 2 : 1) * per_warp;
-  s.total = s.chan_off + (chan ? (2 * 3 * (D / 16) * 32 * 4 + 2 * 64 * 4 + (D / 16) * 32 * 16) : 0);
+  s.misc_off = (s.pref_off + (batch + 1) * 4 + 15) & ~15;
+  s.master_off = s.misc_off + 64;
+  s.ml_off = s.master_off + nw * 4 * nh * (D + 8) * 4;
+  s.chan_off = s.ml_off + nw * 4 * nh * 2 * 4;
+  s.total = s.chan_off + (chan ? (2 * nh * (D / 16) * 32 * 4 + 2 * 64 * 4 + 2 * 8 * 4 + 8 * D * 4) : 0);
   return s;
 }
 
-// Template parameters: head_dim, key bits, value bits, key axis (0 token-wise: keys go through integer MMAs
-// on the raw code bytes with q in 22-bit fixed point split into NL = 3 signed bytes; 1 channel-wise: fp16 MMAs
-// with the channel scales folded into q per page), key / value groups per row, q limbs, consumer warps,
-// resident CTAs per SM.
-template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NL, int NW, int MINB>
+// prmt.b32 with the full selector semantics (a selector nibble with bit 3 set replicates the sign of the byte).
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+// D += A(16x32, row, unsigned bytes) * B(32x8, col, unsigned bytes), int32 accumulate.
+__device__ __forceinline__ void mma16832_u8u8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Four values times `scale` rounded to integers |Q| <= 32512 and split into two balanced signed bytes,
+// Q = hi * 256 + lo; returns the four hi bytes (lo_limb = 0) or the four lo bytes (lo_limb = 1) as one word
+// and adds the four Q to `qsum`.
+__device__ __forceinline__ uint32_t fixed_point_limb(const float (&t)[4], float scale, int lo_limb, int& qsum) {
+  uint32_t w = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int Q = __float2int_rn(t[j] * scale);
+    const int lo = (int)(int8_t)(Q & 0xFF);
+    const int hi = (Q - lo) >> 8;
+    w |= (uint32_t)((lo_limb ? lo : hi) & 0xFF) << (8 * j);
+    qsum += Q;
+  }
+  return w;
+}
+
+constexpr float kQFix = 32512.0f;          // largest |Q| of the 16-bit fixed-point q (hi limb stays within +-127)
+// The softmax weights enter PV as fixed point P = rint(p * s_V * 2^PBITS / s_lim), p = 2^(logit - reference) with the
+// reference kHeadroom bits above the largest logit seen so far, so that a larger logit rarely forces a rescale.
+// Tokens whose P falls below one unit vanish, so the width matters over long contexts: four byte limbs (31 bits)
+// where one lane serves one head, three (24 bits, less headroom) where it serves two.
+template <int NH> constexpr int kPBits = NH == 1 ? 31 : 24;
+template <int NH> constexpr float kHeadroom = NH == 1 ? 6.0f : 1.0f;
+constexpr int kFlushBlocks = 512;          // fold the int32 value accumulators at least this often (no overflow)
+
+// Template parameters: head_dim, key bits, value bits, key axis (0 token-wise, 1 channel-wise), key / value groups
+// per row, NH = query heads per lane (1: up to 4 heads per KV head, 2: up to 8), consumer warps (4: one per
+// 32-token block of a page), resident CTAs per SM.
+//
+// Both contractions run on integer tensor-core MMAs over the raw code bytes (m16n8k32, int32 accumulate).
+// The 8 columns of an MMA carry (head, limb) pairs: q as 16-bit fixed point in two signed bytes for QK^T, the
+// softmax weight times the value scale as 23-bit fixed point in three unsigned bytes for PV.  Lane (g, t) of a
+// warp (g = lane / 4, t = lane % 4) owns query heads t (and t + 4 when NH = 2): its accumulator columns 2t, 2t+1
+// are the limbs of that head, so logits, softmax and the fixed-point weights need no exchange between lanes.
+template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NH, int NW, int MINB>
 __global__ void __launch_bounds__((NW + 1) * 32, MINB)
 decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1, float* __restrict__ ws,
                   int s_cap, int stages) {
-  constexpr int NR = D / 16;                // 16-channel register slots per row (r index of the key layout)
-  constexpr int KS32 = D / 32;              // k-steps of an 8-bit MMA
-  constexpr int MT = D / 16;                // m-tiles of PV (channels)
-  constexpr int KW = D * KB / 128;          // K words per lane per token row
-  constexpr int VW = D * VB / 64;           // V words per lane per 16-token tile
-  constexpr int FPB = 8 / KB;               // key fields per byte
-  constexpr int NPOS = 8 / VB;              // value code positions inside a byte
+  constexpr int NR = D / 16;                // 16-channel register slots per key row
+  constexpr int KS32 = D / 32;              // k-steps of an 8-bit MMA over the channels
+  constexpr int MT = D / 16;                // m-tiles of PV (16 channels each)
+  constexpr int KW = D * KB / 128;          // key words per lane per token row
+  constexpr int FPBV = 8 / VB;              // value codes per byte (channels 16 apart)
+  constexpr int VQ = MT / FPBV;             // quads of value words per lane per 32-token block
+  constexpr int NTV = NH == 1 ? 2 : 3;      // n-tiles of PV: (head, limb) columns
+  constexpr int NHEADS = 4 * NH;
+  constexpr int MSTRIDE = D + 8;
   constexpr int K_ROW_BYTES = D * KB / 8;
-  constexpr int V_TILE_BYTES = 16 * D * VB / 8;
+  constexpr int V_BLOCK_BYTES = 4 * D * VB;
   constexpr int NCONS = NW * 32;
-  constexpr int TPW = (kPageTokens / 16) / NW;   // tiles per warp per page
   constexpr uint32_t FULL = 0xffffffffu;
+  static_assert(NW == 4, "one consumer warp per 32-token block of a page");
   static_assert(KAXIS == 0 || KB != 2, "channel-wise 2-bit keys are not instantiated");
+  static_assert(MT % FPBV == 0, "value m-tiles come in groups that share a byte");
 
   extern __shared__ __align__(128) uint8_t smem[];
-  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D, KAXIS == 1);
+  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, g.B, D, NH, KAXIS == 1);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sl.bar_off);   // full[0..stages), empty[0..stages)
   int* sPref = reinterpret_cast<int*>(smem + sl.pref_off);
   int* sMisc = reinterpret_cast<int*>(smem + sl.misc_off);           // [0] pages_max, [1] abort flag
-  float* sComb = reinterpret_cast<float*>(smem + sl.comb_off);
+  float* sMaster = reinterpret_cast<float*>(smem + sl.master_off);   // [NW][NHEADS][MSTRIDE]
+  float* sML = reinterpret_cast<float*>(smem + sl.ml_off);           // [NW][NHEADS][2] = (reference, l)
 
   const int tid_ = threadIdx.x, lane = tid_ & 31, warp = tid_ >> 5;
   const int gid = lane >> 2, tid = lane & 3;
@@ -159,170 +209,196 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         }
       }
       if (!ok) {
-        // gave up: flag it, then let the copies already in flight land before the CTA exits
         *abort_flag = 1;
         atomicOr(c.status, KVQ_STATUS_DEVICE_TIMEOUT);
-        for (int k = 1; k <= stages && k <= it; ++k) {
-          const int j = it - k;
-          mbar_wait(bar0 + 8 * (j % stages), (j / stages) & 1);
-        }
+      }
+      // Never leave while a copy may still be writing this CTA's shared memory: wait (bounded) for the
+      // last copies issued, whether or not a consumer is still going to.
+      for (int k = 1; k <= stages && k <= it; ++k) {
+        const int j = it - k;
+        mbar_wait(bar0 + 8 * (j % stages), (j / stages) & 1);
       }
     }
     return;
   }
 
   // =========================================================== consumer warps
-  // q operands: signed-byte limbs (token-wise keys) or fp16 pairs (channel-wise keys), heads >= G are zero.
-  // Slot r holds channels 16 r + 4 tid + {0..3} of head gid.
-  uint32_t ql[NL][NR];
-  constexpr int OWN = (NR / NW > 0) ? NR / NW : 1;     // channel-wise keys: slots whose per-page limbs this warp makes
-  float qk[(KAXIS == 1) ? OWN : 1][4];       // ... and the stream's q (rotated if asked) on those slots, fp32
-  float amax_h = 0.f;                        // ... and max |q| of head gid
-  uint32_t* sB = reinterpret_cast<uint32_t*>(smem + sl.chan_off);          // [2][NL][NR][32] per-page q limbs
-  float* sZ = reinterpret_cast<float*>(smem + sl.chan_off + 2 * NL * NR * 32 * 4);   // [2][8 heads][8] partial sums
-  float4* sQ = reinterpret_cast<float4*>(smem + sl.chan_off + 2 * NL * NR * 32 * 4 + 2 * 64 * 4);   // [NR][32]
+  uint32_t qB[NH][NR];         // QK^T B operands: column gid = (head gid/2 + 4 nh, limb gid%2), channels 16 r + 4 tid + {0..3}
+  float hs[NH];                // c1 / fixed-point scale of q, own heads (tid + 4 nh)
+  float qsum[NH][NGK];         // c1 * sum of q over each key group, own heads
+  float zq[NH];                // channel-wise keys: c1 * sum_d q_d z_d of the current page, own heads
+  float amaxB[NH];             // channel-wise keys: max |q| of the operand heads (gid/2 + 4 nh)
+  float m_ref[NH], l[NH], zacc[NH][NGV];
+  int Oi[NTV][MT][4];          // PV accumulators: NH = 1: n-tiles (limb 3, 2 | limb 1, 0) of head tid; NH = 2: (head tid:
+                               // limb 2, 1 | head tid + 4: limb 2, 1 | limb 0 of both)
+  constexpr float PONE = (float)(1u << (kPBits<NH> - 1)) * 2.0f;     // 2^PBITS
+  float s_lim = 9.094947e-13f; // 2^-40: power of two above every value scale folded into the weights so far
+  float sscale = PONE / 9.094947e-13f, inv_sscale = 9.094947e-13f / PONE;
+  int since_flush = 0;
+  uint32_t* sB = reinterpret_cast<uint32_t*>(smem + sl.chan_off);                                  // [2][NH][NR][32]
+  float* sZ = reinterpret_cast<float*>(smem + sl.chan_off + 2 * NH * NR * 32 * 4);                 // [2][8 heads][8]
+  float* sHS = sZ + 2 * 64;                                                                        // [2][8 heads]
+  float* sQ = sHS + 2 * 8;                                                                         // [8 heads][D]
+  float* myM = sMaster + warp * NHEADS * MSTRIDE;
   int page_no = 0;
-  float qsum[2][NGK];                        // c1 * sum of q over each key group, heads (2 tid, 2 tid + 1)
-  float hs0 = 0.f, hs1 = 0.f;                // c1 / fixed-point scale of heads (2 tid, 2 tid + 1)
-  float O[MT][4];
-  float zacc[2][NGV];
-  float m0, m1, l0, l1;
   int stage = 0;
   uint32_t phase = 0;
   bool aborted = false;
-  // byte offsets inside a page of this lane's operands for the warp's first tile (rows warp*16 + gid, +8)
-  constexpr int KCB = (KW < 4 ? KW : 4) * 4, VCB = (VW < 4 ? VW : 4) * 4;     // bytes of a lane chunk's first quad
-  const int lane_k = (warp * 16 + gid) * K_ROW_BYTES + tid * KCB;
-  const int lane_km = g.k_meta_off + (warp * 16 + gid) * 4 * NGK;
-  const int lane_v = g.v_codes_off + warp * V_TILE_BYTES + lane * VCB;
-  const int lane_vm = g.v_meta_off + (warp * 16 + gid) * 4 * NGV;
+  constexpr int KCB = (KW < 4 ? KW : 4) * 4;     // bytes of a lane chunk's first quad of key words
+  const int lane_k = (warp * 32 + gid) * K_ROW_BYTES + tid * KCB;
+  const int lane_km = g.k_meta_off + (warp * 32 + gid) * 4 * NGK;
+  const int lane_v = g.v_codes_off + warp * V_BLOCK_BYTES + lane * 16;
+  const int lane_vm = g.v_meta_off + (warp * 32 + gid) * 4 * NGV;
+
+  // Fold the int32 accumulators into the warp's fp32 master (each (head, channel) belongs to one lane) and clear them.
+  auto flush_acc = [&]() {
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      const float fw = inv_sscale / (float)(1 << (VB * (mt % FPBV)));
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int d = 16 * mt + 8 * r + gid;
+        if constexpr (NH == 1) {
+          const float v = fmaf((float)Oi[0][mt][2 * r], 16777216.f,
+                               fmaf((float)Oi[0][mt][2 * r + 1], 65536.f,
+                                    fmaf((float)Oi[1][mt][2 * r], 256.f, (float)Oi[1][mt][2 * r + 1])));
+          myM[tid * MSTRIDE + d] += v * fw;
+        } else {
+          const float v0 = fmaf((float)Oi[0][mt][2 * r], 65536.f, fmaf((float)Oi[0][mt][2 * r + 1], 256.f,
+                                                                        (float)Oi[2][mt][2 * r]));
+          const float v1 = fmaf((float)Oi[1][mt][2 * r], 65536.f, fmaf((float)Oi[1][mt][2 * r + 1], 256.f,
+                                                                        (float)Oi[2][mt][2 * r + 1]));
+          myM[tid * MSTRIDE + d] += v0 * fw;
+          myM[(tid + 4) * MSTRIDE + d] += v1 * fw;
+        }
+      }
+#pragma unroll
+      for (int nt = 0; nt < NTV; ++nt) { Oi[nt][mt][0] = Oi[nt][mt][1] = Oi[nt][mt][2] = Oi[nt][mt][3] = 0; }
+    }
+    since_flush = 0;
+  };
 
   for (long long x = x_lo; x < x_hi;) {
     const int seg_pages = (int)min((long long)(pages_b - page), x_hi - x);
     const int n_tok = clamped_len(c.seq_len, b, g.capacity);
     const int stream = b * Hkv + h;
 
-    // ---- segment start: q operands and group sums for this stream's heads
+    // ---- segment start: q operands, group sums and a clean state for this stream's heads
     {
-      float part[NGK];
+      if constexpr (KAXIS == 1) named_bar_sync(2, NCONS);            // nobody still reads the previous stream's q
 #pragma unroll
-      for (int j = 0; j < NGK; ++j) part[j] = 0.f;
-      float qv[NR][4];
-      float amax = 0.f;
-      const uint16_t* qrow = q + ((size_t)b * g.Hq + (size_t)h * G + gid) * D;
-#pragma unroll
-      for (int r = 0; r < NR; ++r) {
-        uint2 raw = make_uint2(0u, 0u);
-        if (gid < G) raw = *reinterpret_cast<const uint2*>(qrow + 16 * r + 4 * tid);
-        qv[r][0] = bits16_to_f32((uint16_t)(raw.x & 0xFFFF), g.in_dtype);
-        qv[r][1] = bits16_to_f32((uint16_t)(raw.x >> 16), g.in_dtype);
-        qv[r][2] = bits16_to_f32((uint16_t)(raw.y & 0xFFFF), g.in_dtype);
-        qv[r][3] = bits16_to_f32((uint16_t)(raw.y >> 16), g.in_dtype);
-      }
-      if (c.k_signs != nullptr) {
-        // rotated keys: give q the same rotation, q' = H (signs * q) / sqrt(D); channel 16 r + 4 tid + j,
-        // so the butterflies run over j inside the lane, over tid across lanes, over r inside the lane
+      for (int nh = 0; nh < NH; ++nh) {
+        const int hb = (gid >> 1) + 4 * nh;                          // head of this lane's operand column
+        float qv[NR][4];
+        const uint16_t* qrow = q + ((size_t)b * g.Hq + (size_t)h * G + hb) * D;
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) qv[r][j] *= (float)c.k_signs[16 * r + 4 * tid + j];
-          float a = qv[r][0], bq = qv[r][1], cq = qv[r][2], dq = qv[r][3];
-          qv[r][0] = (a + bq) + (cq + dq); qv[r][1] = (a - bq) + (cq - dq);
-          qv[r][2] = (a + bq) - (cq + dq); qv[r][3] = (a - bq) - (cq - dq);
-#pragma unroll
-          for (int m = 1; m < 4; m <<= 1) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float o = __shfl_xor_sync(FULL, qv[r][j], m);
-              qv[r][j] = (tid & m) ? o - qv[r][j] : qv[r][j] + o;
-            }
-          }
+          uint2 raw = make_uint2(0u, 0u);
+          if (hb < G) raw = *reinterpret_cast<const uint2*>(qrow + 16 * r + 4 * tid);
+          qv[r][0] = bits16_to_f32((uint16_t)(raw.x & 0xFFFF), g.in_dtype);
+          qv[r][1] = bits16_to_f32((uint16_t)(raw.x >> 16), g.in_dtype);
+          qv[r][2] = bits16_to_f32((uint16_t)(raw.y & 0xFFFF), g.in_dtype);
+          qv[r][3] = bits16_to_f32((uint16_t)(raw.y >> 16), g.in_dtype);
         }
-#pragma unroll
-        for (int hh = 1; hh < NR; hh <<= 1) {
+        if (c.k_signs != nullptr) {
+          // rotated keys: give q the same rotation, q' = H (signs * q) / sqrt(D); channel 16 r + 4 tid + j,
+          // so the butterflies run over j inside the lane, over tid across lanes, over r inside the lane
 #pragma unroll
           for (int r = 0; r < NR; ++r) {
-            if ((r & hh) == 0) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) qv[r][j] *= (float)c.k_signs[16 * r + 4 * tid + j];
+            float a = qv[r][0], bq = qv[r][1], cq = qv[r][2], dq = qv[r][3];
+            qv[r][0] = (a + bq) + (cq + dq); qv[r][1] = (a - bq) + (cq - dq);
+            qv[r][2] = (a + bq) - (cq + dq); qv[r][3] = (a - bq) - (cq - dq);
+#pragma unroll
+            for (int m = 1; m < 4; m <<= 1) {
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                const float a = qv[r][j], bq = qv[r + hh][j];
-                qv[r][j] = a + bq;
-                qv[r + hh][j] = a - bq;
+                const float o = __shfl_xor_sync(FULL, qv[r][j], m);
+                qv[r][j] = (tid & m) ? o - qv[r][j] : qv[r][j] + o;
               }
             }
           }
-        }
 #pragma unroll
-        for (int r = 0; r < NR; ++r) {
+          for (int hh = 1; hh < NR; hh <<= 1) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) qv[r][j] *= inv_sqrt_dim<D>();
-        }
-      }
+            for (int r = 0; r < NR; ++r) {
+              if ((r & hh) == 0) {
 #pragma unroll
-      for (int r = 0; r < NR; ++r) {
-        float f[4] = {qv[r][0], qv[r][1], qv[r][2], qv[r][3]};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          amax = fmaxf(amax, fabsf(f[j]));
-          part[r / (NR / NGK)] += f[j];
-        }
-      }
-      static_assert(NL == 3, "three signed 8-bit limbs");
-      amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 1));
-      amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 2));
-      if constexpr (KAXIS == 1) {
-        // channel-wise keys: the limbs depend on the page's scales and are made per page; keep what that needs
-        amax_h = amax;
-#pragma unroll
-        for (int i = 0; i < OWN; ++i) {
-#pragma unroll
-          for (int r = 0; r < NR; ++r) {       // (compile-time indices keep qv in registers)
-            if (r == warp * OWN + i) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) qk[i][j] = qv[r][j];
+                for (int j = 0; j < 4; ++j) {
+                  const float a = qv[r][j], bq = qv[r + hh][j];
+                  qv[r][j] = a + bq;
+                  qv[r + hh][j] = a - bq;
+                }
+              }
             }
           }
-        }
-        named_bar_sync(2, NCONS);                       // nobody still reads the previous stream's copy
-        if (warp == 0) {
 #pragma unroll
-          for (int r = 0; r < NR; ++r) sQ[r * 32 + lane] = make_float4(qv[r][0], qv[r][1], qv[r][2], qv[r][3]);
+          for (int r = 0; r < NR; ++r) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) qv[r][j] *= inv_sqrt_dim<D>();
+          }
         }
-        named_bar_sync(2, NCONS);
-      }
-      if constexpr (KAXIS == 0) {
-        // per head: 22-bit fixed point relative to the head's largest entry, Q = rint(q * 2^k) with
-        // |Q| < 2^22, split into three balanced signed bytes  Q = l0 * 65536 + l1 * 256 + l2
-        int e = (int)((__float_as_uint(amax) >> 23) & 0xFF) - 127;
-        e = max(e, -60);
-        const int k = 21 - e;
-        const float scale = __uint_as_float((uint32_t)(127 + k) << 23);
-        const float hs = c1 * __uint_as_float((uint32_t)(127 - k) << 23);
+        float amax = 0.f;
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
-          fixed_point_limbs(qv[r], scale, ql[0][r], ql[1][r], ql[2][r]);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) amax = fmaxf(amax, fabsf(qv[r][j]));
         }
-        hs0 = __shfl_sync(FULL, hs, (2 * tid) * 4);
-        hs1 = __shfl_sync(FULL, hs, (2 * tid + 1) * 4);
+        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 2));
+        if constexpr (KAXIS == 1) {
+          // channel-wise keys: the operands depend on the page's scales and are made per page from the stream's q
+          amaxB[nh] = amax;
+          if ((gid & 1) == 0) {
+#pragma unroll
+            for (int r = 0; r < NR; ++r)
+              *reinterpret_cast<float4*>(sQ + hb * D + 16 * r + 4 * tid) = make_float4(qv[r][0], qv[r][1], qv[r][2], qv[r][3]);
+          }
+          hs[nh] = 0.f;
+        } else {
+          // 16-bit fixed point relative to the head's largest entry: Q = rint(q * scale), |Q| <= 32512
+          const float scale = amax > 0.f ? kQFix / amax : 0.f;
+          const float hsb = amax > 0.f ? c1 / scale : 0.f;
+          int qs[NGK];
+#pragma unroll
+          for (int j = 0; j < NGK; ++j) qs[j] = 0;
+#pragma unroll
+          for (int r = 0; r < NR; ++r) qB[nh][r] = fixed_point_limb(qv[r], scale, gid & 1, qs[r / (NR / NGK)]);
+          hs[nh] = __shfl_sync(FULL, hsb, 8 * tid);
+          // the zero-point term uses the sum of the same fixed-point q the MMAs see: the two large terms
+          // s (q . c) and z sum(q) of a logit then cancel exactly as they do for the exact q
+#pragma unroll
+          for (int j = 0; j < NGK; ++j) {
+            int v = qs[j];
+            v += __shfl_xor_sync(FULL, v, 1);
+            v += __shfl_xor_sync(FULL, v, 2);
+            qsum[nh][j] = hs[nh] * (float)__shfl_sync(FULL, v, 8 * tid);
+          }
+        }
+        m_ref[nh] = -INFINITY;
+        l[nh] = 0.f;
+        zq[nh] = 0.f;
+#pragma unroll
+        for (int j = 0; j < NGV; ++j) zacc[nh][j] = 0.f;
       }
+      if constexpr (KAXIS == 1) named_bar_sync(2, NCONS);
 #pragma unroll
-      for (int j = 0; j < NGK; ++j) {
-        float v = part[j];
-        v += __shfl_xor_sync(FULL, v, 1);
-        v += __shfl_xor_sync(FULL, v, 2);
-        qsum[0][j] = c1 * __shfl_sync(FULL, v, (2 * tid) * 4);
-        qsum[1][j] = c1 * __shfl_sync(FULL, v, (2 * tid + 1) * 4);
+      for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+        for (int nt = 0; nt < NTV; ++nt) { Oi[nt][mt][0] = Oi[nt][mt][1] = Oi[nt][mt][2] = Oi[nt][mt][3] = 0; }
+#pragma unroll
+        for (int nh = 0; nh < NH; ++nh) {
+          myM[(tid + 4 * nh) * MSTRIDE + 16 * mt + gid] = 0.f;
+          myM[(tid + 4 * nh) * MSTRIDE + 16 * mt + 8 + gid] = 0.f;
+        }
       }
-#pragma unroll
-      for (int mt = 0; mt < MT; ++mt) { O[mt][0] = O[mt][1] = O[mt][2] = O[mt][3] = 0.f; }
-#pragma unroll
-      for (int j = 0; j < NGV; ++j) { zacc[0][j] = zacc[1][j] = 0.f; }
-      m0 = m1 = -INFINITY;
-      l0 = l1 = 0.f;
+      since_flush = 0;
     }
 
     for (int pp = 0; pp < seg_pages; ++pp) {
       const int nv = min(kPageTokens, n_tok - (page + pp) * kPageTokens);
+      const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
       if (!aborted) {
         const bool got = mbar_wait(bar0 + 8 * stage, phase);
         if (!__all_sync(FULL, got)) {
@@ -331,254 +407,281 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           if (lane == 0) atomicOr(c.status, KVQ_STATUS_DEVICE_TIMEOUT);
         }
       }
-      if (!aborted) {
-        const uint8_t* sp = smem + stage * sl.page_stride;
-        // this lane's first byte in each region for the warp's tile 0 (tile u adds a constant)
-        const uint8_t* sp_k = sp + lane_k;
-        const uint8_t* sp_km = sp + lane_km;
-        const uint8_t* sp_v = sp + lane_v;
-        const uint8_t* sp_vm = sp + lane_vm;
-        const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
-        const int ntiles = (nv + 15) >> 4;
+      const uint8_t* sp = smem + stage * sl.page_stride;
 
-        // ---- channel-wise keys: per page, the operand of the integer MMAs is q_d * s_d in 22-bit fixed point
-        // (scale from max|q| of the head times the page's largest channel scale).  Each warp makes the limbs of its
-        // own slots, all warps exchange them through shared memory; sum_d q_d z_d is summed in fp32 the same way.
-        float zq0 = 0.f, zq1 = 0.f;
-        if constexpr (KAXIS == 1) {
-          if (!tail_k) {
-            const int buf = page_no & 1;
-            const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
-            float smax = 0.f;
-            if (4 * lane < D) {
-              const uint4 mm = *reinterpret_cast<const uint4*>(km + 4 * lane);
-              smax = fmaxf(fmaxf(meta_s(mm.x), meta_s(mm.y)), fmaxf(meta_s(mm.z), meta_s(mm.w)));
-            }
+      // ---- channel-wise keys: per page, the operand of the integer MMAs is q_d * s_d in 16-bit fixed point
+      // (scale from max|q| of the head times the page's largest channel scale).  Each warp makes the operands of
+      // its own slots, all warps exchange them through shared memory; sum_d q_d z_d is summed in fp32 the same way.
+      if constexpr (KAXIS == 1) {
+        constexpr int OWN = NR / NW > 0 ? NR / NW : 1;
+        const int buf = page_no & 1;
+        if (!aborted && !tail_k) {
+          const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
+          float smax = 0.f;
+          if (4 * lane < D) {
+            const uint4 mm = *reinterpret_cast<const uint4*>(km + 4 * lane);
+            smax = fmaxf(fmaxf(meta_s(mm.x), meta_s(mm.y)), fmaxf(meta_s(mm.z), meta_s(mm.w)));
+          }
 #pragma unroll
-            for (int off = 1; off < 32; off <<= 1) smax = fmaxf(smax, __shfl_xor_sync(FULL, smax, off));
-            int e = (int)((__float_as_uint(amax_h * smax) >> 23) & 0xFF) - 127;
-            e = max(e, -60);
-            const int k = 21 - e;
-            const float scale = __uint_as_float((uint32_t)(127 + k) << 23);
-            const float hs = c1 * __uint_as_float((uint32_t)(127 - k) << 23);
-            hs0 = __shfl_sync(FULL, hs, (2 * tid) * 4);
-            hs1 = __shfl_sync(FULL, hs, (2 * tid + 1) * 4);
+          for (int off = 1; off < 32; off <<= 1) smax = fmaxf(smax, __shfl_xor_sync(FULL, smax, off));
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) {
+            const int hb = (gid >> 1) + 4 * nh;
+            const float am = amaxB[nh] * smax;
+            const float scale = am > 0.f ? kQFix / am : 0.f;
+            if (warp == 0 && tid == 0 && (gid & 1) == 0) sHS[buf * 8 + hb] = am > 0.f ? c1 / scale : 0.f;
             float zsum = 0.f;
 #pragma unroll
             for (int i = 0; i < OWN; ++i) {
               const int r = warp * OWN + i;
               if (r < NR) {
-                const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);   // (s,z) of 4 channels
+                const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);   // (s, z) of 4 channels
+                const float4 qq = *reinterpret_cast<const float4*>(sQ + hb * D + 16 * r + 4 * tid);
                 const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
+                const float qa[4] = {qq.x, qq.y, qq.z, qq.w};
                 float t[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                   const float2 sz = __half22float2(as_h2(mw[j]));
-                  t[j] = qk[i][j] * sz.x;
-                  zsum = fmaf(qk[i][j], sz.y, zsum);
+                  t[j] = qa[j] * sz.x;
+                  zsum = fmaf(qa[j], sz.y, zsum);
                 }
-                uint32_t w0, w1, w2;
-                fixed_point_limbs(t, scale, w0, w1, w2);
-                sB[((buf * NL + 0) * NR + r) * 32 + lane] = w0;
-                sB[((buf * NL + 1) * NR + r) * 32 + lane] = w1;
-                sB[((buf * NL + 2) * NR + r) * 32 + lane] = w2;
+                int unused = 0;
+                sB[((buf * NH + nh) * NR + r) * 32 + lane] = fixed_point_limb(t, scale, gid & 1, unused);
               }
             }
             zsum += __shfl_xor_sync(FULL, zsum, 1);
             zsum += __shfl_xor_sync(FULL, zsum, 2);
-            if (tid == 0 && warp * OWN < NR) sZ[(buf * 8 + gid) * 8 + warp] = zsum;
+            if (tid == 0 && (gid & 1) == 0 && warp * OWN < NR) sZ[(buf * 8 + hb) * 8 + warp] = zsum;
+          }
+        }
+        // every warp takes part in the exchange barrier of a full page, also after a timeout
+        if (!tail_k) named_bar_sync(2, NCONS);
+        if (!aborted && !tail_k) {
+          constexpr int NWR = (NR / OWN < NW) ? NR / OWN : NW;      // warps that contributed
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) {
+#pragma unroll
+            for (int r = 0; r < NR; ++r) qB[nh][r] = sB[((buf * NH + nh) * NR + r) * 32 + lane];
+            float z = 0.f;
+#pragma unroll
+            for (int w = 0; w < NWR; ++w) z += sZ[(buf * 8 + tid + 4 * nh) * 8 + w];
+            zq[nh] = c1 * z;
+            hs[nh] = sHS[buf * 8 + tid + 4 * nh];
           }
         }
       }
-      if constexpr (KAXIS == 1) {
-        // every warp takes part in the exchange barrier of a full page, also after a timeout
-        const int nv_b = min(kPageTokens, n_tok - (page + pp) * kPageTokens);
-        if (nv_b == kPageTokens) named_bar_sync(2, NCONS);
-      }
-      if (!aborted) {
-        const uint8_t* sp = smem + stage * sl.page_stride;
+
+      if (!aborted && warp * 32 < nv) {
         const uint8_t* sp_k = sp + lane_k;
         const uint8_t* sp_km = sp + lane_km;
         const uint8_t* sp_v = sp + lane_v;
         const uint8_t* sp_vm = sp + lane_vm;
-        const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
-        const int ntiles = (nv + 15) >> 4;
-        float zq0 = 0.f, zq1 = 0.f;
-        if constexpr (KAXIS == 1) {
-          if (!tail_k) {
-            const int buf = page_no & 1;
-#pragma unroll
-            for (int l = 0; l < NL; ++l) {
-#pragma unroll
-              for (int r = 0; r < NR; ++r) ql[l][r] = sB[((buf * NL + l) * NR + r) * 32 + lane];
-            }
-            constexpr int NWR = (NR / OWN < NW) ? NR / OWN : NW;      // warps that contributed
-#pragma unroll
-            for (int w = 0; w < NWR; ++w) {
-              zq0 += sZ[(buf * 8 + 2 * tid) * 8 + w];
-              zq1 += sZ[(buf * 8 + 2 * tid + 1) * 8 + w];
-            }
-            zq0 *= c1;
-            zq1 *= c1;
-          }
-        }
 
-        // The TPW tiles this warp owns in the page (tile = warp + NW * u) are processed together: logits of all
-        // of them, one joint running-max check, then probabilities and PV.  MASKED handles a partial page.
-        auto logits = [&](const int u, const int tok0, const bool v0, const bool v1, float (&L)[4]) {
-          if (KAXIS == 1 && tail_k) {
-            // tokens of the incomplete block: fp16 keys from the tail against q as fp16 high + low parts
-            float S[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};   // two chains, summed below
-            const uint16_t* tl = c.k_tail + ((size_t)stream * kPageTokens + tok0) * D;
-#pragma unroll
-            for (int r = 0; r < NR; ++r) {
-              uint2 ra = make_uint2(0u, 0u), rb = make_uint2(0u, 0u);
-              if (v0) ra = *reinterpret_cast<const uint2*>(tl + 16 * r + 4 * tid);
-              if (v1) rb = *reinterpret_cast<const uint2*>(tl + 8 * D + 16 * r + 4 * tid);
-              const float4 qq = sQ[r * 32 + lane];
-              uint32_t h0, l0_, h1, l1_;
-              split_h2(qq.x, qq.z, h0, l0_);
-              split_h2(qq.y, qq.w, h1, l1_);
-              const uint32_t a0 = __byte_perm(ra.x, ra.y, 0x5410), a1 = __byte_perm(rb.x, rb.y, 0x5410);
-              const uint32_t a2 = __byte_perm(ra.x, ra.y, 0x7632), a3 = __byte_perm(rb.x, rb.y, 0x7632);
-              mma16816(S[r & 1], a0, a1, a2, a3, h0, h1);
-              mma16816(S[r & 1], a0, a1, a2, a3, l0_, l1_);
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) L[i] = c1 * (S[0][i] + S[1][i]);
-          } else {
-            uint32_t ka[KW], kb2[KW];
-            const uint8_t* krow = sp_k + u * (NW * 16 * K_ROW_BYTES);      // this lane's chunk of row tok0
-            load_words<KW>(krow, 64, ka);
-            load_words<KW>(krow + 8 * K_ROW_BYTES, 64, kb2);
-            int S[NGK][NL][4];
-#pragma unroll
-            for (int j = 0; j < NGK; ++j) {
-#pragma unroll
-              for (int l = 0; l < NL; ++l) { S[j][l][0] = S[j][l][1] = S[j][l][2] = S[j][l][3] = 0; }
-            }
-#pragma unroll
-            for (int s = 0; s < KS32; ++s) {
-              const int j = s / (KS32 / NGK);
-              const uint32_t a0 = key_slot<KB, KW>(ka, 2 * s), a1 = key_slot<KB, KW>(kb2, 2 * s);
-              const uint32_t a2 = key_slot<KB, KW>(ka, 2 * s + 1), a3 = key_slot<KB, KW>(kb2, 2 * s + 1);
-#pragma unroll
-              for (int l = 0; l < NL; ++l) mma16832_u8s8(S[j][l], a0, a1, a2, a3, ql[l][2 * s], ql[l][2 * s + 1]);
-            }
-            const uint32_t* km = reinterpret_cast<const uint32_t*>(sp_km + u * (NW * 16 * 4 * NGK));   // row tok0
-            L[0] = L[1] = L[2] = L[3] = 0.f;
-#pragma unroll
-            for (int j = 0; j < NGK; ++j) {
-              float t[4];
-#pragma unroll
-              for (int i = 0; i < 4; ++i)       // sum_d code_d * Q_d = (S0 * 256 + S1) * 256 + S2, exact up to the last step
-                t[i] = fmaf((float)(S[j][0][i] * 256 + S[j][1][i]), 256.f, (float)S[j][2][i]);
-              if constexpr (KAXIS == 1) {       // scales are already inside Q; the zero-points are one sum per page
-                L[0] = fmaf(t[0], hs0, zq0); L[1] = fmaf(t[1], hs1, zq1);
-                L[2] = fmaf(t[2], hs0, zq0); L[3] = fmaf(t[3], hs1, zq1);
-                continue;
-              }
-              const float2 ma = __half22float2(as_h2(km[j]));                       // (scale, zero)
-              const float2 mb = __half22float2(as_h2(km[8 * NGK + j]));
-              L[0] += fmaf(ma.x * hs0, t[0], ma.y * qsum[0][j]);
-              L[1] += fmaf(ma.x * hs1, t[1], ma.y * qsum[1][j]);
-              L[2] += fmaf(mb.x * hs0, t[2], mb.y * qsum[0][j]);
-              L[3] += fmaf(mb.x * hs1, t[3], mb.y * qsum[1][j]);
-            }
-          }
-          if (!v0) { L[0] = -INFINITY; L[1] = -INFINITY; }
-          if (!v1) { L[2] = -INFINITY; L[3] = -INFINITY; }
-        };
-
-        // values of one tile: fold the scale into p, keep the zero-point term as a scalar per group
-        auto values = [&](const int u, const bool v0, const bool v1, const float (&p)[4]) {
-          const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp_vm + u * (NW * 16 * 4 * NGV));   // row tok0
-          const uint32_t pa01 = pack_h2(p[0], p[1]), pb01 = pack_h2(p[2], p[3]);
-          uint32_t bw[NGV][2];
-#pragma unroll
-          for (int j = 0; j < NGV; ++j) {
-            const uint32_t ma = v0 ? vm[j] : 0u;
-            const uint32_t mb = v1 ? vm[8 * NGV + j] : 0u;
-            // zero-point of the centred codes: z + s * MID
-            const float za = fmaf(meta_s(ma), kCodeMid<VB>, meta_z(ma)), zb = fmaf(meta_s(mb), kCodeMid<VB>, meta_z(mb));
-            zacc[0][j] += p[0] * za + p[2] * zb;
-            zacc[1][j] += p[1] * za + p[3] * zb;
-            // (p * s) in fp16: both heads of a row share the row's scale
-            const uint32_t sa2 = __byte_perm(ma, ma, 0x1010), sb2 = __byte_perm(mb, mb, 0x1010);
-            bw[j][0] = movmatrix_trans(as_u32(__hmul2(as_h2(pa01), as_h2(sa2))));
-            bw[j][1] = movmatrix_trans(as_u32(__hmul2(as_h2(pb01), as_h2(sb2))));
-          }
-          // Codes become fp16 with one LOP3 (field bits into the mantissa of 1024.0) and one HFMA2 that strips the
-          // 1024, undoes the field's bit position and centres the code on MID: the MMA then sums p*s*(code - MID),
-          // which is small where sum p*s*code and sum p*z would cancel, and MID moves into the zero-point above.
-          uint32_t vw[VW];
-          load_words<VW>(sp_v + u * (NW * V_TILE_BYTES), 512, vw);
-          uint32_t vh[VW];
-#pragma unroll
-          for (int w = 0; w < VW; ++w) vh[w] = vw[w] >> 8;        // tokens 8..15 of the tile
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-            const int j = mt / (MT / NGV);
-            const uint32_t a0 = centered_pair<VB>(vw[(2 * mt) / NPOS], (2 * mt) % NPOS);
-            const uint32_t a1 = centered_pair<VB>(vw[(2 * mt + 1) / NPOS], (2 * mt + 1) % NPOS);
-            const uint32_t a2 = centered_pair<VB>(vh[(2 * mt) / NPOS], (2 * mt) % NPOS);
-            const uint32_t a3 = centered_pair<VB>(vh[(2 * mt + 1) / NPOS], (2 * mt + 1) % NPOS);
-            mma16816(O[mt], a0, a1, a2, a3, bw[j][0], bw[j][1]);
-          }
-        };
-
-        auto do_tiles = [&](auto masked_tag) {
+        auto do_block = [&](auto masked_tag) {
           constexpr bool MASKED = decltype(masked_tag)::value;
-          float L[TPW][4];
-          bool v0[TPW], v1[TPW];
-          float t0 = -INFINITY, t1 = -INFINITY;
+          float L[2][2][NH];                 // [tile][row gid / gid + 8][head]
+          bool vld[2][2];
+          // ------------------------------------------------------------ logits of the block's two 16-token tiles
 #pragma unroll
-          for (int u = 0; u < TPW; ++u) {
-            const int tok0 = (warp + NW * u) * 16 + gid;        // page-local tokens of this lane's two rows
-            v0[u] = !MASKED || tok0 < nv;
-            v1[u] = !MASKED || tok0 + 8 < nv;
-            if (!MASKED || (warp + NW * u) < ntiles) {
-              logits(u, tok0, v0[u], v1[u], L[u]);
+          for (int u = 0; u < 2; ++u) {
+            const int tok0 = warp * 32 + 16 * u + gid;        // page-local tokens of this lane's two rows: tok0, tok0 + 8
+            vld[u][0] = !MASKED || tok0 < nv;
+            vld[u][1] = !MASKED || tok0 + 8 < nv;
+            if (KAXIS == 1 && tail_k) {
+              // tokens of the incomplete block: fp16 keys from the tail against q as fp16 high + low parts;
+              // column gid of the operand = (head gid/2 + 4 nh, part gid%2), so lane columns 2 tid, 2 tid + 1 are the
+              // two parts of head tid + 4 nh
+              const uint16_t* tl = c.k_tail + ((size_t)stream * kPageTokens + tok0) * D;
+#pragma unroll
+              for (int nh = 0; nh < NH; ++nh) {
+                const int hb = (gid >> 1) + 4 * nh;
+                float S[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                  uint2 ra = make_uint2(0u, 0u), rb = make_uint2(0u, 0u);
+                  if (vld[u][0]) ra = *reinterpret_cast<const uint2*>(tl + 16 * r + 4 * tid);
+                  if (vld[u][1]) rb = *reinterpret_cast<const uint2*>(tl + 8 * D + 16 * r + 4 * tid);
+                  const float4 qq = *reinterpret_cast<const float4*>(sQ + hb * D + 16 * r + 4 * tid);
+                  uint32_t h0, l0_, h1, l1_;
+                  split_h2(qq.x, qq.z, h0, l0_);
+                  split_h2(qq.y, qq.w, h1, l1_);
+                  const uint32_t a0 = __byte_perm(ra.x, ra.y, 0x5410), a1 = __byte_perm(rb.x, rb.y, 0x5410);
+                  const uint32_t a2 = __byte_perm(ra.x, ra.y, 0x7632), a3 = __byte_perm(rb.x, rb.y, 0x7632);
+                  mma16816(S, a0, a1, a2, a3, (gid & 1) ? l0_ : h0, (gid & 1) ? l1_ : h1);
+                }
+                L[u][0][nh] = c1 * (S[0] + S[1]);
+                L[u][1][nh] = c1 * (S[2] + S[3]);
+              }
             } else {
-              L[u][0] = L[u][1] = L[u][2] = L[u][3] = -INFINITY;
+              uint32_t ka[KW], kb2[KW];
+              const uint8_t* krow = sp_k + u * (16 * K_ROW_BYTES);           // this lane's chunk of row tok0
+              load_words<KW>(krow, 64, ka);
+              load_words<KW>(krow + 8 * K_ROW_BYTES, 64, kb2);
+              int S[NGK][NH][4];
+#pragma unroll
+              for (int j = 0; j < NGK; ++j) {
+#pragma unroll
+                for (int nh = 0; nh < NH; ++nh) { S[j][nh][0] = S[j][nh][1] = S[j][nh][2] = S[j][nh][3] = 0; }
+              }
+#pragma unroll
+              for (int s = 0; s < KS32; ++s) {
+                const int j = s / (KS32 / NGK);
+                const uint32_t a0 = key_slot<KB, KW>(ka, 2 * s), a1 = key_slot<KB, KW>(kb2, 2 * s);
+                const uint32_t a2 = key_slot<KB, KW>(ka, 2 * s + 1), a3 = key_slot<KB, KW>(kb2, 2 * s + 1);
+#pragma unroll
+                for (int nh = 0; nh < NH; ++nh)
+                  mma16832_u8s8(S[j][nh], a0, a1, a2, a3, qB[nh][2 * s], qB[nh][2 * s + 1]);
+              }
+              // accumulator columns 2 tid, 2 tid + 1 = (hi, lo) limbs of head tid + 4 nh: sum_d code_d Q_d = 256 hi + lo
+              if constexpr (KAXIS == 1) {
+#pragma unroll
+                for (int nh = 0; nh < NH; ++nh) {
+                  L[u][0][nh] = fmaf((float)(S[0][nh][0] * 256 + S[0][nh][1]), hs[nh], zq[nh]);
+                  L[u][1][nh] = fmaf((float)(S[0][nh][2] * 256 + S[0][nh][3]), hs[nh], zq[nh]);
+                }
+              } else {
+                const uint32_t* km = reinterpret_cast<const uint32_t*>(sp_km + u * (16 * 4 * NGK));   // row tok0
+#pragma unroll
+                for (int nh = 0; nh < NH; ++nh) { L[u][0][nh] = 0.f; L[u][1][nh] = 0.f; }
+#pragma unroll
+                for (int j = 0; j < NGK; ++j) {
+                  const float2 ma = __half22float2(as_h2(km[j]));                       // (scale, zero) of row tok0
+                  const float2 mb = __half22float2(as_h2(km[8 * NGK + j]));             // ... of row tok0 + 8
+#pragma unroll
+                  for (int nh = 0; nh < NH; ++nh) {
+                    const float t0 = (float)(S[j][nh][0] * 256 + S[j][nh][1]);
+                    const float t1 = (float)(S[j][nh][2] * 256 + S[j][nh][3]);
+                    L[u][0][nh] += fmaf(ma.x * hs[nh], t0, ma.y * qsum[nh][j]);
+                    L[u][1][nh] += fmaf(mb.x * hs[nh], t1, mb.y * qsum[nh][j]);
+                  }
+                }
+              }
             }
-            t0 = fmaxf(t0, fmaxf(L[u][0], L[u][2]));
-            t1 = fmaxf(t1, fmaxf(L[u][1], L[u][3]));
-          }
-          // online softmax: rescale only when some logit exceeds the running max
-          if (__any_sync(FULL, (t0 > m0) | (t1 > m1))) {
-            float u0 = t0, u1 = t1;
+            if (MASKED) {
 #pragma unroll
-            for (int off = 4; off < 32; off <<= 1) {
-              u0 = fmaxf(u0, __shfl_xor_sync(FULL, u0, off));
-              u1 = fmaxf(u1, __shfl_xor_sync(FULL, u1, off));
+              for (int nh = 0; nh < NH; ++nh) {
+                if (!vld[u][0]) L[u][0][nh] = -INFINITY;
+                if (!vld[u][1]) L[u][1][nh] = -INFINITY;
+              }
             }
-            const float n0 = fmaxf(m0, u0), n1 = fmaxf(m1, u1);
-            const float a0 = (n0 == -INFINITY) ? 1.f : ex2(m0 - n0);
-            const float a1 = (n1 == -INFINITY) ? 1.f : ex2(m1 - n1);
-            m0 = n0; m1 = n1;
-            l0 *= a0; l1 *= a1;
-#pragma unroll
-            for (int j = 0; j < NGV; ++j) { zacc[0][j] *= a0; zacc[1][j] *= a1; }
-#pragma unroll
-            for (int mt = 0; mt < MT; ++mt) { O[mt][0] *= a0; O[mt][1] *= a1; O[mt][2] *= a0; O[mt][3] *= a1; }
           }
+
+          // ------------------------------------------------------------ value scales and zero-points of the four rows
+          float sv[2][2][NGV], zv[2][2][NGV];
+          float smax = 0.f;
 #pragma unroll
-          for (int u = 0; u < TPW; ++u) {
-            if (!MASKED || (warp + NW * u) < ntiles) {
-              float p[4];
-              p[0] = ex2(L[u][0] - m0); p[1] = ex2(L[u][1] - m1); p[2] = ex2(L[u][2] - m0); p[3] = ex2(L[u][3] - m1);
-              l0 += p[0] + p[2];
-              l1 += p[1] + p[3];
-              values(u, v0[u], v1[u], p);
+          for (int u = 0; u < 2; ++u) {
+            const uint32_t* vm = reinterpret_cast<const uint32_t*>(sp_vm + u * (16 * 4 * NGV));
+#pragma unroll
+            for (int j = 0; j < NGV; ++j) {
+              const uint32_t ma = vld[u][0] ? vm[j] : 0u;
+              const uint32_t mb = vld[u][1] ? vm[8 * NGV + j] : 0u;
+              const float2 fa = __half22float2(as_h2(ma)), fb = __half22float2(as_h2(mb));
+              sv[u][0][j] = fa.x; zv[u][0][j] = fa.y;
+              sv[u][1][j] = fb.x; zv[u][1][j] = fb.y;
+              smax = fmaxf(smax, fmaxf(fa.x, fb.x));
+            }
+          }
+
+          // ------------------------------------------------------------ softmax reference / scale check (rarely taken)
+          float bmax[NH];
+          bool trig = (smax >= s_lim) | (since_flush >= kFlushBlocks);
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) {
+            bmax[nh] = fmaxf(fmaxf(L[0][0][nh], L[0][1][nh]), fmaxf(L[1][0][nh], L[1][1][nh]));
+            trig |= bmax[nh] > m_ref[nh];
+          }
+          if (__any_sync(FULL, trig)) {
+            flush_acc();                                   // with the scale the accumulated weights were made with
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) smax = fmaxf(smax, __shfl_xor_sync(FULL, smax, off));
+            if (smax >= s_lim) {
+              // next power of two above the largest value scale: p * s * sscale < 2^PBITS for every p <= 1
+              s_lim = __uint_as_float((__float_as_uint(smax) & 0x7F800000u) + 0x00800000u);
+              sscale = PONE / s_lim;
+              inv_sscale = s_lim / PONE;
+            }
+#pragma unroll
+            for (int nh = 0; nh < NH; ++nh) {
+              float bm = bmax[nh];
+#pragma unroll
+              for (int off = 4; off < 32; off <<= 1) bm = fmaxf(bm, __shfl_xor_sync(FULL, bm, off));
+              if (bm > m_ref[nh]) {
+                const float nref = bm + kHeadroom<NH>;
+                const float a = (m_ref[nh] == -INFINITY) ? 0.f : ex2(m_ref[nh] - nref);
+                m_ref[nh] = nref;
+                l[nh] *= a;
+#pragma unroll
+                for (int j = 0; j < NGV; ++j) zacc[nh][j] *= a;
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                  myM[(tid + 4 * nh) * MSTRIDE + 16 * mt + gid] *= a;
+                  myM[(tid + 4 * nh) * MSTRIDE + 16 * mt + 8 + gid] *= a;
+                }
+              }
+            }
+          }
+          ++since_flush;
+
+          // ------------------------------------------------------------ weights: p = 2^(logit - reference) <= 2^-headroom,
+          // P = rint(p * s_V * sscale) < 2^PBITS
+          uint32_t bV[NGV][NTV][2];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            float p[2][NH];
+#pragma unroll
+            for (int nh = 0; nh < NH; ++nh) {
+              p[0][nh] = ex2(L[u][0][nh] - m_ref[nh]);
+              p[1][nh] = ex2(L[u][1][nh] - m_ref[nh]);
+              l[nh] += p[0][nh] + p[1][nh];
+            }
+#pragma unroll
+            for (int j = 0; j < NGV; ++j) {
+              const float sa = sv[u][0][j] * sscale, sb = sv[u][1][j] * sscale;
+              uint32_t Pa[NH], Pb[NH];
+#pragma unroll
+              for (int nh = 0; nh < NH; ++nh) {
+                zacc[nh][j] = fmaf(p[0][nh], zv[u][0][j], fmaf(p[1][nh], zv[u][1][j], zacc[nh][j]));
+                Pa[nh] = __float2uint_rn(p[0][nh] * sa);      // token tok0
+                Pb[nh] = __float2uint_rn(p[1][nh] * sb);      // token tok0 + 8
+              }
+              // one 16-bit element per (column, lane row) = that column's limb of tokens (tok0, tok0 + 8); the 8x8
+              // transpose turns lane columns into the B operand (column = lane/4, tokens 2t, 2t+8, 2t+1, 2t+9)
+              if constexpr (NH == 1) {
+                bV[j][0][u] = movmatrix_trans(prmt(Pa[0], Pb[0], 0x6273));       // limbs (3, 2): bytes a3 b3 a2 b2
+                bV[j][1][u] = movmatrix_trans(prmt(Pa[0], Pb[0], 0x4051));       // limbs (1, 0): bytes a1 b1 a0 b0
+              } else {
+                bV[j][0][u] = movmatrix_trans(prmt(Pa[0], Pb[0], 0x5162));       // head tid: (hi, mid)
+                bV[j][1][u] = movmatrix_trans(prmt(Pa[1], Pb[1], 0x5162));       // head tid + 4: (hi, mid)
+                bV[j][2][u] = movmatrix_trans(prmt(prmt(Pa[0], Pb[0], 0x0040), prmt(Pa[1], Pb[1], 0x0040), 0x5410));
+              }
+            }
+          }
+
+          // ------------------------------------------------------------ PV on the raw code bytes: one mask per register.
+          // Field f of every byte belongs to m-tile FPBV q + f, whose accumulators carry the factor 2^(VB f).
+#pragma unroll
+          for (int qd = 0; qd < VQ; ++qd) {
+            const uint4 vw = *reinterpret_cast<const uint4*>(sp_v + qd * 512);
+#pragma unroll
+            for (int f = 0; f < FPBV; ++f) {
+              const int mt = FPBV * qd + f;
+              const int j = mt / (MT / NGV);
+              uint32_t a0 = vw.x, a2 = vw.y, a1 = vw.z, a3 = vw.w;     // words (rh, kh) = (0,0), (0,1), (1,0), (1,1)
+              if constexpr (VB != 8) {
+                constexpr uint32_t M0 = ((1u << VB) - 1u) * 0x01010101u;
+                const uint32_t mask = M0 << (VB * f);
+                a0 &= mask; a1 &= mask; a2 &= mask; a3 &= mask;
+              }
+#pragma unroll
+              for (int nt = 0; nt < NTV; ++nt) mma16832_u8u8(Oi[nt][mt], a0, a1, a2, a3, bV[j][nt][0], bV[j][nt][1]);
             }
           }
         };
 
-        if (ntiles > warp) {                     // a short last page may leave this warp without a tile
-          if (nv == kPageTokens) do_tiles(std::false_type{});
-          else do_tiles(std::true_type{});
-        }
+        if (nv - warp * 32 >= 32) do_block(std::false_type{});
+        else do_block(std::true_type{});
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar0 + 8 * (stages + stage));
@@ -588,74 +691,49 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
     // ---- segment end: finish this warp's state, combine the NW warps, write the partial
     {
+      flush_acc();
 #pragma unroll
-      for (int off = 4; off < 32; off <<= 1) {
-        l0 += __shfl_xor_sync(FULL, l0, off);
-        l1 += __shfl_xor_sync(FULL, l1, off);
+      for (int nh = 0; nh < NH; ++nh) {
 #pragma unroll
-        for (int j = 0; j < NGV; ++j) {
-          zacc[0][j] += __shfl_xor_sync(FULL, zacc[0][j], off);
-          zacc[1][j] += __shfl_xor_sync(FULL, zacc[1][j], off);
+        for (int off = 4; off < 32; off <<= 1) {
+          l[nh] += __shfl_xor_sync(FULL, l[nh], off);
+#pragma unroll
+          for (int j = 0; j < NGV; ++j) zacc[nh][j] += __shfl_xor_sync(FULL, zacc[nh][j], off);
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          const int j = mt / (MT / NGV);
+          myM[(tid + 4 * nh) * MSTRIDE + 16 * mt + gid] += zacc[nh][j];
+          myM[(tid + 4 * nh) * MSTRIDE + 16 * mt + 8 + gid] += zacc[nh][j];
+        }
+        if (gid == 0) {
+          sML[(warp * NHEADS + tid + 4 * nh) * 2 + 0] = m_ref[nh];
+          sML[(warp * NHEADS + tid + 4 * nh) * 2 + 1] = l[nh];
         }
       }
+      named_bar_sync(1, NCONS);
+      const long long xs = (long long)sPref[b] + (long long)h * pages_b;     // first page of this stream
+      const int slot = (int)blockIdx.x - plan.cta_of(xs);
+      if (slot >= 0 && slot < s_cap) {
+        for (int idx = tid_; idx < G * D; idx += NCONS) {
+          const int head = idx / D, d = idx % D;
+          float mstar = -INFINITY;
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        const int j = mt / (MT / NGV);
-        O[mt][0] += zacc[0][j]; O[mt][1] += zacc[1][j]; O[mt][2] += zacc[0][j]; O[mt][3] += zacc[1][j];
-      }
-      constexpr int PER_LANE = MT * 4 + 4;
+          for (int w = 0; w < NW; ++w) mstar = fmaxf(mstar, sML[(w * NHEADS + head) * 2]);
+          float o = 0.f, lsum = 0.f;
 #pragma unroll
-      for (int step = NW / 2; step >= 1; step >>= 1) {
-        if (warp >= step && warp < 2 * step) {
-          float* dst = sComb + (size_t)(warp - step) * PER_LANE * 32 + lane;
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-#pragma unroll
-            for (int r = 0; r < 4; ++r) dst[(mt * 4 + r) * 32] = O[mt][r];
+          for (int w = 0; w < NW; ++w) {
+            const float mw = sML[(w * NHEADS + head) * 2];
+            const float f = (mw == -INFINITY) ? 0.f : ex2(mw - mstar);
+            o = fmaf(f, sMaster[(w * NHEADS + head) * MSTRIDE + d], o);
+            lsum = fmaf(f, sML[(w * NHEADS + head) * 2 + 1], lsum);
           }
-          dst[(MT * 4 + 0) * 32] = m0; dst[(MT * 4 + 1) * 32] = m1;
-          dst[(MT * 4 + 2) * 32] = l0; dst[(MT * 4 + 3) * 32] = l1;
-        }
-        named_bar_sync(1, NCONS);
-        if (warp < step) {
-          const float* src = sComb + (size_t)warp * PER_LANE * 32 + lane;
-          const float om0 = src[(MT * 4 + 0) * 32], om1 = src[(MT * 4 + 1) * 32];
-          const float n0 = fmaxf(m0, om0), n1 = fmaxf(m1, om1);
-          const float fa0 = (n0 == -INFINITY) ? 0.f : ex2(m0 - n0), fb0 = (n0 == -INFINITY) ? 0.f : ex2(om0 - n0);
-          const float fa1 = (n1 == -INFINITY) ? 0.f : ex2(m1 - n1), fb1 = (n1 == -INFINITY) ? 0.f : ex2(om1 - n1);
-#pragma unroll
-          for (int mt = 0; mt < MT; ++mt) {
-            O[mt][0] = O[mt][0] * fa0 + src[(mt * 4 + 0) * 32] * fb0;
-            O[mt][1] = O[mt][1] * fa1 + src[(mt * 4 + 1) * 32] * fb1;
-            O[mt][2] = O[mt][2] * fa0 + src[(mt * 4 + 2) * 32] * fb0;
-            O[mt][3] = O[mt][3] * fa1 + src[(mt * 4 + 3) * 32] * fb1;
-          }
-          l0 = l0 * fa0 + src[(MT * 4 + 2) * 32] * fb0;
-          l1 = l1 * fa1 + src[(MT * 4 + 3) * 32] * fb1;
-          m0 = n0; m1 = n1;
-        }
-        named_bar_sync(1, NCONS);
-      }
-      if (warp == 0) {
-        const long long xs = (long long)sPref[b] + (long long)h * pages_b;     // first page of this stream
-        const int slot = (int)blockIdx.x - plan.cta_of(xs);
-        if (slot >= 0 && slot < s_cap) {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int head = 2 * tid + e;
-            if (head < G) {
-              float* dst = ws + (((size_t)stream * s_cap + slot) * G + head) * (D + 2);
-              if (gid == 0) { dst[0] = e ? m1 : m0; dst[1] = e ? l1 : l0; }
-#pragma unroll
-              for (int mt = 0; mt < MT; ++mt) {
-                // accumulator rows (gid, gid + 8) of m-tile mt are channels 64 (mt/4) + 8 gid + 2 (mt%4) + {0, 1}
-                dst[2 + 64 * (mt >> 2) + 8 * gid + 2 * (mt & 3)] = O[mt][e];
-                dst[2 + 64 * (mt >> 2) + 8 * gid + 2 * (mt & 3) + 1] = O[mt][2 + e];
-              }
-            }
-          }
+          float* dst = ws + (((size_t)stream * s_cap + slot) * G + head) * (D + 2);
+          if (d == 0) { dst[0] = mstar; dst[1] = lsum; }
+          dst[2 + d] = o;
         }
       }
+      named_bar_sync(1, NCONS);
     }
 
     // ---- advance the cursor past this segment
@@ -673,15 +751,15 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 }
 
 // Launches one instantiation; defined per instantiation unit.
-template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NL, int NW, int MINB>
+template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NH, int NW, int MINB>
 int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap,
                     cudaStream_t stream) {
   const int budget = (227 * 1024) / MINB - 1024;            // shared memory per CTA for MINB resident CTAs per SM
-  int stages = (budget - smem_layout(0, 0, NW, D, KAXIS == 1).total) / ((g.page_bytes + 127) & ~127);
+  int stages = (budget - smem_layout(0, 0, NW, g.B, D, NH, KAXIS == 1).total) / ((g.page_bytes + 127) & ~127);
   if (stages > 8) stages = 8;
   if (stages < 2) return KVQ_ERR_UNSUPPORTED;
-  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, D, KAXIS == 1);
-  auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NL, NW, MINB>;
+  const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, g.B, D, NH, KAXIS == 1);
+  auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
     return KVQ_ERR_CUDA_LAUNCH;
   kern<<<148 * MINB, (NW + 1) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap,

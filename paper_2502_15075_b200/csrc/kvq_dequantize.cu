@@ -55,26 +55,26 @@ __device__ __forceinline__ void expand_keys(const uint8_t* spage, const Geom& g,
 template <int B>
 __device__ __forceinline__ void expand_values(const uint8_t* spage, const Geom& g, uint16_t* tile, int tid) {
   const int D = g.D;
-  constexpr int NF = 32 / B;
-  const int wpt = D * B / 2;           // words per 16-token tile
-  const int wpc = D * B / 64;          // words per chunk
-  const uint8_t* codes = spage + g.v_codes_off;
+  constexpr int FPB = 8 / B;
+  const int wpb = D * B;               // words per 32-token block
+  const uint32_t* codes = reinterpret_cast<const uint32_t*>(spage + g.v_codes_off);
   const uint32_t* meta = reinterpret_cast<const uint32_t*>(spage + g.v_meta_off);
   const int lgv = ilog2(g.gv), ngv = D >> lgv;
-  const int lwpt = ilog2(wpt), lwpc = ilog2(wpc);
-  for (int idx = tid; idx < 8 * wpt; idx += kThreads) {
-    const int vt = idx >> lwpt, wi = idx & (wpt - 1);
-    const int chunk = wi >> lwpc, word = wi & (wpc - 1);
-    const uint32_t w = *reinterpret_cast<const uint32_t*>(codes + (size_t)vt * (16 * D * B / 8) +
-                                                           chunk_word_byte(chunk, word, wpc, 32));
+  const int lwpb = ilog2(wpb);
+  for (int idx = tid; idx < 4 * wpb; idx += kThreads) {
+    const int blk = idx >> lwpb, w = idx & (wpb - 1);
+    const uint32_t word = codes[idx];
 #pragma unroll
-    for (int f = 0; f < NF; ++f) {
-      int tau, d;
-      v_field_pos(chunk, word, f, B, D, tau, d);
-      const int t = vt * 16 + tau;
-      const uint32_t m = meta[t * ngv + (d >> lgv)];
-      const float code = (float)((w >> (f * B)) & ((1u << B) - 1u));
-      tile[t * D + d] = f32_to_bits16(fmaf(code, meta_scale(m), meta_zero(m)), g.in_dtype);
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+      for (int f = 0; f < FPB; ++f) {
+        int tau, d;
+        v_field_pos(w, j, f, B, tau, d);
+        const int t = blk * 32 + tau;
+        const uint32_t m = meta[t * ngv + (d >> lgv)];
+        const float code = (float)((word >> (8 * j + B * f)) & ((1u << B) - 1u));
+        tile[t * D + d] = f32_to_bits16(fmaf(code, meta_scale(m), meta_zero(m)), g.in_dtype);
+      }
     }
   }
 }

@@ -3,12 +3,14 @@
 // groups along head_dim, or channel-wise groups over a 128-token block with an
 // fp16 residual tail) and packing into the page layout.
 //
-// Token-wise kernel: one warp per 16-token tile of one stream.  Every lane loads
-// 16 bytes (8 consecutive channels of one token), groups reduce min/max with
-// shuffles, the 8 codes of a lane are merged into at most four partial words and
-// OR-ed into an image of the packed tile in shared memory, and the finished image
-// leaves with 16-byte coalesced stores.  The kernel is bound by reading the 16-bit
-// inputs from HBM.
+// Token-wise kernel: one warp per block of 32 tokens (64 for head_dim 64 at 2 bits) of one
+// stream and one side (keys or values).  A byte of the packed page holds codes of channels that
+// lie 16 apart, so a lane loads, for each of its tokens, the 8/b 16-byte pieces whose codes share
+// bytes: every output byte, and with four tokens (values) or four channels (keys) every output
+// word, is then assembled in that lane's registers and stored directly - no shared memory, no
+// atomics, no read-modify-write; a token that is not new is simply not stored (byte stores for
+// values).  Group minima and maxima are reduced with a few shuffles between the lanes of a row.
+// The kernel is bound by reading the 16-bit inputs from HBM.
 #include "kvq_internal.h"
 
 namespace kvq {
@@ -18,201 +20,323 @@ namespace {
 constexpr int kThreads = 128;
 constexpr int kWarps = kThreads / 32;
 constexpr uint32_t FULL = 0xffffffffu;
+constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to nearest-even at integer precision
 
-// Quantize one side (keys or values) of a 16-token tile held in global memory as rows of D 16-bit values.
-// `img` is the warp's shared-memory image of the packed codes of the tile: for keys 16 token rows of
-// D*BITS/8 bytes, for values the tile's D*BITS*2 bytes.  Tokens outside [lo, hi) are left alone.
+// Tokens handled by one warp task: 32, or 64 where 32 tokens would leave a lane fewer than the four tokens
+// that make up a word of value codes.
+__host__ __device__ constexpr int task_tokens(int D, int bits) { return (D == 64 && bits == 2) ? 64 : 32; }
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+
+// Four byte values held as exact float integers (0..255) -> one little-endian word.
+__device__ __forceinline__ uint32_t pack_bytes(float b0, float b1, float b2, float b3) {
+  const float lo = __fmaf_rn(b1, 256.0f, b0), hi = __fmaf_rn(b3, 256.0f, b2);        // < 65536: exact
+  return prmt(__float_as_uint(__fadd_rn(lo, 8388608.0f)), __float_as_uint(__fadd_rn(hi, 8388608.0f)), 0x5410);
+}
+
+// Quantize one side of a task of TT tokens.  src: row of the task's first token in the input; tokens
+// [lo, hi) of the task are new.  codes: keys - the page's key row of the task's first token; values - the
+// page's value block of the task's first token.  meta_out: metadata row of the task's first token.
+//
+// Lane = (row slot rs, word column mw, row half rh): it owns, for each of its tokens, the FPB pieces of
+// 8 channels 16 (FPB mw + f) + 8 rh + {0..7}, f < FPB, whose codes share bytes.
 template <int BITS, bool IS_V, int D, int DTYPE, bool ROT>
-__device__ __forceinline__ void quantize_tile_side(const uint16_t* __restrict__ src, int64_t st, int gsz,
-                                                   int lo, int hi, uint32_t* img,
-                                                   uint32_t* __restrict__ meta_out, bool clear_first, int lane,
-                                                   const int8_t* __restrict__ signs) {
-  constexpr int lpr = D >> 3;                // lanes per token row (8 channels each)
-  constexpr int rps = 32 / lpr;              // rows per step
-  const int l = lane & (lpr - 1);
-  const int d0 = l * 8;
-  const int lpg = gsz >> 3;                  // lanes per group
-  const int ng = D / gsz;
+__device__ __forceinline__ void quantize_task(const uint16_t* __restrict__ src, int64_t st, int gsz, int lo, int hi,
+                                              uint8_t* __restrict__ codes, uint32_t* __restrict__ meta_out,
+                                              int lane, const int8_t* __restrict__ signs) {
+  constexpr int FPB = 8 / BITS;
+  constexpr int NMW = (D / 16) / FPB;        // word columns per row half
+  constexpr int LR = 2 * NMW;                // lanes per token row
+  constexpr int RS = 32 / LR;                // token rows per load instruction
+  constexpr int TT = task_tokens(D, BITS);
+  constexpr int TPL = TT / RS;               // tokens per lane
+  constexpr int K_ROW_BYTES = D * BITS / 8;
+  static_assert(TPL % 4 == 0, "a lane holds whole groups of four tokens");
+  const int rs = lane / LR, cs = lane % LR, mw = cs >> 1, rh = cs & 1;
   const float qmax = (float)((1 << BITS) - 1);
-#pragma unroll 4
-  for (int step = 0; step < 16 / rps; ++step) {
-    if (step * rps + rps <= lo || step * rps >= hi) continue;      // no new token in this step's rows (warp-uniform)
-    const int tau = step * rps + lane / lpr;
+  const int spg = gsz >> 4;                                  // 16-channel slices per group
+  const bool split = FPB > spg;                              // a lane's fields belong to two groups (FPB 4, groups of 32)
+  const int lpg = split ? 2 : 2 * spg / FPB;                 // lanes per group
+  const int ng = D / gsz;
+
+  // block-local token of token slot k
+  auto token_of = [&](int k) {
+    if constexpr (IS_V) {
+      const int cmb = (k >> 2) * RS + rs, j = k & 3;         // cmb = (block, half, t) of the word; j = byte
+      return 32 * (cmb >> 3) + 16 * ((cmb >> 2) & 1) + 2 * (cmb & 3) + (j >> 1) + 8 * (j & 1);
+    } else {
+      return k * RS + rs;
+    }
+  };
+
+  // ---- all loads first (TPL * FPB 16-byte loads in flight per lane)
+  uint4 raw[TPL][FPB];
+#pragma unroll
+  for (int k = 0; k < TPL; ++k) {
+    const int tau = token_of(k);
     const bool valid = tau >= lo && tau < hi;
-    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-    if (valid) raw = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + d0);
-    const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
-    float x[8];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      if constexpr (DTYPE == KVQ_BF16) {
-        x[2 * i] = __uint_as_float(rw[i] << 16);
-        x[2 * i + 1] = __uint_as_float(rw[i] & 0xFFFF0000u);
-      } else {
-        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&rw[i]));
-        x[2 * i] = f.x;
-        x[2 * i + 1] = f.y;
+    for (int f = 0; f < FPB; ++f) {
+      raw[k][f] = make_uint4(0u, 0u, 0u, 0u);
+      if (valid) raw[k][f] = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + 16 * (FPB * mw + f) + 8 * rh);
+    }
+  }
+
+  float vbyte[4][8];      // values: byte values (exact float integers) of the four tokens of the words being built
+#pragma unroll
+  for (int k = 0; k < TPL; ++k) {
+    const int tau = token_of(k);
+    const bool valid = tau >= lo && tau < hi;
+    float x[FPB][8];
+#pragma unroll
+    for (int f = 0; f < FPB; ++f) {
+      const uint32_t rw[4] = {raw[k][f].x, raw[k][f].y, raw[k][f].z, raw[k][f].w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if constexpr (DTYPE == KVQ_BF16) {
+          x[f][2 * i] = __uint_as_float(rw[i] << 16);
+          x[f][2 * i + 1] = __uint_as_float(rw[i] & 0xFFFF0000u);
+        } else {
+          const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&rw[i]));
+          x[f][2 * i] = v.x;
+          x[f][2 * i + 1] = v.y;
+        }
       }
     }
-    if constexpr (ROT) rotate_row8<D>(x, signs, l);      // keys only: y = H (signs * x) / sqrt(D)
-    float mn = INFINITY, mx = -INFINITY;
+    if constexpr (ROT) {
+      // keys only: y = H (signs * x) / sqrt(D); channel d = 16 (FPB mw + f) + 8 rh + i.  Butterfly stages in
+      // the order h = 1, 2, 4, ...: bits of i in the lane, rh across lanes, bits of f in the lane, bits of mw across lanes.
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      mn = fminf(mn, x[i]);
-      mx = fmaxf(mx, x[i]);
+      for (int f = 0; f < FPB; ++f) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[f][i] = __fmul_rn(x[f][i], (float)signs[16 * (FPB * mw + f) + 8 * rh + i]);
+#pragma unroll
+        for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if ((i & h) == 0) {
+              const float a = x[f][i], b = x[f][i + h];
+              x[f][i] = __fadd_rn(a, b);
+              x[f][i + h] = __fsub_rn(a, b);
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int f = 0; f < FPB; ++f) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float o = __shfl_xor_sync(FULL, x[f][i], 1);
+          x[f][i] = rh ? __fsub_rn(o, x[f][i]) : __fadd_rn(x[f][i], o);
+        }
+      }
+#pragma unroll
+      for (int hf = 1; hf < FPB; hf <<= 1) {
+#pragma unroll
+        for (int f = 0; f < FPB; ++f) {
+          if ((f & hf) == 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const float a = x[f][i], b = x[f + hf][i];
+              x[f][i] = __fadd_rn(a, b);
+              x[f + hf][i] = __fsub_rn(a, b);
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int hm = 1; hm < NMW; hm <<= 1) {
+        const bool upper = (mw & hm) != 0;
+#pragma unroll
+        for (int f = 0; f < FPB; ++f) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float o = __shfl_xor_sync(FULL, x[f][i], 2 * hm);
+            x[f][i] = upper ? __fsub_rn(o, x[f][i]) : __fadd_rn(x[f][i], o);
+          }
+        }
+      }
+#pragma unroll
+      for (int f = 0; f < FPB; ++f) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[f][i] = __fmul_rn(x[f][i], inv_sqrt_dim<D>());
+      }
+    }
+
+    // ---- group minimum / maximum: fields in the lane, then the lanes of the group
+    float mnf[FPB], mxf[FPB];
+#pragma unroll
+    for (int f = 0; f < FPB; ++f) {
+      mnf[f] = fminf(fminf(fminf(x[f][0], x[f][1]), fminf(x[f][2], x[f][3])),
+                     fminf(fminf(x[f][4], x[f][5]), fminf(x[f][6], x[f][7])));
+      mxf[f] = fmaxf(fmaxf(fmaxf(x[f][0], x[f][1]), fmaxf(x[f][2], x[f][3])),
+                     fmaxf(fmaxf(x[f][4], x[f][5]), fmaxf(x[f][6], x[f][7])));
+    }
+    float mnA = mnf[0], mxA = mxf[0], mnB = mnf[FPB - 1], mxB = mxf[FPB - 1];
+    if constexpr (FPB == 2) {
+      mnA = mnB = fminf(mnf[0], mnf[1]);
+      mxA = mxB = fmaxf(mxf[0], mxf[1]);
+    }
+    if constexpr (FPB == 4) {
+      mnA = fminf(mnf[0], mnf[1]); mxA = fmaxf(mxf[0], mxf[1]);
+      mnB = fminf(mnf[2], mnf[3]); mxB = fmaxf(mxf[2], mxf[3]);
+      if (!split) {
+        mnA = mnB = fminf(mnA, mnB);
+        mxA = mxB = fmaxf(mxA, mxB);
+      }
     }
 #pragma unroll
-    for (int off = 1; off < 16; off <<= 1) {
+    for (int off = 1; off < LR; off <<= 1) {
       if (off < lpg) {
-        mn = fminf(mn, __shfl_xor_sync(FULL, mn, off));
-        mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, off));
+        mnA = fminf(mnA, __shfl_xor_sync(FULL, mnA, off));
+        mxA = fmaxf(mxA, __shfl_xor_sync(FULL, mxA, off));
+        if constexpr (FPB == 4) {
+          if (split) {
+            mnB = fminf(mnB, __shfl_xor_sync(FULL, mnB, off));
+            mxB = fmaxf(mxB, __shfl_xor_sync(FULL, mxB, off));
+          }
+        }
       }
     }
-    const GroupParams p = group_params(mn, mx, qmax);
-    if (!valid) continue;
-    if ((l & (lpg - 1)) == 0) meta_out[tau * ng + d0 / gsz] = p.meta;
-    uint32_t code[8];
+    const GroupParams pA = group_params(mnA, mxA, qmax);
+    GroupParams pB = pA;
+    if constexpr (FPB == 4) {
+      if (split) pB = group_params(mnB, mxB, qmax);
+    }
+    if (valid && (cs & (lpg - 1)) == 0) {
+      const int gi = (16 * FPB * mw) / gsz;                 // group of the lane's first field
+      meta_out[tau * ng + gi] = pA.meta;
+      if constexpr (FPB == 4) {
+        if (split) meta_out[tau * ng + gi + 1] = pB.meta;
+      }
+    }
+
+    // ---- codes as exact float integers, the FPB fields of a byte combined: byte = sum_f code_f * 2^(BITS f)
+    float bytev[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) code[i] = code_of_fast(x[i], p, qmax);
+    for (int i = 0; i < 8; ++i) bytev[i] = 0.f;
+#pragma unroll
+    for (int f = FPB - 1; f >= 0; --f) {
+      const GroupParams& p = (FPB == 4 && f >= 2) ? pB : pA;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float u = __fmul_rn(__fsub_rn(x[f][i], p.z), p.inv);
+        u = fminf(fmaxf(u, 0.0f), qmax);
+        const float r = __fsub_rn(__fadd_rn(u, kRoundMagic), kRoundMagic);      // rint(u), exact
+        bytev[i] = __fmaf_rn(bytev[i], (float)(1 << BITS), r);                  // exact: < 256
+      }
+    }
 
     if constexpr (!IS_V) {
-      // keys: channels d0..d0+3 and d0+4..d0+7 are the four bytes of one word each (chunks 2(l%2), 2(l%2)+1),
-      // register slot r = d0/16, field r % fpb of every byte
-      constexpr int FPB = 8 / BITS;
-      const int wpc = D * BITS / 128;
-      const int r = l >> 1;
-      const int sh = BITS * (r % FPB);
-      const int word = r / FPB;
-      const int row_words = D * BITS / 32;
+      // keys: bytes 0..3 of a word are channels 4 hh + {0..3} of this lane's 8, chunk 2 rh + hh, word mw of the row
+      if (valid) {
+        constexpr int wpc = D * BITS / 128;
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const uint32_t w = (code[4 * hh] | (code[4 * hh + 1] << 8) | (code[4 * hh + 2] << 16) |
-                            (code[4 * hh + 3] << 24)) << sh;
-        const int chunk = 2 * (l & 1) + hh;
-        atomicOr(&img[tau * row_words + chunk_word_byte(chunk, word, wpc, 4) / 4], w);
+        for (int hh = 0; hh < 2; ++hh) {
+          const uint32_t w = pack_bytes(bytev[4 * hh], bytev[4 * hh + 1], bytev[4 * hh + 2], bytev[4 * hh + 3]);
+          *reinterpret_cast<uint32_t*>(codes + (size_t)tau * K_ROW_BYTES + chunk_word_byte(2 * rh + hh, mw, wpc, 4)) = w;
+        }
       }
     } else {
-      // values: the lane's 8 channels d0 + kk belong to one lane-chunk group gidc = (d0/8) % 8, k = 8 (d0/64) + kk
-      constexpr int PPW = 16 / BITS;
-      const int wpc = D * BITS / 64;
-      const int gidc = l & 7, h = l >> 3;            // d0 = 64 h + 8 gidc
-      const int tidT = (tau & 7) >> 1, hiT = tau >> 3, oddT = tau & 1;
-      const int chunk = 4 * gidc + tidT;
-      constexpr int NWORD = BITS;                    // words this lane contributes to (8 codes, 8/BITS per word)
-      uint32_t part[NWORD], mask[NWORD];
-      int widx[NWORD];
 #pragma unroll
-      for (int i = 0; i < NWORD; ++i) { part[i] = 0; mask[i] = 0; widx[i] = 0; }
+      for (int i = 0; i < 8; ++i) vbyte[k & 3][i] = bytev[i];
+      if ((k & 3) == 3) {
+        // the four tokens (bytes) of this lane's words are complete: word of channel slot i at lane chunk 4 i + t
+        const int cmb = (k >> 2) * RS + rs;
+        uint8_t* wbase = codes + (size_t)(cmb >> 3) * (4 * D * BITS) + mw * 512 + (cmb & 3) * 16 +
+                         4 * (2 * rh + ((cmb >> 2) & 1));
+        const int t4 = 32 * (cmb >> 3) + 16 * ((cmb >> 2) & 1) + 2 * (cmb & 3);   // token of byte 0; bytes 1..3: +8, +1, +9
+        const bool v0 = t4 >= lo && t4 < hi, v1 = t4 + 8 >= lo && t4 + 8 < hi;
+        const bool v2 = t4 + 1 >= lo && t4 + 1 < hi, v3 = t4 + 9 >= lo && t4 + 9 < hi;
+        if (v0 && v1 && v2 && v3) {
 #pragma unroll
-      for (int kk = 0; kk < 8; ++kk) {
-        constexpr int NPOS = 8 / BITS;
-        const int k = 8 * h + kk;
-        const int word = k / NPOS;
-        const int field = k % NPOS + NPOS * hiT + PPW * oddT;
-        const int wo = kk / NPOS;
-        widx[wo] = word;
-        part[wo] |= code[kk] << (field * BITS);
-        mask[wo] |= ((1u << BITS) - 1u) << (field * BITS);
-      }
+          for (int i = 0; i < 8; ++i)
+            *reinterpret_cast<uint32_t*>(wbase + 64 * i) = pack_bytes(vbyte[0][i], vbyte[1][i], vbyte[2][i], vbyte[3][i]);
+        } else if (v0 || v1 || v2 || v3) {
 #pragma unroll
-      for (int i = 0; i < NWORD; ++i) {
-        uint32_t* dst = &img[chunk_word_byte(chunk, widx[i], wpc, 32) / 4];
-        if (clear_first) atomicAnd(dst, ~mask[i]);
-        atomicOr(dst, part[i]);
+          for (int i = 0; i < 8; ++i) {
+            if (v0) wbase[64 * i + 0] = (uint8_t)vbyte[0][i];
+            if (v1) wbase[64 * i + 1] = (uint8_t)vbyte[1][i];
+            if (v2) wbase[64 * i + 2] = (uint8_t)vbyte[2][i];
+            if (v3) wbase[64 * i + 3] = (uint8_t)vbyte[3][i];
+          }
+        }
       }
     }
   }
 }
 
-// 16-bit passthrough of one side of a tile: rows [lo, hi) copied to the page as they are.
-__device__ __forceinline__ void copy_tile_side(const uint16_t* __restrict__ src, int64_t st, int D, int lo, int hi,
+// 16-bit passthrough of one side of a task: rows [lo, hi) copied to the page as they are.
+__device__ __forceinline__ void copy_task_side(const uint16_t* __restrict__ src, int64_t st, int D, int lo, int hi,
                                                uint16_t* __restrict__ dst_rows, int lane) {
   const int lpr = D >> 3, rps = 32 / lpr, l = lane & (lpr - 1);
-  for (int step = 0; step < 16 / rps; ++step) {
-    if (step * rps + rps <= lo || step * rps >= hi) continue;
-    const int tau = step * rps + lane / lpr;
-    if (tau >= lo && tau < hi)
-      *reinterpret_cast<uint4*>(dst_rows + (size_t)tau * D + l * 8) =
-          *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + l * 8);
-  }
+  for (int row = lo + lane / lpr; row < hi; row += rps)
+    *reinterpret_cast<uint4*>(dst_rows + (size_t)row * D + l * 8) =
+        *reinterpret_cast<const uint4*>(src + (int64_t)row * st + l * 8);
 }
 
-template <bool IS_V, int D, int DTYPE, bool ROT>
-__device__ __forceinline__ void quantize_tile_side_bits(int bits, const uint16_t* src, int64_t st, int gsz,
-                                                        int lo, int hi, uint32_t* img, uint32_t* meta_out,
-                                                        bool clear_first, int lane, const int8_t* signs) {
-  if (bits == 2)
-    quantize_tile_side<2, IS_V, D, DTYPE, ROT>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane, signs);
-  else if (bits == 4)
-    quantize_tile_side<4, IS_V, D, DTYPE, ROT>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane, signs);
-  else
-    quantize_tile_side<8, IS_V, D, DTYPE, ROT>(src, st, gsz, lo, hi, img, meta_out, clear_first, lane, signs);
+// An append of t_new tokens at position t0 fits the cache; written without a sum that could overflow.
+__host__ __device__ __forceinline__ bool append_fits(int t0, int t_new, int capacity) {
+  return t0 >= 0 && t0 <= capacity - t_new;
 }
 
-// Token-wise quantization of V (always) and of K (when do_k).  grid.y = stream, grid.x strides over the
-// 16-token tiles touched by this append, one warp per tile.
+// Token-wise quantization of V (blockIdx.z == 0) and of K (blockIdx.z == 1).  grid.y = stream, grid.x strides
+// over the warp tasks touched by this append.
 template <int D, int DTYPE>
 __global__ void __launch_bounds__(kThreads)
 quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
-                   int64_t sb, int64_t sh, int64_t st, int t_new, int do_k) {
-  __shared__ __align__(16) uint32_t sImg[kWarps][2][512];   // per warp: key image, value image (<= 2 KB each)
+                   int64_t sb, int64_t sh, int64_t st, int t_new) {
+  const bool is_v = blockIdx.z == 0;
   const int bh = blockIdx.y;
   const int b = bh / g.Hkv, h = bh % g.Hkv;
   const int t0 = c.seq_len[b];
-  if (t0 < 0 || t0 + t_new > g.capacity) return;
+  if (!append_fits(t0, t_new, g.capacity)) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int first_tile = t0 >> 4;
-  const int n_tiles = ((t0 + t_new + 15) >> 4) - first_tile;
-  uint32_t* kimg = sImg[warp][0];
-  uint32_t* vimg = sImg[warp][1];
-  const int k_row_words = D * g.kb / 32;          // words per key row (quantized)
-  const int v_tile_words = D * g.vb / 2;          // words per value tile (quantized)
+  const int bits = is_v ? g.vb : g.kb;
+  const int TT = bits == 16 ? 32 : task_tokens(D, bits);
+  const int first_task = t0 / TT;
+  const int n_tasks = (t0 + t_new + TT - 1) / TT - first_task;
+  const uint16_t* in = is_v ? v_new : k_new;
+  const int gsz = is_v ? g.gv : g.gk;
 
-  for (int j = blockIdx.x * kWarps + warp; j < n_tiles; j += gridDim.x * kWarps) {
-    const int tile = first_tile + j;
-    const int tbeg = max(t0, tile * 16), tend = min(t0 + t_new, tile * 16 + 16);
-    const int lo = tbeg & 15, hi = lo + (tend - tbeg);
-    const bool full = (hi - lo) == 16;
-    const int page = tile >> 3, tp0 = (tile & 7) * 16;        // page-local token of the tile's first row
+  for (int j = blockIdx.x * kWarps + warp; j < n_tasks; j += gridDim.x * kWarps) {
+    const int tk0 = (first_task + j) * TT;                     // first token of the task
+    const int lo = max(t0, tk0) - tk0, hi = min(t0 + t_new, tk0 + TT) - tk0;
+    const int page = tk0 >> 7, tp0 = tk0 & 127;                // page-local token of the task's first row
     uint8_t* pg = c.pages + ((size_t)bh * g.n_pages + page) * g.page_bytes;
-    // row 0 of the tile in the input (may lie before the first new token; never dereferenced there)
-    const int64_t off = (int64_t)b * sb + (int64_t)h * sh + (int64_t)(tile * 16 - t0) * st;
-
-    // ---- values
-    if (g.vb == 16) {
-      copy_tile_side(v_new + off, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg + g.v_codes_off) + (size_t)tp0 * D, lane);
+    // row 0 of the task in the input (may lie before the first new token; never dereferenced there)
+    const uint16_t* src = in + (int64_t)b * sb + (int64_t)h * sh + (int64_t)(tk0 - t0) * st;
+    if (is_v) {
+      if (bits == 16) {
+        copy_task_side(src, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg + g.v_codes_off) + (size_t)tp0 * D, lane);
+        continue;
+      }
+      uint8_t* vb = pg + g.v_codes_off + (size_t)(tp0 >> 5) * (4 * D * bits);
+      uint32_t* vm = reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / gsz);
+      if (bits == 2) quantize_task<2, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane, nullptr);
+      else if (bits == 4) quantize_task<4, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane, nullptr);
+      else quantize_task<8, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane, nullptr);
     } else {
-      uint4* gv = reinterpret_cast<uint4*>(pg + g.v_codes_off + (size_t)(tile & 7) * (v_tile_words * 4));
-      for (int i = lane; i < v_tile_words / 4; i += 32)
-        reinterpret_cast<uint4*>(vimg)[i] = full ? make_uint4(0u, 0u, 0u, 0u) : gv[i];
-      __syncwarp();
-      quantize_tile_side_bits<true, D, DTYPE, false>(g.vb, v_new + off, st, g.gv, lo, hi, vimg,
-                                    reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / g.gv), !full, lane,
-                                    nullptr);
-      __syncwarp();
-      for (int i = lane; i < v_tile_words / 4; i += 32) gv[i] = reinterpret_cast<const uint4*>(vimg)[i];
-    }
-    // ---- keys
-    if (do_k) {
-      if (g.kb == 16) {
-        copy_tile_side(k_new + off, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg) + (size_t)tp0 * D, lane);
+      if (bits == 16) {
+        copy_task_side(src, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg) + (size_t)tp0 * D, lane);
+        continue;
+      }
+      uint8_t* kr = pg + (size_t)tp0 * (D * bits / 8);
+      uint32_t* km = reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / gsz);
+      if (c.k_signs) {
+        if (bits == 2) quantize_task<2, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
+        else if (bits == 4) quantize_task<4, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
+        else quantize_task<8, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
       } else {
-        for (int i = lane; i < 16 * k_row_words / 4; i += 32) reinterpret_cast<uint4*>(kimg)[i] = make_uint4(0u, 0u, 0u, 0u);
-        __syncwarp();
-        uint32_t* kmeta = reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / g.gk);
-        if (c.k_signs)
-          quantize_tile_side_bits<false, D, DTYPE, true>(g.kb, k_new + off, st, g.gk, lo, hi, kimg, kmeta, false,
-                                                         lane, c.k_signs);
-        else
-          quantize_tile_side_bits<false, D, DTYPE, false>(g.kb, k_new + off, st, g.gk, lo, hi, kimg, kmeta, false,
-                                                          lane, nullptr);
-        __syncwarp();
-        uint4* gk = reinterpret_cast<uint4*>(pg + (size_t)tp0 * (k_row_words * 4));
-        const int v_lo = lo * k_row_words / 4, v_hi = hi * k_row_words / 4;   // 16-byte vectors of the new rows
-        for (int i = v_lo + lane; i < v_hi; i += 32) gk[i] = reinterpret_cast<const uint4*>(kimg)[i];
+        if (bits == 2) quantize_task<2, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane, nullptr);
+        else if (bits == 4) quantize_task<4, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane, nullptr);
+        else quantize_task<8, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane, nullptr);
       }
     }
-    __syncwarp();
   }
 }
 
@@ -248,7 +372,7 @@ quant_kchan_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new,
   const int bh = blockIdx.y;
   const int b = bh / g.Hkv, h = bh % g.Hkv;
   const int t0 = c.seq_len[b];
-  if (t0 < 0 || t0 + t_new > g.capacity) return;
+  if (!append_fits(t0, t_new, g.capacity)) return;
   const int end = t0 + t_new;
   const int first_page = t0 >> 7;
   const int nblk = ((end + 127) >> 7) - first_page;
@@ -331,7 +455,7 @@ __global__ void bump_seq_len_kernel(Geom g, CachePtrs c, int t_new) {
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= g.B) return;
   int t0 = c.seq_len[b];
-  if (t0 < 0 || t0 + t_new > g.capacity) {
+  if (!append_fits(t0, t_new, g.capacity)) {
     atomicOr(c.status, KVQ_STATUS_CAPACITY);
   } else {
     c.seq_len[b] = t0 + t_new;
@@ -344,22 +468,21 @@ int launch_quantize_append(const Geom& g, const CachePtrs& c, const void* k_new,
                            int64_t sb, int64_t sh, int64_t st, int t_new, cudaStream_t stream) {
   const uint16_t* k = static_cast<const uint16_t*>(k_new);
   const uint16_t* v = static_cast<const uint16_t*>(v_new);
-  // tiles touched per stream: at most ceil(t_new / 16) + 1; one warp per tile, CTAs stride over them
-  const int max_tiles = (t_new + 15) / 16 + 1;
-  int gx = (max_tiles + kWarps - 1) / kWarps;
+  // warp tasks touched per stream: at most ceil(t_new / 32) + 1; one warp per task, CTAs stride over them
+  const int max_tasks = (t_new + 31) / 32 + 1;
+  int gx = (max_tasks + kWarps - 1) / kWarps;
   const int streams = g.B * g.Hkv;
-  const int want = (148 * 16 + streams - 1) / streams;       // enough CTAs to fill the GPU, not one per tile
+  const int want = (148 * 16 + streams - 1) / streams;       // enough CTAs to fill the GPU, not one per task
   if (gx > want) gx = want;
-  dim3 grid1(gx, streams);
-  const int do_k = g.k_axis == 0 ? 1 : 0;
+  dim3 grid1(gx, streams, g.k_axis == 0 ? 2 : 1);            // z = 0 values, z = 1 token-wise keys
   if (g.D == 128 && g.in_dtype == KVQ_BF16)
-    quant_token_kernel<128, KVQ_BF16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, do_k);
+    quant_token_kernel<128, KVQ_BF16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
   else if (g.D == 128)
-    quant_token_kernel<128, KVQ_FP16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, do_k);
+    quant_token_kernel<128, KVQ_FP16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
   else if (g.in_dtype == KVQ_BF16)
-    quant_token_kernel<64, KVQ_BF16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, do_k);
+    quant_token_kernel<64, KVQ_BF16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
   else
-    quant_token_kernel<64, KVQ_FP16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new, do_k);
+    quant_token_kernel<64, KVQ_FP16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
   if (g.k_axis == 1) {
     size_t smem = (size_t)kPageTokens * g.D * 3;
     cudaFuncSetAttribute(quant_kchan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 3);
