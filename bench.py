@@ -7,11 +7,13 @@ attention over the full context, and a dequantize of the newest 128-token page.
 The reported value is the packed K + V + metadata bytes the decode step has to
 stream (all layers) divided by the step time, in GB/s.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--sweep]
 
-N > 1 runs under torchrun, one rank per GPU; the path shards by batch with no
-collective, so every rank runs the same per-GPU workload (weak scaling).
+N > 1: one rank per GPU (started here through torch.distributed.run when the
+launcher has not already done so); the path shards by batch with no collective,
+so every rank runs the same per-GPU workload (weak scaling).
 `--impl reference` times the CPU oracle on a bounded sample of the workload.
+`--sweep` runs every model-shaped variant once and prints one line per variant.
 """
 from __future__ import annotations
 
@@ -19,9 +21,11 @@ import argparse
 import hashlib
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
+import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -34,17 +38,18 @@ from paper_2502_15075_b200 import workloads as wl  # noqa: E402
 
 METRIC = "decode-attention HBM GB/s (packed K+V+metadata bytes per decode step / time), K4V2, 32k context"
 UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (bytes), keyed by the sha256 of the
-# kernel source it was taken from; reported as null once that file has changed.
-NCU_TRAFFIC = {"ba0a2a7127d6efbb20d92d017f81aa64248ffbac0e25a1297d0c33a0fe1c0a80": 441370368}   # dram read 436.51 MB + write 4.86 MB
+# kernel source it was taken from; reported as null once that source has changed.
+NCU_TRAFFIC = {}
 DECODE_KERNEL_SOURCES = ("kvq_decode_mma.cuh", "kvq_decode_mma_kernel.cuh", "kvq_decode_mma_list.inc")
+
+WORKLOADS = {"tiny": wl.TINY, "1b": wl.LLAMA_1B, "8b": wl.LLAMA_8B, "14b": wl.SHAPED_14B, "70b": wl.LLAMA_70B}
 
 
 def workload_from_env() -> wl.Workload:
-    name = os.environ.get("KVQ_BENCH_WORKLOAD", "8b")
-    table = {"tiny": wl.TINY, "1b": wl.LLAMA_1B, "8b": wl.LLAMA_8B, "14b": wl.SHAPED_14B, "70b": wl.LLAMA_70B}
-    w = table[name]
+    w = WORKLOADS[os.environ.get("KVQ_BENCH_WORKLOAD", "8b")]
     if "KVQ_BENCH_LAYERS" in os.environ:
         w = w.with_(layers=int(os.environ["KVQ_BENCH_LAYERS"]))
     if "KVQ_BENCH_CONTEXT" in os.environ:
@@ -55,8 +60,22 @@ def workload_from_env() -> wl.Workload:
     return w
 
 
-def decode_bytes_per_layer(w: wl.Workload) -> float:
-    return w.batch * w.n_kv_heads * w.context * wl.packed_bytes_per_token(w)
+def decode_bytes_per_layer(w: wl.Workload, tokens=None) -> float:
+    """Algorithmic bytes of one decode launch: packed K + V + metadata of every cached token (the fp16 tail of an
+    incomplete channel-wise block counts as its 2 bytes per key element)."""
+    T = w.context if tokens is None else tokens
+    streams = w.batch * w.n_kv_heads
+    if w.k_axis == 1 and T % 128:
+        full, tail = T - T % 128, T % 128
+        v_tok = w.head_dim * w.vb / 8 + (0.0 if w.vb == 16 else 4.0 * w.head_dim / w.gv)
+        return streams * (full * wl.packed_bytes_per_token(w) + tail * (v_tok + 2.0 * w.head_dim))
+    return streams * T * wl.packed_bytes_per_token(w)
+
+
+def source_bytes_per_layer(w: wl.Workload, tokens=None) -> float:
+    """16-bit K and V of one layer."""
+    T = w.context if tokens is None else tokens
+    return 2.0 * w.batch * w.n_kv_heads * T * w.head_dim * 2
 
 
 def dist_env():
@@ -79,49 +98,74 @@ def whole_job_gbs(bytes_per_rank_step: float, ms_per_step: float, world: int) ->
     return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
 
 
+def free_port() -> int:
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def respawn_under_launcher(n: int) -> None:
+    """`bench.py --gpus N` started without a launcher: start N ranks of this same command (one per GPU)."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    os.execv(sys.executable, cmd)
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """SM clock and throttle reasons sampled every few milliseconds during the timed region (NVML, read-only)."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
-    def __init__(self, index: int):
-        self.proc = None
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.sm, self.reasons, self.max_mhz, self.err = [], set(), None, None
+        self._stop = threading.Event()
+        self._thr = None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "50", "-i", str(index)], stdout=subprocess.PIPE,
-                                         stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            pass
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:                         # noqa: BLE001
+            self.err = f"nvml unavailable: {e}"
+            return
+        self._period = period_s
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h) if hasattr(
+                    nv, "nvmlDeviceGetCurrentClocksEventReasons") else nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in self.REASONS.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception as e:                     # noqa: BLE001
+                self.err = str(e)
+                return
+            self._stop.wait(self._period)
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-            out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0]))
-                mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join(timeout=2)
+        if not self.sm:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "samples": 0, "reasons": [self.err or "no samples"]}
+        return {"sm_mhz": statistics.median(self.sm), "sm_min_mhz": min(self.sm), "sm_max_mhz": self.max_mhz,
+                "samples": len(self.sm), "reasons": sorted(self.reasons)}
 
 
 # ----------------------------------------------------------------------------- oracle legs
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
 def oracle_sample_cache(w: wl.Workload, layer: int = 0):
     """One (batch, kv-head) stream of the workload at full context, built by the oracle on the CPU."""
     from oracle.cache import OracleCache
@@ -170,77 +214,148 @@ def run_reference(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": config_dict(w),
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "host_cores_available": host_cores(),
+                             "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
 
-def config_dict(w: wl.Workload):
+def config_dict(w: wl.Workload, tokens=None, ragged=False):
+    T = w.context if tokens is None else tokens
     return {"workload": f"{w.name}: {w.layers} layers, batch {w.batch}, {w.n_q_heads}q/{w.n_kv_heads}kv heads, "
-                        f"head_dim {w.head_dim}, context {w.context}, {w.dtype}, K{w.kb}V{w.vb}, "
-                        f"group {w.gk}/{w.gv}, k_axis {w.k_axis}",
+                        f"head_dim {w.head_dim}, context {T}{' (ragged U(T/2,T))' if ragged else ''}, {w.dtype}, "
+                        f"K{w.kb}V{w.vb}, group {w.gk}/{w.gv}, k_axis {w.k_axis}",
             "step": "per layer: append 1 token/sequence, decode attention over the full context, "
                     "dequantize the newest page",
-            "l2": "inputs larger than L2 (one layer's packed cache exceeds it and layers rotate)",
+            "l2": ("inputs larger than L2 (one layer's packed cache exceeds it and layers rotate)"
+                   if decode_bytes_per_layer(w, T) * w.layers > 2.5e8 else
+                   "working set below L2 capacity: launch/L2-bound, not HBM-bound"),
             "parallelism": "replicas (batch-sharded, no collective)"}
 
 
-# ----------------------------------------------------------------------------- GPU arm
-def main_gpu(args):
-    rank, local_rank, world = dist_env()
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    from paper_2502_15075_b200 import build
-    if rank == 0:
-        build.build()
-    if world > 1:
-        dist.barrier()
-    from paper_2502_15075_b200 import kvq
+def oracle_leg(kvq, w, cfg, cache, q, out_gpu, budget_s=12.0):
+    """Time the oracle's decode on sampled streams of layer 0 (about 10-30 s of CPU work) and check the GPU
+    output of those streams against it."""
+    from threadpoolctl import threadpool_limits
+    from oracle.cache import OracleCache
+    B, H = w.batch, w.n_kv_heads
+    G = w.n_q_heads // H
+    cap = cfg.capacity_tokens
+    pages = cache.pages_view()
+    qb = q.cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+    seq = cache.seq_len.cpu().numpy()
+    n_streams = B * H
+    order = [(i * 37) % n_streams for i in range(min(n_streams, 48))]      # a fixed spread over the streams
+    streams = [(s // H, s % H) for s in dict.fromkeys(order)]
+    got_all = out_gpu.double().cpu().numpy()
+    t_used, n_done, n_tok, errs = 0.0, 0, 0, []
+    with threadpool_limits(limits=1):
+        for (b, h) in streams:
+            oc = OracleCache(1, 1, w.head_dim, w.kb, w.vb, w.gk, w.gv, w.k_axis, w.dtype, cap)
+            oc.pages = pages[b:b + 1, h:h + 1].cpu().numpy().copy()
+            if oc.k_tail is not None:
+                oc.k_tail = cache.tail_view()[b:b + 1, h:h + 1].cpu().view(torch.int16).numpy().view(np.uint16).copy()
+            oc.seq_len[:] = seq[b]
+            t0 = time.perf_counter()
+            want = oc.decode(qb[b:b + 1, h * G:(h + 1) * G])
+            t_used += time.perf_counter() - t0
+            n_done += 1
+            n_tok += int(seq[b])
+            got = got_all[b:b + 1, h * G:(h + 1) * G]
+            den = np.linalg.norm(want)
+            errs.append((float(np.linalg.norm(got - want) / (den if den > 0 else 1.0)), float(np.abs(got - want).max())))
+            if t_used > budget_s:
+                break
+    sample_bytes = n_tok * wl.packed_bytes_per_token(w)
+    return {"baseline": {"value": sample_bytes / t_used / 1e9, "unit": UNIT, "cores": 1,
+                         "host_cores_available": host_cores(), "kind": "oracle",
+                         "sample": f"decode attention of {n_done} of {B * H} (batch, kv-head) streams of layer 0 at "
+                                   f"full context, {t_used:.1f} s"},
+            "parity": {"streams": n_done, "rel_l2_max": max(e[0] for e in errs), "max_abs_max": max(e[1] for e in errs),
+                       "tolerance": {"rel_l2": 2e-3, "max_abs": 1e-2}}}
 
-    w = workload_from_env()
-    T, B, L = w.context, w.batch, w.layers
+
+def peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def stats_us(ms_list):
+    return {"median": statistics.median(ms_list) * 1e3, "min": min(ms_list) * 1e3,
+            "mean": sum(ms_list) / len(ms_list) * 1e3, "n": len(ms_list)}
+
+
+def hbm_block(kernel, bytes_per_launch, us, peak, peak_src, traffic=None, note=None):
+    ach = bytes_per_launch / (us["median"] * 1e-6) / 1e9
+    d = {"bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+         "frac": ach / peak, "frac_of_8TBps_nominal": ach / NOMINAL_HBM_GBS, "us_per_launch": us["median"],
+         "us_per_launch_min": us["min"], "us_per_launch_mean": us["mean"], "launches_timed": us["n"],
+         "algorithmic_bytes_per_launch": bytes_per_launch, "traffic": traffic}
+    if note:
+        d["note"] = note
+    return d
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, warmup: int, tokens=None,
+                 ragged=False, append_tokens=0, oracle_budget_s=12.0, do_e2e=True):
+    """Build all layers of `w` on the device, then time `steps` steps of the hot path.  Returns the result line."""
+    import torch.distributed as dist
+    T, B, L = (w.context if tokens is None else tokens), w.batch, w.layers
     cap = ((T + 127) // 128) * 128 + 128
     cfg = kvq.make_config(B, w.n_q_heads, w.n_kv_heads, w.head_dim, w.kb, w.vb, w.gk, w.gv, w.k_axis,
                           w.torch_dtype, cap)
     ws_buf = torch.empty(max(16, kvq.kvq_workspace_bytes(cfg)), dtype=torch.uint8, device=dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)  # noqa: E731
 
     # ---- build all layers (bulk quantize-append of T-1 tokens), timing the quantizer
     caches, qs, k1s, v1s = [], [], [], []
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    quant_ms = []
+    quant_ms, append_ms = [], []
+    bulk = T - 1 - append_tokens
     for layer in range(L):
-        k, v = wl.make_kv(w, layer=layer + 100 * rank, device=dev)
+        k, v = wl.make_kv(w, layer=layer + 100 * rank, device=dev, tokens=T)
         c = kvq.Cache(cfg, device=dev)
+        e0, e1, e2 = ev(), ev(), ev()
         e0.record()
-        kvq.kvq_quantize_append(cfg, c, k[:, :, :T - 1], v[:, :, :T - 1])
+        kvq.kvq_quantize_append(cfg, c, k[:, :, :bulk], v[:, :, :bulk])
         e1.record()
+        if append_tokens:
+            kvq.kvq_quantize_append(cfg, c, k[:, :, bulk:T - 1], v[:, :, bulk:T - 1])
+        e2.record()
         torch.cuda.synchronize()
         quant_ms.append(e0.elapsed_time(e1))
+        if append_tokens:
+            append_ms.append(e1.elapsed_time(e2))
         caches.append(c)
         k1s.append(k[:, :, T - 1:].contiguous())
         v1s.append(v[:, :, T - 1:].contiguous())
         qs.append(wl.make_q(w, layer=layer + 100 * rank, device=dev))
         del k, v
-    quant_ms_med = statistics.median(quant_ms[1:] or quant_ms)
-    quant_tokens_s = B * (T - 1) / (quant_ms_med * 1e-3)
-    quant_gbs = (2 * B * w.n_kv_heads * (T - 1) * w.head_dim * 2 + decode_bytes_per_layer(w)) / (quant_ms_med * 1e-3) / 1e9
+    lens = None
+    if ragged:
+        lens = wl.ragged_seq_lens(w, T, B).to(dev)
+    q_us = stats_us(quant_ms[1:] or quant_ms)
 
     outs = [torch.empty((B, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev) for _ in range(L)]
     page0 = ((T - 1) // 128) * 128
     deq_k = torch.empty((B, w.n_kv_heads, cap, w.head_dim), dtype=w.torch_dtype, device=dev)
     deq_v = torch.empty_like(deq_k)
 
+    def reset_len(c):
+        if lens is None:
+            c.seq_len.fill_(T - 1)
+        else:
+            c.seq_len.copy_(lens - 1)
+
     def step_device(events=None):
         for i in range(L):
             c = caches[i]
-            c.seq_len.fill_(T - 1)
+            reset_len(c)
             kvq.kvq_quantize_append(cfg, c, k1s[i], v1s[i])
             if events is not None:
-                a = torch.cuda.Event(enable_timing=True)
-                b_ = torch.cuda.Event(enable_timing=True)
+                a, b_ = ev(), ev()
                 a.record()
             kvq.kvq_decode_attention(cfg, c, qs[i], outs[i], ws_buf)
             if events is not None:
@@ -258,7 +373,7 @@ def main_gpu(args):
     def step_e2e():
         for i in range(L):
             c = caches[i]
-            c.seq_len.fill_(T - 1)
+            reset_len(c)
             kvq.quantize_append_host(cfg, c, hk[i], hv[i], dk, dv)
             kvq.decode_attention_host(cfg, c, hq[i], hout[i], dq, outs[i], ws_buf)
             kvq.kvq_dequantize(cfg, c, deq_k, deq_v, page0, T)
@@ -269,110 +384,154 @@ def main_gpu(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    def timed(fn, steps, events=None):
+    def timed(fn, n, events=None):
         barrier()
-        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s, e = ev(), ev()
         s.record()
-        for _ in range(steps):
+        for _ in range(n):
             fn(events) if events is not None else fn()
         e.record()
         barrier()
         return max_over_ranks(s.elapsed_time(e), world, dev)
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step_device()
+    local_rank = dev.index or 0
     sampler = ClockSampler(local_rank) if rank == 0 else None
     events = []
-    total_ms = timed(step_device, args.steps, events)
+    total_ms = timed(step_device, steps, events)
     clocks = sampler.stop() if sampler else None
-    ms_per_step = total_ms / args.steps
-    dec_ms = [a.elapsed_time(b_) for a, b_ in events]
-    dec_ms_avg = sum(dec_ms) / len(dec_ms)
+    ms_per_step = total_ms / steps
+    dec_us = stats_us([a.elapsed_time(b_) for a, b_ in events])
 
-    for _ in range(max(1, args.warmup // 2)):
-        step_e2e()
-    e2e_ms = timed(step_e2e, args.steps) / args.steps
+    e2e_ms = None
+    if do_e2e:
+        for _ in range(max(1, warmup // 2)):
+            step_e2e()
+        e2e_ms = timed(step_e2e, steps) / steps
+
+    # ---- dequantize of whole layers (reads the packed layer, writes 16-bit K and V), layers rotating
+    deq_ms = []
+    for r in range(min(max(4, L), 12) + 1):
+        c = caches[r % L]
+        a, b_ = ev(), ev()
+        a.record()
+        kvq.kvq_dequantize(cfg, c, deq_k, deq_v, 0, T)
+        b_.record()
+        torch.cuda.synchronize()
+        if r:
+            deq_ms.append(a.elapsed_time(b_))
+    dq_us = stats_us(deq_ms)
     if kvq.kvq_check_status(caches[0]) != 0:
         raise RuntimeError("library reported a status error")
 
-    bytes_layer = decode_bytes_per_layer(w)
+    n_tok = T if lens is None else float(lens.sum().item()) / B      # mean cached tokens per sequence
+    bytes_layer = decode_bytes_per_layer(w, T) * (n_tok / T)
     bytes_step = bytes_layer * L
     value = whole_job_gbs(bytes_step, ms_per_step, world)
-    e2e_value = whole_job_gbs(bytes_step, e2e_ms, world)
-
     if rank != 0:
-        return
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
-    else:
-        peak, peak_src = 6650.0, "fallback"
-    achieved = bytes_layer / (dec_ms_avg * 1e-3) / 1e9
+        return None
+    peak, peak_src = peak_hbm()
     hsh = hashlib.sha256()
     for name in DECODE_KERNEL_SOURCES:
         hsh.update(open(os.path.join(ROOT, "paper_2502_15075_b200", "csrc", name), "rb").read())
-    sha = hsh.hexdigest()
-    roofline = {"bound": "hbm", "kernel": "kvq_decode_attention (split kernel + merge)", "achieved": achieved,
-                "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                "frac_of_8TBps_nominal": achieved / 8000.0, "us_per_launch": dec_ms_avg * 1e3,
-                "algorithmic_bytes_per_launch": bytes_layer, "traffic": NCU_TRAFFIC.get(sha)}
+    traffic = NCU_TRAFFIC.get(hsh.hexdigest()) if (w.name, w.kb, w.vb, T, ragged) == (wl.LLAMA_8B.name, 4, 2, 32768, False) else None
+    roofline = hbm_block("kvq_decode_attention (one fused kernel: split decode + merge)", bytes_layer, dec_us, peak,
+                         peak_src, traffic)
+    src_bulk = source_bytes_per_layer(w, bulk)
+    packed_bulk = decode_bytes_per_layer(w, T) * bulk / T
+    roof_q = hbm_block("kvq_quantize_append, bulk build of one layer (reads 16-bit K and V, writes the packed layer)",
+                       src_bulk + packed_bulk, q_us, peak, peak_src)
+    roof_dq = hbm_block("kvq_dequantize of one whole layer (reads the packed layer, writes 16-bit K and V)",
+                        decode_bytes_per_layer(w, T) + source_bytes_per_layer(w, T), dq_us, peak, peak_src)
 
-    # ---- CPU oracle on a bounded sample of the same workload, with a parity check of the GPU output
-    cpu = oracle_leg(kvq, w, cfg, caches[0], qs[0], outs[0])
-
-    n_launch = L * (2 + 2 + 1 + (1 if w.k_axis == 1 else 0))   # append (quantize [+ K channel] + bump), decode + merge, dequantize
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32 accumulate over f16 operands", "data": "synthetic",
-            "config": config_dict(w), "roofline": roofline, "cpu_baseline": cpu["baseline"],
-            "parity_sample": cpu["parity"],
-            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": L * (2 * k1s[0].numel() * 2 + qs[0].numel() * 2),
-                    "d2h_bytes_per_step": L * outs[0].numel() * 4},
-            "gpu_launches": n_launch * args.steps,
-            "quantize": {"tokens_per_s": quant_tokens_s * world, "ms_per_layer_bulk": quant_ms_med,
-                         "GBps_read_plus_write": quant_gbs, "tokens_per_call": B * (T - 1)},
+    cpu = oracle_leg(kvq, w, cfg, caches[0], qs[0], outs[0], oracle_budget_s)
+    kern_per_layer = (2 if w.k_axis == 0 else 3) + 1 + 1      # append (quantize [+ channel-wise K] + bump), decode, dequantize
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int32 accumulate over 8-bit operands (fp32 softmax and merge)",
+            "data": "synthetic", "config": config_dict(w, T, ragged), "roofline": roofline,
+            "roofline_quantize": roof_q, "roofline_dequantize": roof_dq,
+            "cpu_baseline": cpu["baseline"], "parity_sample": cpu["parity"],
+            "gpu_launches": L * kern_per_layer * steps,
+            "quantize": {"tokens_per_s": world * B * bulk / (q_us["median"] * 1e-6), "us_per_layer_bulk": q_us,
+                         "tokens_per_call": B * bulk},
             "clocks": clocks}
-    print(json.dumps(line))
+    if e2e_ms is not None:
+        line["e2e"] = {"value": whole_job_gbs(bytes_step, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
+                       "h2d_bytes_per_step": L * (2 * k1s[0].numel() * 2 + qs[0].numel() * 2),
+                       "d2h_bytes_per_step": L * outs[0].numel() * 4}
+    if append_ms:
+        a_us = stats_us(append_ms[1:] or append_ms)
+        line["append"] = {"tokens_per_call": B * append_tokens, "us_per_call": a_us,
+                          "tokens_per_s": B * append_tokens / (a_us["median"] * 1e-6)}
+    return line
 
 
-def oracle_leg(kvq, w, cfg, cache, q, out_gpu):
-    """Time the oracle's decode on sampled streams of layer 0 (about 10-30 s of CPU work) and check the GPU
-    output of those streams against it."""
-    from threadpoolctl import threadpool_limits
-    from oracle.cache import OracleCache
-    B, H = w.batch, w.n_kv_heads
-    G = w.n_q_heads // H
-    cap = cfg.capacity_tokens
-    pages = cache.pages_view()
-    qb = q.cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
-    seq = cache.seq_len.cpu().numpy()
-    n_streams = B * H
-    order = [(i * 37) % n_streams for i in range(min(n_streams, 48))]      # a fixed spread over the streams
-    streams = [(s // H, s % H) for s in dict.fromkeys(order)]
-    got_all = out_gpu.double().cpu().numpy()
-    t_used, n_done, errs = 0.0, 0, []
-    with threadpool_limits(limits=1):
-        for (b, h) in streams:
-            oc = OracleCache(1, 1, w.head_dim, w.kb, w.vb, w.gk, w.gv, w.k_axis, w.dtype, cap)
-            oc.pages = pages[b:b + 1, h:h + 1].cpu().numpy().copy()
-            if oc.k_tail is not None:
-                oc.k_tail = cache.tail_view()[b:b + 1, h:h + 1].cpu().view(torch.int16).numpy().view(np.uint16).copy()
-            oc.seq_len[:] = seq[b]
-            t0 = time.perf_counter()
-            want = oc.decode(qb[b:b + 1, h * G:(h + 1) * G])
-            t_used += time.perf_counter() - t0
-            n_done += 1
-            got = got_all[b:b + 1, h * G:(h + 1) * G]
-            errs.append((float(np.linalg.norm(got - want) / np.linalg.norm(want)), float(np.abs(got - want).max())))
-            if t_used > 12.0:
-                break
-    sample_bytes = n_done * w.context * wl.packed_bytes_per_token(w)
-    return {"baseline": {"value": sample_bytes / t_used / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": f"decode attention of {n_done} of {B * H} (batch, kv-head) streams of layer 0 at "
-                                   f"full context, {t_used:.1f} s"},
-            "parity": {"streams": n_done, "rel_l2_max": max(e[0] for e in errs), "max_abs_max": max(e[1] for e in errs),
-                       "tolerance": {"rel_l2": 2e-3, "max_abs": 1e-2}}}
+SWEEP = (
+    # (label, workload key, overrides, tokens, ragged, append_tokens)
+    ("tiny K4V2 g32", "tiny", {}, None, False, 0),
+    ("1B-shaped K4V2 g64, bulk 3968 + append 128", "1b", {}, None, False, 127),
+    ("8B-shaped K4V2", "8b", {}, None, False, 0),
+    ("8B-shaped K2V4", "8b", {"kb": 2, "vb": 4}, None, False, 0),
+    ("8B-shaped K4V4", "8b", {"kb": 4, "vb": 4}, None, False, 0),
+    ("8B-shaped K8V4", "8b", {"kb": 8, "vb": 4}, None, False, 0),
+    ("8B-shaped K4V2, ragged lengths", "8b", {}, None, True, 0),
+    ("14B-shaped K4V2 channel-wise keys, T=16384", "14b", {}, None, False, 0),
+    ("14B-shaped K4V2 channel-wise keys, T=16383 (127-token tail)", "14b", {}, 16383, False, 0),
+    ("14B-shaped K8V2 channel-wise keys, T=16384", "14b", {"kb": 8}, None, False, 0),
+    ("14B-shaped K8V2 channel-wise keys, T=16383 (127-token tail)", "14b", {"kb": 8}, 16383, False, 0),
+    ("70B-shaped K4V2, 80 layers resident", "70b", {}, None, False, 0),
+)
+
+
+def main_gpu(args):
+    rank, local_rank, world = dist_env()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2502_15075_b200 import build
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2502_15075_b200 import kvq
+
+    if not args.sweep:
+        line = run_workload(kvq, workload_from_env(), dev, rank, world, args.steps, args.warmup)
+        if rank == 0:
+            print(json.dumps(line))
+        return
+    only = os.environ.get("KVQ_BENCH_SWEEP_ONLY")
+    for label, key, over, tokens, ragged, app in SWEEP:
+        if only and only not in label:
+            continue
+        w = WORKLOADS[key].with_(**over)
+        if "KVQ_BENCH_LAYERS" in os.environ:
+            w = w.with_(layers=min(w.layers, int(os.environ["KVQ_BENCH_LAYERS"])))
+        line = run_workload(kvq, w, dev, rank, world, args.steps, args.warmup, tokens=tokens, ragged=ragged,
+                            append_tokens=app, oracle_budget_s=4.0, do_e2e=False)
+        if rank == 0:
+            line["sweep"] = label
+            print(json.dumps(line), flush=True)
+        torch.cuda.empty_cache()
+
+
+def selftest_ranks(args):
+    """Rank plumbing only (gloo, CPU): rendezvous, barrier, max-over-ranks and the whole-job aggregate."""
+    import torch.distributed as dist
+    rank, _, world = dist_env()
+    if world > 1:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms = max_over_ranks(10.0 + rank, world, torch.device("cpu"))
+    if rank == 0:
+        print(json.dumps({"selftest": True, "n_gpus": world, "ms_per_step": ms,
+                          "value": whole_job_gbs(1e9, ms, world)}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 if __name__ == "__main__":
@@ -381,8 +540,14 @@ if __name__ == "__main__":
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="kvq", choices=["kvq", "reference"])
+    ap.add_argument("--sweep", action="store_true", help="run every model-shaped variant, one line each")
+    ap.add_argument("--selftest-ranks", action="store_true", help=argparse.SUPPRESS)
     a = ap.parse_args()
-    if a.impl == "reference":
+    if a.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        respawn_under_launcher(a.gpus)
+    if a.selftest_ranks:
+        selftest_ranks(a)
+    elif a.impl == "reference":
         run_reference(a)
     else:
         main_gpu(a)

@@ -34,8 +34,9 @@ struct SmemLayout {
   int page_stride, ring_bytes, bar_off, pref_off, misc_off, master_off, ml_off, chan_off, total;
 };
 // master: per consumer warp, 4 NH heads x (D + 8) floats (the row padding keeps a warp's accesses conflict-free).
-// chan: channel-wise keys need two buffers of per-page q operands (NH x D/16 x 32 words), the partial zero-point
-// sums (2 x 8 heads x 8 floats), the page's fixed-point scale per head (2 x 8) and the stream's q in fp32 (8 x D).
+// chan: channel-wise keys need, per group of four warps, two buffers of per-page q operands (NH x D/16 x 32 words),
+// the partial zero-point sums (2 x 8 heads x 8 floats) and the page's fixed-point scale per head (2 x 8), and once
+// the stream's q in fp32 (8 x D).
 __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, int nw, int batch, int D, int nh,
                                                   bool chan) {
   SmemLayout s;
@@ -47,7 +48,8 @@ __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, in
   s.master_off = s.misc_off + 64;
   s.ml_off = s.master_off + nw * 4 * nh * (D + 8) * 4;
   s.chan_off = s.ml_off + nw * 4 * nh * 2 * 4;
-  s.total = s.chan_off + (chan ? (2 * nh * (D / 16) * 32 * 4 + 2 * 64 * 4 + 2 * 8 * 4 + 8 * D * 4) : 0);
+  const int ng = nw / 4;
+  s.total = s.chan_off + (chan ? (2 * ng * nh * (D / 16) * 32 * 4 + 2 * ng * 64 * 4 + 2 * ng * 8 * 4 + 8 * D * 4) : 0);
   return s;
 }
 
@@ -81,6 +83,24 @@ __device__ __forceinline__ uint32_t fixed_point_limb(const float (&t)[4], float 
   return w;
 }
 
+// Split partials of a stream are merged by whichever CTA publishes the last of them: after storing its partial a
+// CTA counts itself in the stream's word, which holds (launch id << 24 | count).  A word that carries another id
+// (stale contents, an earlier launch) restarts at 1, so the workspace needs no initialisation; the CTA that
+// reaches the expected count merges and clears the word, so that a replayed launch with the same id starts clean.
+__device__ __forceinline__ unsigned tagged_count(unsigned long long* p, unsigned long long id40) {
+  unsigned long long old = *reinterpret_cast<volatile unsigned long long*>(p);
+  while (true) {
+    const unsigned long long nw = ((old >> 24) == id40) ? old + 1ull : ((id40 << 24) | 1ull);
+    const unsigned long long r = atomicCAS(p, old, nw);
+    if (r == old) return (unsigned)(nw & 0xFFFFFFull);
+    old = r;
+  }
+}
+// Offset (in floats) of the count words behind the partials: [streams] 64-bit words.
+__host__ __device__ inline size_t tag_offset_floats(int streams, int s_cap, int G, int D) {
+  return ((size_t)streams * s_cap * G * (D + 2) + 3) & ~(size_t)3;
+}
+
 constexpr float kQFix = 32512.0f;          // largest |Q| of the 16-bit fixed-point q (hi limb stays within +-127)
 // The softmax weights enter PV as fixed point P = rint(p * s_V * 2^PBITS / s_lim), p = 2^(logit - reference) with the
 // reference kHeadroom bits above the largest logit seen so far, so that a larger logit rarely forces a rescale.
@@ -102,7 +122,7 @@ constexpr int kFlushBlocks = 512;          // fold the int32 value accumulators 
 template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NH, int NW, int MINB>
 __global__ void __launch_bounds__((NW + 1) * 32, MINB)
 decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1, float* __restrict__ ws,
-                  int s_cap, int stages) {
+                  int s_cap, int stages, void* __restrict__ out, int out_dtype, unsigned long long call_id) {
   constexpr int NR = D / 16;                // 16-channel register slots per key row
   constexpr int KS32 = D / 32;              // k-steps of an 8-bit MMA over the channels
   constexpr int MT = D / 16;                // m-tiles of PV (16 channels each)
@@ -114,9 +134,14 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   constexpr int MSTRIDE = D + 8;
   constexpr int K_ROW_BYTES = D * KB / 8;
   constexpr int V_BLOCK_BYTES = 4 * D * VB;
+  // page geometry (the same numbers the host put into Geom)
+  constexpr int K_META_OFF = kPageTokens * K_ROW_BYTES;
+  constexpr int V_CODES_OFF = K_META_OFF + (KAXIS == 1 ? 4 * D : kPageTokens * NGK * 4);
+  constexpr int V_META_OFF = V_CODES_OFF + 4 * V_BLOCK_BYTES;
   constexpr int NCONS = NW * 32;
+  constexpr int NG = NW / 4;                // groups of four consumer warps; a group takes every NG-th page
   constexpr uint32_t FULL = 0xffffffffu;
-  static_assert(NW == 4, "one consumer warp per 32-token block of a page");
+  static_assert(NW % 4 == 0, "four consumer warps per page, one per 32-token block");
   static_assert(KAXIS == 0 || KB != 2, "channel-wise 2-bit keys are not instantiated");
   static_assert(MT % FPBV == 0, "value m-tiles come in groups that share a byte");
 
@@ -157,13 +182,24 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   if (tid_ == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(smem_u32(&bars[s]), 1);
-      mbar_init(smem_u32(&bars[stages + s]), NW);
+      mbar_init(smem_u32(&bars[stages + s]), 4);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // an empty sequence has no page and therefore no CTA of its own: its output rows are zero
+  for (int bb = blockIdx.x; bb < B; bb += gridDim.x) {
+    if (sPref[bb + 1] == sPref[bb]) {
+      for (int i = tid_; i < g.Hq * D; i += blockDim.x) {
+        const size_t oi = (size_t)bb * g.Hq * D + i;
+        if (out_dtype == KVQ_FP32) static_cast<float*>(out)[oi] = 0.f;
+        else static_cast<uint16_t*>(out)[oi] = 0;
+      }
+    }
+  }
   const FlatPlan plan = make_plan(sPref[B], sMisc[0], gridDim.x, s_cap);
   if (plan.N == 0 || (int)blockIdx.x >= plan.c_eff) return;
+  unsigned long long* counts = reinterpret_cast<unsigned long long*>(ws + tag_offset_floats(B * Hkv, s_cap, G, D));
   const long long x_lo = plan.lo(blockIdx.x), x_hi = plan.lo(blockIdx.x + 1);
 
   // ---- cursor: first page of this CTA -> (b, h, page)
@@ -182,6 +218,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   const uint32_t ring = smem_u32(smem);
   const uint32_t bar0 = smem_u32(bars);
   volatile int* abort_flag = sMisc + 1;
+  volatile int* n_published = sMisc + 2;      // count returned for the partial just published
+  const unsigned long long id40 = (call_id & 0xFFFFFFFFFFull) ? (call_id & 0xFFFFFFFFFFull) : 1ull;
 
   // =========================================================== producer warp
   if (warp == NW) {
@@ -232,29 +270,30 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   int Oi[NTV][MT][4];          // PV accumulators: NH = 1: n-tiles (limb 3, 2 | limb 1, 0) of head tid; NH = 2: (head tid:
                                // limb 2, 1 | head tid + 4: limb 2, 1 | limb 0 of both)
   constexpr float PONE = (float)(1u << (kPBits<NH> - 1)) * 2.0f;     // 2^PBITS
-  float s_lim = 9.094947e-13f; // 2^-40: power of two above every value scale folded into the weights so far
-  float sscale = PONE / 9.094947e-13f, inv_sscale = 9.094947e-13f / PONE;
-  int since_flush = 0;
-  uint32_t* sB = reinterpret_cast<uint32_t*>(smem + sl.chan_off);                                  // [2][NH][NR][32]
-  float* sZ = reinterpret_cast<float*>(smem + sl.chan_off + 2 * NH * NR * 32 * 4);                 // [2][8 heads][8]
-  float* sHS = sZ + 2 * 64;                                                                        // [2][8 heads]
-  float* sQ = sHS + 2 * 8;                                                                         // [8 heads][D]
+  // sscale = 2^PBITS / s_lim, s_lim a power of two above every value scale folded into the weights so far (2^-40 at first)
+  float sscale = PONE / 9.094947e-13f;
+  uint32_t* sB = reinterpret_cast<uint32_t*>(smem + sl.chan_off);                                  // [2 NG][NH][NR][32]
+  float* sZ = reinterpret_cast<float*>(smem + sl.chan_off + 2 * NG * NH * NR * 32 * 4);            // [2 NG][8 heads][8]
+  float* sHS = sZ + 2 * NG * 64;                                                                   // [2 NG][8 heads]
+  float* sQ = sHS + 2 * NG * 8;                                                                         // [8 heads][D]
   float* myM = sMaster + warp * NHEADS * MSTRIDE;
+  const int grp = warp >> 2, wq = warp & 3;       // page group of this warp, and its 32-token block inside a page
   int page_no = 0;
-  int stage = 0;
+  int stage = grp;             // ring slot and parity of this group's next page (pages go to the groups in turn)
   uint32_t phase = 0;
+  int turn = 0;                // CTA-wide page counter modulo NG
   bool aborted = false;
   constexpr int KCB = (KW < 4 ? KW : 4) * 4;     // bytes of a lane chunk's first quad of key words
-  const int lane_k = (warp * 32 + gid) * K_ROW_BYTES + tid * KCB;
-  const int lane_km = g.k_meta_off + (warp * 32 + gid) * 4 * NGK;
-  const int lane_v = g.v_codes_off + warp * V_BLOCK_BYTES + lane * 16;
-  const int lane_vm = g.v_meta_off + (warp * 32 + gid) * 4 * NGV;
+  const int lane_k = (wq * 32 + gid) * K_ROW_BYTES + tid * KCB;
+  const int lane_km = K_META_OFF + (wq * 32 + gid) * 4 * NGK;
+  const int lane_v = V_CODES_OFF + wq * V_BLOCK_BYTES + lane * 16;
+  const int lane_vm = V_META_OFF + (wq * 32 + gid) * 4 * NGV;
 
   // Fold the int32 accumulators into the warp's fp32 master (each (head, channel) belongs to one lane) and clear them.
   auto flush_acc = [&]() {
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-      const float fw = inv_sscale / (float)(1 << (VB * (mt % FPBV)));
+      const float fw = (1.0f / sscale) / (float)(1 << (VB * (mt % FPBV)));      // sscale is a power of two
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
         const int d = 16 * mt + 8 * r + gid;
@@ -275,7 +314,6 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
       for (int nt = 0; nt < NTV; ++nt) { Oi[nt][mt][0] = Oi[nt][mt][1] = Oi[nt][mt][2] = Oi[nt][mt][3] = 0; }
     }
-    since_flush = 0;
   };
 
   for (long long x = x_lo; x < x_hi;) {
@@ -285,7 +323,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
     // ---- segment start: q operands, group sums and a clean state for this stream's heads
     {
-      if constexpr (KAXIS == 1) named_bar_sync(2, NCONS);            // nobody still reads the previous stream's q
+      if constexpr (KAXIS == 1) named_bar_sync(1, NCONS);            // nobody still reads the previous stream's q
 #pragma unroll
       for (int nh = 0; nh < NH; ++nh) {
         const int hb = (gid >> 1) + 4 * nh;                          // head of this lane's operand column
@@ -382,7 +420,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
         for (int j = 0; j < NGV; ++j) zacc[nh][j] = 0.f;
       }
-      if constexpr (KAXIS == 1) named_bar_sync(2, NCONS);
+      if constexpr (KAXIS == 1) named_bar_sync(1, NCONS);
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
@@ -393,10 +431,12 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           myM[(tid + 4 * nh) * MSTRIDE + 16 * mt + 8 + gid] = 0.f;
         }
       }
-      since_flush = 0;
     }
 
     for (int pp = 0; pp < seg_pages; ++pp) {
+      const bool mine = turn == grp;
+      if (++turn == NG) turn = 0;
+      if (!mine) continue;
       const int nv = min(kPageTokens, n_tok - (page + pp) * kPageTokens);
       const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
       if (!aborted) {
@@ -413,10 +453,10 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       // (scale from max|q| of the head times the page's largest channel scale).  Each warp makes the operands of
       // its own slots, all warps exchange them through shared memory; sum_d q_d z_d is summed in fp32 the same way.
       if constexpr (KAXIS == 1) {
-        constexpr int OWN = NR / NW > 0 ? NR / NW : 1;
-        const int buf = page_no & 1;
+        constexpr int OWN = NR / 4 > 0 ? NR / 4 : 1;
+        const int buf = 2 * grp + (page_no & 1);
         if (!aborted && !tail_k) {
-          const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + g.k_meta_off);
+          const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + K_META_OFF);
           float smax = 0.f;
           if (4 * lane < D) {
             const uint4 mm = *reinterpret_cast<const uint4*>(km + 4 * lane);
@@ -429,11 +469,11 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             const int hb = (gid >> 1) + 4 * nh;
             const float am = amaxB[nh] * smax;
             const float scale = am > 0.f ? kQFix / am : 0.f;
-            if (warp == 0 && tid == 0 && (gid & 1) == 0) sHS[buf * 8 + hb] = am > 0.f ? c1 / scale : 0.f;
+            if (wq == 0 && tid == 0 && (gid & 1) == 0) sHS[buf * 8 + hb] = am > 0.f ? c1 / scale : 0.f;
             float zsum = 0.f;
 #pragma unroll
             for (int i = 0; i < OWN; ++i) {
-              const int r = warp * OWN + i;
+              const int r = wq * OWN + i;
               if (r < NR) {
                 const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);   // (s, z) of 4 channels
                 const float4 qq = *reinterpret_cast<const float4*>(sQ + hb * D + 16 * r + 4 * tid);
@@ -452,13 +492,13 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             }
             zsum += __shfl_xor_sync(FULL, zsum, 1);
             zsum += __shfl_xor_sync(FULL, zsum, 2);
-            if (tid == 0 && (gid & 1) == 0 && warp * OWN < NR) sZ[(buf * 8 + hb) * 8 + warp] = zsum;
+            if (tid == 0 && (gid & 1) == 0 && wq * OWN < NR) sZ[(buf * 8 + hb) * 8 + wq] = zsum;
           }
         }
         // every warp takes part in the exchange barrier of a full page, also after a timeout
-        if (!tail_k) named_bar_sync(2, NCONS);
+        if (!tail_k) named_bar_sync(2 + grp, 128);
         if (!aborted && !tail_k) {
-          constexpr int NWR = (NR / OWN < NW) ? NR / OWN : NW;      // warps that contributed
+          constexpr int NWR = (NR / OWN < 4) ? NR / OWN : 4;        // warps that contributed
 #pragma unroll
           for (int nh = 0; nh < NH; ++nh) {
 #pragma unroll
@@ -472,7 +512,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         }
       }
 
-      if (!aborted && warp * 32 < nv) {
+      if (!aborted && wq * 32 < nv) {
         const uint8_t* sp_k = sp + lane_k;
         const uint8_t* sp_km = sp + lane_km;
         const uint8_t* sp_v = sp + lane_v;
@@ -485,7 +525,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           // ------------------------------------------------------------ logits of the block's two 16-token tiles
 #pragma unroll
           for (int u = 0; u < 2; ++u) {
-            const int tok0 = warp * 32 + 16 * u + gid;        // page-local tokens of this lane's two rows: tok0, tok0 + 8
+            const int tok0 = wq * 32 + 16 * u + gid;        // page-local tokens of this lane's two rows: tok0, tok0 + 8
             vld[u][0] = !MASKED || tok0 < nv;
             vld[u][1] = !MASKED || tok0 + 8 < nv;
             if (KAXIS == 1 && tail_k) {
@@ -586,7 +626,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
           // ------------------------------------------------------------ softmax reference / scale check (rarely taken)
           float bmax[NH];
-          bool trig = (smax >= s_lim) | (since_flush >= kFlushBlocks);
+          // (the int32 accumulators are also folded every kFlushBlocks pages, long before they can overflow)
+          bool trig = (smax * sscale >= PONE) | ((page_no & (kFlushBlocks - 1)) == kFlushBlocks - 1);
 #pragma unroll
           for (int nh = 0; nh < NH; ++nh) {
             bmax[nh] = fmaxf(fmaxf(L[0][0][nh], L[0][1][nh]), fmaxf(L[1][0][nh], L[1][1][nh]));
@@ -596,11 +637,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             flush_acc();                                   // with the scale the accumulated weights were made with
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) smax = fmaxf(smax, __shfl_xor_sync(FULL, smax, off));
-            if (smax >= s_lim) {
+            if (smax * sscale >= PONE) {
               // next power of two above the largest value scale: p * s * sscale < 2^PBITS for every p <= 1
-              s_lim = __uint_as_float((__float_as_uint(smax) & 0x7F800000u) + 0x00800000u);
-              sscale = PONE / s_lim;
-              inv_sscale = s_lim / PONE;
+              sscale = PONE / __uint_as_float((__float_as_uint(smax) & 0x7F800000u) + 0x00800000u);
             }
 #pragma unroll
             for (int nh = 0; nh < NH; ++nh) {
@@ -622,7 +661,6 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               }
             }
           }
-          ++since_flush;
 
           // ------------------------------------------------------------ weights: p = 2^(logit - reference) <= 2^-headroom,
           // P = rint(p * s_V * sscale) < 2^PBITS
@@ -680,12 +718,13 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           }
         };
 
-        if (nv - warp * 32 >= 32) do_block(std::false_type{});
+        if (nv - wq * 32 >= 32) do_block(std::false_type{});
         else do_block(std::true_type{});
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(bar0 + 8 * (stages + stage));
-      if (++stage == stages) { stage = 0; phase ^= 1; }
+      stage += NG;
+      if (stage >= stages) { stage -= stages; phase ^= 1; }
       ++page_no;
     }
 
@@ -712,8 +751,13 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         }
       }
       named_bar_sync(1, NCONS);
+      // The flat split gives a stream to a run of consecutive CTAs, one partial slot each.  A CTA that holds the
+      // whole stream writes the output at once; otherwise it stores its partial, counts itself in, and the CTA
+      // that completes the count merges all partials of the stream by log-sum-exp and stores the output.
       const long long xs = (long long)sPref[b] + (long long)h * pages_b;     // first page of this stream
-      const int slot = (int)blockIdx.x - plan.cta_of(xs);
+      const int c_first = plan.cta_of(xs);
+      const int slot = (int)blockIdx.x - c_first;
+      const int n_part = plan.cta_of(xs + pages_b - 1) - c_first + 1;        // partials of this stream
       if (slot >= 0 && slot < s_cap) {
         for (int idx = tid_; idx < G * D; idx += NCONS) {
           const int head = idx / D, d = idx % D;
@@ -728,9 +772,61 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             o = fmaf(f, sMaster[(w * NHEADS + head) * MSTRIDE + d], o);
             lsum = fmaf(f, sML[(w * NHEADS + head) * 2 + 1], lsum);
           }
-          float* dst = ws + (((size_t)stream * s_cap + slot) * G + head) * (D + 2);
-          if (d == 0) { dst[0] = mstar; dst[1] = lsum; }
-          dst[2 + d] = o;
+          if (n_part == 1) {
+            const float r = lsum > 0.f ? o / lsum : 0.f;
+            const size_t oi = ((size_t)b * g.Hq + (size_t)h * G + head) * D + d;
+            if (out_dtype == KVQ_FP32) static_cast<float*>(out)[oi] = r;
+            else static_cast<uint16_t*>(out)[oi] = f32_to_bits16(r, out_dtype);
+          } else {
+            float* dst = ws + (((size_t)stream * s_cap + slot) * G + head) * (D + 2);
+            if (d == 0) { dst[0] = mstar; dst[1] = lsum; }
+            dst[2 + d] = o;
+          }
+        }
+        if (n_part > 1) {
+          __threadfence();
+          named_bar_sync(1, NCONS);
+          if (tid_ == 0) *n_published = (int)tagged_count(counts + stream, id40);
+          named_bar_sync(1, NCONS);
+          if (*n_published == n_part) {
+            __threadfence();
+            for (int idx = tid_; idx < G * D; idx += NCONS) {
+              const int head = idx / D, d = idx % D;
+              const float* base = ws + (((size_t)stream * s_cap) * G + head) * (D + 2);
+              const size_t slot_stride = (size_t)G * (D + 2);
+              float mstar = -INFINITY, num = 0.f, den = 0.f;
+              for (int j0 = 0; j0 < n_part; j0 += 4) {
+                float mj[4], lj[4], oj[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {                   // issue the loads of a batch before using any
+                  const bool on = j0 + u < n_part;
+                  const float* pj = base + (size_t)(on ? j0 + u : 0) * slot_stride;
+                  mj[u] = on ? __ldcg(pj) : -INFINITY;
+                  lj[u] = on ? __ldcg(pj + 1) : 0.f;
+                  oj[u] = on ? __ldcg(pj + 2 + d) : 0.f;
+                }
+                float mb = mstar;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) mb = fmaxf(mb, mj[u]);
+                if (mb == -INFINITY) continue;
+                const float keep = (mstar == -INFINITY) ? 0.f : ex2(mstar - mb);
+                num *= keep;
+                den *= keep;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                  const float wgt = (mj[u] == -INFINITY) ? 0.f : ex2(mj[u] - mb);
+                  num = fmaf(wgt, oj[u], num);
+                  den = fmaf(wgt, lj[u], den);
+                }
+                mstar = mb;
+              }
+              const float r = den > 0.f ? num / den : 0.f;
+              const size_t oi = ((size_t)b * g.Hq + (size_t)h * G + head) * D + d;
+              if (out_dtype == KVQ_FP32) static_cast<float*>(out)[oi] = r;
+              else static_cast<uint16_t*>(out)[oi] = f32_to_bits16(r, out_dtype);
+            }
+            if (tid_ == 0) counts[stream] = 0ull;
+          }
         }
       }
       named_bar_sync(1, NCONS);
@@ -753,17 +849,17 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 // Launches one instantiation; defined per instantiation unit.
 template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NH, int NW, int MINB>
 int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap,
-                    cudaStream_t stream) {
+                    void* out, int out_dtype, unsigned long long call_id, cudaStream_t stream) {
   const int budget = (227 * 1024) / MINB - 1024;            // shared memory per CTA for MINB resident CTAs per SM
   int stages = (budget - smem_layout(0, 0, NW, g.B, D, NH, KAXIS == 1).total) / ((g.page_bytes + 127) & ~127);
-  if (stages > 8) stages = 8;
-  if (stages < 2) return KVQ_ERR_UNSUPPORTED;
+  if (stages > 16) stages = 16;
+  if (stages < 2 || stages < NW / 4) return KVQ_ERR_UNSUPPORTED;
   const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, g.B, D, NH, KAXIS == 1);
   auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
     return KVQ_ERR_CUDA_LAUNCH;
   kern<<<148 * MINB, (NW + 1) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap,
-                                                         stages);
+                                                         stages, out, out_dtype, call_id);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
 

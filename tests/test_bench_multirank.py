@@ -42,3 +42,18 @@ def test_single_rank_is_identity():
     import bench
     assert bench.max_over_ranks(7.5, 1, torch.device("cpu")) == 7.5
     assert bench.whole_job_gbs(1e9, 1.0, 1) == 1000.0
+
+
+def test_gpus_flag_starts_its_own_ranks():
+    """`bench.py --gpus 2` without a launcher re-executes itself under the launcher with two ranks (here: the
+    CPU-only rank plumbing, gloo): rank 0 prints one line for a two-rank job with the slowest rank's time."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-ranks"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 11.0
+    assert abs(lines[0]["value"] - 2 * 1e9 / 11e-3 / 1e9) < 1e-9
