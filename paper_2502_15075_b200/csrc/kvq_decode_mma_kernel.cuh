@@ -34,7 +34,7 @@ struct SmemLayout {
   int page_stride, ring_bytes, bar_off, pref_off, misc_off, master_off, ml_off, chan_off, total;
 };
 // master: per consumer warp, 4 NH heads x (D + 8) floats (the row padding keeps a warp's accesses conflict-free).
-// chan: channel-wise keys need, per group of four warps, two buffers of per-page q operands (NH x D/16 x 32 words),
+// chan: channel-wise keys need, per group of four warps, two buffers of per-page q operands (NH x 2 x D/16 x 32 words),
 // the partial zero-point sums (2 x 8 heads x 8 floats) and the page's fixed-point scale per head (2 x 8), and once
 // the stream's q in fp32 (8 x D).
 __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, int nw, int batch, int D, int nh,
@@ -49,7 +49,7 @@ __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, in
   s.ml_off = s.master_off + nw * 4 * nh * (D + 8) * 4;
   s.chan_off = s.ml_off + nw * 4 * nh * 2 * 4;
   const int ng = nw / 4;
-  s.total = s.chan_off + (chan ? (2 * ng * nh * (D / 16) * 32 * 4 + 2 * ng * 64 * 4 + 2 * ng * 8 * 4 + 8 * D * 4) : 0);
+  s.total = s.chan_off + (chan ? (2 * ng * nh * 2 * (D / 16) * 32 * 4 + 2 * ng * 64 * 4 + 2 * ng * 8 * 4 + 8 * D * 4) : 0);
   return s;
 }
 
@@ -102,6 +102,24 @@ __host__ __device__ inline size_t tag_offset_floats(int streams, int s_cap, int 
 }
 
 constexpr float kQFix = 32512.0f;          // largest |Q| of the 16-bit fixed-point q (hi limb stays within +-127)
+constexpr float kQFix3 = 8300000.0f;       // ... of the 24-bit fixed-point q * s of channel-wise keys (three limbs)
+
+// Limb `which` (0 = lowest) of the balanced three-byte split Q = (l2 * 256 + l1) * 256 + l0 of four values times
+// `scale`, |Q| <= kQFix3, as one word of four signed bytes; which < 0 gives zero.
+__device__ __forceinline__ uint32_t fixed_point_limb3(const float (&t)[4], float scale, int which) {
+  uint32_t w = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int Q = __float2int_rn(t[j] * scale);
+    const int l0 = (int)(int8_t)(Q & 0xFF);
+    const int Q1 = (Q - l0) >> 8;
+    const int l1 = (int)(int8_t)(Q1 & 0xFF);
+    const int l2 = (Q1 - l1) >> 8;
+    const int v = which == 0 ? l0 : (which == 1 ? l1 : (which == 2 ? l2 : 0));
+    w |= (uint32_t)(v & 0xFF) << (8 * j);
+  }
+  return w;
+}
 // The softmax weights enter PV as fixed point P = rint(p * s_V * 2^PBITS / s_lim), p = 2^(logit - reference) with the
 // reference kHeadroom bits above the largest logit seen so far, so that a larger logit rarely forces a rescale.
 // Tokens whose P falls below one unit vanish, so the width matters over long contexts: four byte limbs (31 bits)
@@ -130,6 +148,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   constexpr int FPBV = 8 / VB;              // value codes per byte (channels 16 apart)
   constexpr int VQ = MT / FPBV;             // quads of value words per lane per 32-token block
   constexpr int NTV = NH == 1 ? 2 : 3;      // n-tiles of PV: (head, limb) columns
+  constexpr int NTK = KAXIS == 1 ? 2 : 1;   // n-tiles of QK^T per head set: two byte limbs of q, or three of q * s
   constexpr int NHEADS = 4 * NH;
   constexpr int MSTRIDE = D + 8;
   constexpr int K_ROW_BYTES = D * KB / 8;
@@ -261,7 +280,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   }
 
   // =========================================================== consumer warps
-  uint32_t qB[NH][NR];         // QK^T B operands: column gid = (head gid/2 + 4 nh, limb gid%2), channels 16 r + 4 tid + {0..3}
+  uint32_t qB[NH][NTK][NR];    // QK^T B operands: column gid = (head gid/2 + 4 nh, limb gid%2), channels 16 r + 4 tid + {0..3};
+                               // channel-wise keys: n-tile 0 carries limbs (2, 1), n-tile 1 limbs (0, none)
   float hs[NH];                // c1 / fixed-point scale of q, own heads (tid + 4 nh)
   float qsum[NH][NGK];         // c1 * sum of q over each key group, own heads
   float zq[NH];                // channel-wise keys: c1 * sum_d q_d z_d of the current page, own heads
@@ -272,8 +292,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   constexpr float PONE = (float)(1u << (kPBits<NH> - 1)) * 2.0f;     // 2^PBITS
   // sscale = 2^PBITS / s_lim, s_lim a power of two above every value scale folded into the weights so far (2^-40 at first)
   float sscale = PONE / 9.094947e-13f;
-  uint32_t* sB = reinterpret_cast<uint32_t*>(smem + sl.chan_off);                                  // [2 NG][NH][NR][32]
-  float* sZ = reinterpret_cast<float*>(smem + sl.chan_off + 2 * NG * NH * NR * 32 * 4);            // [2 NG][8 heads][8]
+  uint32_t* sB = reinterpret_cast<uint32_t*>(smem + sl.chan_off);                                  // [2 NG][NH][2][NR][32]
+  float* sZ = reinterpret_cast<float*>(smem + sl.chan_off + 2 * NG * NH * 2 * NR * 32 * 4);        // [2 NG][8 heads][8]
   float* sHS = sZ + 2 * NG * 64;                                                                   // [2 NG][8 heads]
   float* sQ = sHS + 2 * NG * 8;                                                                         // [8 heads][D]
   float* myM = sMaster + warp * NHEADS * MSTRIDE;
@@ -402,7 +422,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
           for (int j = 0; j < NGK; ++j) qs[j] = 0;
 #pragma unroll
-          for (int r = 0; r < NR; ++r) qB[nh][r] = fixed_point_limb(qv[r], scale, gid & 1, qs[r / (NR / NGK)]);
+          for (int r = 0; r < NR; ++r) qB[nh][0][r] = fixed_point_limb(qv[r], scale, gid & 1, qs[r / (NR / NGK)]);
           hs[nh] = __shfl_sync(FULL, hsb, 8 * tid);
           // the zero-point term uses the sum of the same fixed-point q the MMAs see: the two large terms
           // s (q . c) and z sum(q) of a logit then cancel exactly as they do for the exact q
@@ -468,7 +488,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           for (int nh = 0; nh < NH; ++nh) {
             const int hb = (gid >> 1) + 4 * nh;
             const float am = amaxB[nh] * smax;
-            const float scale = am > 0.f ? kQFix / am : 0.f;
+            const float scale = am > 0.f ? kQFix3 / am : 0.f;
             if (wq == 0 && tid == 0 && (gid & 1) == 0) sHS[buf * 8 + hb] = am > 0.f ? c1 / scale : 0.f;
             float zsum = 0.f;
 #pragma unroll
@@ -486,8 +506,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
                   t[j] = qa[j] * sz.x;
                   zsum = fmaf(qa[j], sz.y, zsum);
                 }
-                int unused = 0;
-                sB[((buf * NH + nh) * NR + r) * 32 + lane] = fixed_point_limb(t, scale, gid & 1, unused);
+                sB[(((buf * NH + nh) * 2 + 0) * NR + r) * 32 + lane] = fixed_point_limb3(t, scale, (gid & 1) ? 1 : 2);
+                sB[(((buf * NH + nh) * 2 + 1) * NR + r) * 32 + lane] = fixed_point_limb3(t, scale, (gid & 1) ? -1 : 0);
               }
             }
             zsum += __shfl_xor_sync(FULL, zsum, 1);
@@ -502,7 +522,10 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
           for (int nh = 0; nh < NH; ++nh) {
 #pragma unroll
-            for (int r = 0; r < NR; ++r) qB[nh][r] = sB[((buf * NH + nh) * NR + r) * 32 + lane];
+            for (int nt = 0; nt < NTK; ++nt) {
+#pragma unroll
+              for (int r = 0; r < NR; ++r) qB[nh][nt][r] = sB[(((buf * NH + nh) * 2 + nt) * NR + r) * 32 + lane];
+            }
             float z = 0.f;
 #pragma unroll
             for (int w = 0; w < NWR; ++w) z += sZ[(buf * 8 + tid + 4 * nh) * 8 + w];
@@ -558,11 +581,14 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               const uint8_t* krow = sp_k + u * (16 * K_ROW_BYTES);           // this lane's chunk of row tok0
               load_words<KW>(krow, 64, ka);
               load_words<KW>(krow + 8 * K_ROW_BYTES, 64, kb2);
-              int S[NGK][NH][4];
+              int S[NGK][NH][NTK][4];
 #pragma unroll
               for (int j = 0; j < NGK; ++j) {
 #pragma unroll
-                for (int nh = 0; nh < NH; ++nh) { S[j][nh][0] = S[j][nh][1] = S[j][nh][2] = S[j][nh][3] = 0; }
+                for (int nh = 0; nh < NH; ++nh) {
+#pragma unroll
+                  for (int nt = 0; nt < NTK; ++nt) { S[j][nh][nt][0] = S[j][nh][nt][1] = S[j][nh][nt][2] = S[j][nh][nt][3] = 0; }
+                }
               }
 #pragma unroll
               for (int s = 0; s < KS32; ++s) {
@@ -570,15 +596,21 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
                 const uint32_t a0 = key_slot<KB, KW>(ka, 2 * s), a1 = key_slot<KB, KW>(kb2, 2 * s);
                 const uint32_t a2 = key_slot<KB, KW>(ka, 2 * s + 1), a3 = key_slot<KB, KW>(kb2, 2 * s + 1);
 #pragma unroll
-                for (int nh = 0; nh < NH; ++nh)
-                  mma16832_u8s8(S[j][nh], a0, a1, a2, a3, qB[nh][2 * s], qB[nh][2 * s + 1]);
+                for (int nh = 0; nh < NH; ++nh) {
+#pragma unroll
+                  for (int nt = 0; nt < NTK; ++nt)
+                    mma16832_u8s8(S[j][nh][nt], a0, a1, a2, a3, qB[nh][nt][2 * s], qB[nh][nt][2 * s + 1]);
+                }
               }
               // accumulator columns 2 tid, 2 tid + 1 = (hi, lo) limbs of head tid + 4 nh: sum_d code_d Q_d = 256 hi + lo
+              // (channel-wise keys: limbs (2, 1) in n-tile 0 and limb 0 in n-tile 1, combined in fp32)
               if constexpr (KAXIS == 1) {
 #pragma unroll
                 for (int nh = 0; nh < NH; ++nh) {
-                  L[u][0][nh] = fmaf((float)(S[0][nh][0] * 256 + S[0][nh][1]), hs[nh], zq[nh]);
-                  L[u][1][nh] = fmaf((float)(S[0][nh][2] * 256 + S[0][nh][3]), hs[nh], zq[nh]);
+                  const float t0 = fmaf((float)S[0][nh][0][0], 65536.f, (float)(S[0][nh][0][1] * 256 + S[0][nh][NTK - 1][0]));
+                  const float t1 = fmaf((float)S[0][nh][0][2], 65536.f, (float)(S[0][nh][0][3] * 256 + S[0][nh][NTK - 1][2]));
+                  L[u][0][nh] = fmaf(t0, hs[nh], zq[nh]);
+                  L[u][1][nh] = fmaf(t1, hs[nh], zq[nh]);
                 }
               } else {
                 const uint32_t* km = reinterpret_cast<const uint32_t*>(sp_km + u * (16 * 4 * NGK));   // row tok0
@@ -590,8 +622,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
                   const float2 mb = __half22float2(as_h2(km[8 * NGK + j]));             // ... of row tok0 + 8
 #pragma unroll
                   for (int nh = 0; nh < NH; ++nh) {
-                    const float t0 = (float)(S[j][nh][0] * 256 + S[j][nh][1]);
-                    const float t1 = (float)(S[j][nh][2] * 256 + S[j][nh][3]);
+                    const float t0 = (float)(S[j][nh][0][0] * 256 + S[j][nh][0][1]);
+                    const float t1 = (float)(S[j][nh][0][2] * 256 + S[j][nh][0][3]);
                     L[u][0][nh] += fmaf(ma.x * hs[nh], t0, ma.y * qsum[nh][j]);
                     L[u][1][nh] += fmaf(mb.x * hs[nh], t1, mb.y * qsum[nh][j]);
                   }
