@@ -10,16 +10,17 @@
  *
  * What is computed (arxiv 2502.15075, "Quantize What Counts: More for Keys,
  * Less for Values"): keys and values of the cache (K = X W^K, V = X W^V, one
- * L x d_head matrix per head, Sec. 3 / App. B.3) are stored with a uniform scalar
- * quantizer (App. B.1: scale = range / steps, Q = round(A / scale), A^ = scale Q)
- * at independent bit widths b_K, b_V (Theorem 2: more bits for keys), in groups
- * of 32/64/128 elements, token-wise or channel-wise, with recent tokens of an
- * incomplete channel-wise block kept in 16-bit precision (Sec. 4.1).  A decode
- * step computes softmax(q K^T / sqrt(d)) V (App. A.1 notation) over the
+ * L x d_head matrix per head, Sec. 3 / App. B.4) are stored with a uniform scalar
+ * quantizer at independent bit widths b_K, b_V (Theorem 2: more bits for keys),
+ * in groups of 32/64/128 elements, token-wise or channel-wise, with recent tokens
+ * of an incomplete channel-wise block kept in 16-bit precision (Sec. 4.1).  A
+ * decode step computes softmax(q K^T / sqrt(d)) V (App. A.1 notation) over the
  * reconstructed cache.
  *
- * Quantizer (fixed formula; every operation an individually rounded IEEE fp32
- * operation, ties to even):
+ * Quantizer.  App. B.1 defines the symmetric uniform quantizer (alpha = M / (2^(b-1) - 1),
+ * Q = round(A / alpha), A^ = alpha Q); this library applies the same uniform rounding per
+ * group with the group minimum as offset (an asymmetric variant: scale = range / (2^b - 1)).
+ * Fixed formula; every operation an individually rounded IEEE fp32 operation, ties to even:
  *     mn, mx  = min, max of the group, each + 0.0f   (-0 becomes +0)
  *     s16     = fp16_rn((mx - mn) / qmax), z16 = fp16_rn(mn), saturating at +-65504
  *     s, z    = (float)s16, (float)z16,  qmax = 2^b - 1
@@ -27,20 +28,21 @@
  *     x^      = fmaf(code, s, z)
  * Inputs must be finite.
  *
- * Packed page (layout version 1): 128 consecutive tokens of one
+ * Packed page (layout version 2): 128 consecutive tokens of one
  * (batch, kv-head) stream, regions [K codes | K meta | V codes | V meta], each
- * a multiple of 16 bytes, little-endian.  Field f of a 32-bit word holds bits
- * [f*b, f*b+b); ppw = 16/b (V codes).
+ * a multiple of 16 bytes, little-endian.  Field f of a byte or word holds bits [f*b, f*b+b).
  *   K codes, b in {2,4,8}: rows of D*b/8 bytes per token, each holding 4 chunks of
  *     wpc = D*b/128 words; with fpb = 8/b fields per byte, channel d: chunk (d%16)/4,
  *     r = d/16, word r/fpb, bit 8*(d%4) + b*(r%fpb)  (byte j of a word holds channels
  *     16r + 4*chunk + j: one mask per field gives four consecutive channels as four bytes).
- *   V codes, b in {2,4,8}: 8 tiles of 16 tokens, each holding 32 chunks of
- *     wpc = D*b/64 words; with k = 8*(d/64) + d%8 and npos = 8/b, channel d of tile-local
- *     token tau: chunk 4*((d/8)%8) + (tau%8)/2, word k/npos,
- *     field k%npos + npos*(tau/8) + ppw*(tau%2).
- *   (chunk, word) inside a row / tile of nchunks chunks, with qw = min(wpc, 4):
- *     byte = (word/4)*(nchunks*4*qw) + chunk*(4*qw) + (word%4)*4   (quads of words, quad-major).
+ *     (chunk, word) inside a row, with qw = min(wpc, 4):
+ *     byte = (word/4)*(16*qw) + chunk*(4*qw) + (word%4)*4   (quads of words, quad-major).
+ *   V codes, b in {2,4,8}: 4 blocks of 32 tokens, 4*D*b bytes each.  A byte holds the codes of
+ *     one token for the fpb = 8/b channels that lie 16 apart.  With m = d/16, f = m%fpb,
+ *     mw = m/fpb, rh = (d%16)/8, g = d%8 and, for block-local token tau, kh = tau/16,
+ *     u = tau%16, t = (u%8)/2, j = 2*(u%2) + u/8:
+ *     byte = block*(4*D*b) + mw*512 + (4*g + t)*16 + 4*(2*rh + kh) + j,  bit = b*f
+ *     (the bytes of a word are tokens 2t, 2t+8, 2t+1, 2t+9 of one half of the block).
  *   b = 16: rows [token][D] of the input's 16-bit patterns, no meta.
  *   Meta: (scale fp16, zero fp16) per group; per-token axis [128][D/g],
  *     per-channel K [D].
@@ -59,7 +61,7 @@
 extern "C" {
 #endif
 
-#define KVQ_LAYOUT_VERSION 1
+#define KVQ_LAYOUT_VERSION 2   /* changes whenever the bytes of a packed page change */
 #define KVQ_PAGE_TOKENS 128
 
 /* return codes (0 = success) */
@@ -102,7 +104,7 @@ typedef struct {
   int32_t* status;  /* device, one word of KVQ_STATUS_* bits */
   const int8_t* k_signs; /* device [head_dim] of +1 / -1, or NULL.  Not NULL: keys are rotated before
                             quantization by y = H (signs * x) / sqrt(head_dim), H the Sylvester Hadamard matrix
-                            (Sec. 4.3, key-only rotation, which the paper finds sufficient); decode applies the
+                            (Sec. 4.4, key-only rotation, which the paper finds sufficient); decode applies the
                             same rotation to q, dequantize rotates back.  Needs kb != 16.  The transform is
                             computed in fp32 with butterfly stages h = 1, 2, 4, ... in this order, (a, b) ->
                             (a + b, a - b), then one multiplication by (float)(1/sqrt(head_dim)). */
@@ -138,12 +140,13 @@ int kvq_quantize_append(const kvq_config* cfg, const kvq_cache* cache,
  * over t < seq_len[b] (App. A.1: S = Q K^T / sqrt(d), A = softmax(S), A V), streaming the
  * packed pages and reconstructing K^, V^ on the fly; tokens of an incomplete channel-wise
  * key block are read from the fp16 tail.  Split over the sequence, partial results merged by
- * log-sum-exp in a second pass.  seq_len[b] == 0 gives zeros.
+ * log-sum-exp.  seq_len[b] == 0 gives zeros.
  *   q: device, in_dtype, [batch][n_q_heads][head_dim] contiguous.
  *   out: device, [batch][n_q_heads][head_dim] contiguous, out_dtype (KVQ_FP16/BF16/FP32).
  *   softmax_scale <= 0 selects 1/sqrt(head_dim).
  *   workspace: device scratch of at least kvq_workspace_bytes(), 16-byte aligned; contents
- *     need no initialisation and are undefined afterwards.
+ *     need no initialisation and are undefined afterwards.  Calls that may overlap on the GPU
+ *     need separate workspaces.
  * Asynchronous on cuda_stream; reads the cache only.
  */
 int kvq_decode_attention(const kvq_config* cfg, const kvq_cache* cache,

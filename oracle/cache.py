@@ -24,7 +24,7 @@ ERR_CAPACITY_BIT = 1
 class OracleCache:
     def __init__(self, batch, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, dtype, capacity_tokens, k_signs=None):
         """k_signs: None, or +-1 per channel: keys are rotated by the randomized Hadamard transform
-        y = H (signs * x) / sqrt(D) before quantization (Sec. 4.3, key-only rotation); queries get the same
+        y = H (signs * x) / sqrt(D) before quantization (Sec. 4.4, key-only rotation); queries get the same
         rotation at decode time and dequantize rotates back."""
         assert capacity_tokens % PAGE_TOKENS == 0
         assert not (k_axis == 1 and kb == 16)

@@ -172,7 +172,7 @@ def mse(A: np.ndarray, Ahat: np.ndarray) -> float:
 
 
 # ----------------------------------------------------------------------------
-# Randomized Hadamard rotation of keys (Sec. 4.3: rotate the keys before quantization)
+# Randomized Hadamard rotation of keys (Sec. 4.4: rotate the keys before quantization)
 # ----------------------------------------------------------------------------
 def fwht_f32(x: np.ndarray) -> np.ndarray:
     """Unnormalised fast Walsh-Hadamard transform along the last axis in fp32, butterfly stages

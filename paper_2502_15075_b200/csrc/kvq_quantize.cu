@@ -270,6 +270,216 @@ __device__ __forceinline__ void quantize_task(const uint16_t* __restrict__ src, 
   }
 }
 
+// Minimum and maximum of the eight 16-bit values of a 16-byte piece, taken in the 16-bit type itself (two at a
+// time; exact, since every 16-bit value is an fp32 value and the order is the same).
+template <int DTYPE>
+__device__ __forceinline__ void minmax8(const uint4& r, float& mn, float& mx) {
+  if constexpr (DTYPE == KVQ_BF16) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&r);
+    const __nv_bfloat162 lo = __hmin2(__hmin2(h[0], h[1]), __hmin2(h[2], h[3]));
+    const __nv_bfloat162 hi = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));
+    mn = fminf(__low2float(lo), __high2float(lo));
+    mx = fmaxf(__low2float(hi), __high2float(hi));
+  } else {
+    const __half2* h = reinterpret_cast<const __half2*>(&r);
+    const __half2 lo = __hmin2(__hmin2(h[0], h[1]), __hmin2(h[2], h[3]));
+    const __half2 hi = __hmax2(__hmax2(h[0], h[1]), __hmax2(h[2], h[3]));
+    mn = fminf(__low2float(lo), __high2float(lo));
+    mx = fmaxf(__low2float(hi), __high2float(hi));
+  }
+}
+
+// quantize_task without rotation, four tokens per pass: the group minima / maxima of the four tokens are
+// reduced with a shuffle reduce-scatter, so that the group parameters (two divisions) are computed once per
+// group rather than once per lane, and are then broadcast to the lanes of the group.  FULLBLK: every token of
+// the task is new (no predicates).  Same results as quantize_task, bit for bit.
+template <int BITS, bool IS_V, int D, int DTYPE, bool FULLBLK>
+__device__ __forceinline__ void quantize_task_fast(const uint16_t* __restrict__ src, int64_t st, int gsz, int lo,
+                                                   int hi, uint8_t* __restrict__ codes,
+                                                   uint32_t* __restrict__ meta_out, int lane) {
+  constexpr int FPB = 8 / BITS;
+  constexpr int NMW = (D / 16) / FPB;
+  constexpr int LR = 2 * NMW;
+  constexpr int RS = 32 / LR;
+  constexpr int TT = task_tokens(D, BITS);
+  constexpr int TPL = TT / RS;
+  constexpr int K_ROW_BYTES = D * BITS / 8;
+  constexpr int NSET = FPB == 4 ? 2 : 1;      // a lane's fields may belong to two groups (groups of 32 at 2 bits)
+  const int rs = lane / LR, cs = lane % LR, mw = cs >> 1, rh = cs & 1;
+  const float qmax = (float)((1 << BITS) - 1);
+  const int spg = gsz >> 4;
+  const bool split = FPB > spg;
+  const int lpg = split ? 2 : 2 * spg / FPB;                 // lanes per group: 2, 4, 8 or 16
+  const int ng = D / gsz;
+  const int b0 = cs & 1, b1 = (cs >> 1) & 1;
+  const int gbase = lane & ~(lpg - 1);                       // first lane of this lane's group
+
+  auto token_of = [&](int k) {
+    if constexpr (IS_V) {
+      const int cmb = (k >> 2) * RS + rs, j = k & 3;
+      return 32 * (cmb >> 3) + 16 * ((cmb >> 2) & 1) + 2 * (cmb & 3) + (j >> 1) + 8 * (j & 1);
+    } else {
+      return k * RS + rs;
+    }
+  };
+
+#pragma unroll 1
+  for (int pass = 0; pass < TPL / 4; ++pass) {
+    uint4 raw[4][FPB];
+    bool valid[4];
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      const int tau = token_of(4 * pass + kk);
+      valid[kk] = FULLBLK || (tau >= lo && tau < hi);
+#pragma unroll
+      for (int f = 0; f < FPB; ++f) {
+        raw[kk][f] = make_uint4(0u, 0u, 0u, 0u);
+        if (valid[kk]) raw[kk][f] = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + 16 * (FPB * mw + f) + 8 * rh);
+      }
+    }
+    // ---- phase 1: minima / maxima of the lane's fields, per token and per set
+    float mn[NSET][4], mx[NSET][4];
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      float fm[FPB], fx[FPB];
+#pragma unroll
+      for (int f = 0; f < FPB; ++f) minmax8<DTYPE>(raw[kk][f], fm[f], fx[f]);
+      if constexpr (FPB == 1) { mn[0][kk] = fm[0]; mx[0][kk] = fx[0]; }
+      if constexpr (FPB == 2) { mn[0][kk] = fminf(fm[0], fm[1]); mx[0][kk] = fmaxf(fx[0], fx[1]); }
+      if constexpr (FPB == 4) {
+        mn[0][kk] = fminf(fm[0], fm[1]); mx[0][kk] = fmaxf(fx[0], fx[1]);
+        mn[1][kk] = fminf(fm[2], fm[3]); mx[1][kk] = fmaxf(fx[2], fx[3]);
+        if (!split) {
+          mn[0][kk] = mn[1][kk] = fminf(mn[0][kk], mn[1][kk]);
+          mx[0][kk] = mx[1][kk] = fmaxf(mx[0][kk], mx[1][kk]);
+        }
+      }
+    }
+    // ---- reduce-scatter over the lanes of the group: after lane bit 0 a lane holds tokens 2 b0 + {0, 1}, after
+    // bit 1 (groups of 4 lanes or more) token 2 b0 + b1; higher bits are plain butterflies
+    float pz[NSET][2], pinv[NSET][2];
+    uint32_t pmeta[NSET][2];
+#pragma unroll
+    for (int e = 0; e < NSET; ++e) {
+      if (e == 1 && !split) break;
+      float a0, a1, c0, c1;
+      {
+        const float sm0 = b0 ? mn[e][0] : mn[e][2], sm1 = b0 ? mn[e][1] : mn[e][3];
+        const float sx0 = b0 ? mx[e][0] : mx[e][2], sx1 = b0 ? mx[e][1] : mx[e][3];
+        a0 = fminf(b0 ? mn[e][2] : mn[e][0], __shfl_xor_sync(FULL, sm0, 1));
+        a1 = fminf(b0 ? mn[e][3] : mn[e][1], __shfl_xor_sync(FULL, sm1, 1));
+        c0 = fmaxf(b0 ? mx[e][2] : mx[e][0], __shfl_xor_sync(FULL, sx0, 1));
+        c1 = fmaxf(b0 ? mx[e][3] : mx[e][1], __shfl_xor_sync(FULL, sx1, 1));
+      }
+      if (lpg >= 4) {
+        const float sm = b1 ? a0 : a1, sx = b1 ? c0 : c1;
+        a0 = fminf(b1 ? a1 : a0, __shfl_xor_sync(FULL, sm, 2));
+        c0 = fmaxf(b1 ? c1 : c0, __shfl_xor_sync(FULL, sx, 2));
+      }
+      if (lpg >= 8) {
+        a0 = fminf(a0, __shfl_xor_sync(FULL, a0, 4));
+        c0 = fmaxf(c0, __shfl_xor_sync(FULL, c0, 4));
+      }
+      if (lpg >= 16) {
+        a0 = fminf(a0, __shfl_xor_sync(FULL, a0, 8));
+        c0 = fmaxf(c0, __shfl_xor_sync(FULL, c0, 8));
+      }
+      const GroupParams p0 = group_params(a0, c0, qmax);
+      pz[e][0] = p0.z; pinv[e][0] = p0.inv; pmeta[e][0] = p0.meta;
+      pz[e][1] = 0.f; pinv[e][1] = 0.f; pmeta[e][1] = 0u;
+      if (lpg == 2) {
+        const GroupParams p1 = group_params(a1, c1, qmax);
+        pz[e][1] = p1.z; pinv[e][1] = p1.inv; pmeta[e][1] = p1.meta;
+      }
+      // the lane (one per group) that holds a token's parameters stores its metadata word
+      if ((cs & (lpg - 1) & ~3) == 0) {
+        const int gi = (16 * FPB * mw) / gsz + e;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          if (i == 1 && lpg != 2) break;
+          const int kk = 2 * b0 + (lpg >= 4 ? b1 : i);
+          const int tau = token_of(4 * pass + kk);
+          if (FULLBLK || (tau >= lo && tau < hi)) meta_out[tau * ng + gi] = pmeta[e][i];
+        }
+      }
+    }
+    // ---- phase 2: codes, token by token, with the group's parameters fetched from the lane that made them
+    float vbyte[4][8];
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      const int tau = token_of(4 * pass + kk);
+      const int srcl = gbase + (lpg >= 4 ? (kk >> 1) + 2 * (kk & 1) : (kk >> 1));
+      const int el = (lpg >= 4) ? 0 : (kk & 1);
+      float zA, iA, zB, iB;
+      zA = __shfl_sync(FULL, el ? pz[0][1] : pz[0][0], srcl);
+      iA = __shfl_sync(FULL, el ? pinv[0][1] : pinv[0][0], srcl);
+      zB = zA; iB = iA;
+      if constexpr (NSET == 2) {
+        if (split) {
+          zB = __shfl_sync(FULL, el ? pz[1][1] : pz[1][0], srcl);
+          iB = __shfl_sync(FULL, el ? pinv[1][1] : pinv[1][0], srcl);
+        }
+      }
+      float bytev[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) bytev[i] = 0.f;
+#pragma unroll
+      for (int f = FPB - 1; f >= 0; --f) {
+        const float z = (FPB == 4 && f >= 2) ? zB : zA, inv = (FPB == 4 && f >= 2) ? iB : iA;
+        const uint32_t rw[4] = {raw[kk][f].x, raw[kk][f].y, raw[kk][f].z, raw[kk][f].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          float xa, xb;
+          if constexpr (DTYPE == KVQ_BF16) {
+            xa = __uint_as_float(rw[i] << 16);
+            xb = __uint_as_float(rw[i] & 0xFFFF0000u);
+          } else {
+            const float2 v = __half22float2(*reinterpret_cast<const __half2*>(&rw[i]));
+            xa = v.x; xb = v.y;
+          }
+          float ua = __fmul_rn(__fsub_rn(xa, z), inv), ub = __fmul_rn(__fsub_rn(xb, z), inv);
+          ua = fminf(fmaxf(ua, 0.0f), qmax);
+          ub = fminf(fmaxf(ub, 0.0f), qmax);
+          const float ra = __fsub_rn(__fadd_rn(ua, kRoundMagic), kRoundMagic);
+          const float rb = __fsub_rn(__fadd_rn(ub, kRoundMagic), kRoundMagic);
+          bytev[2 * i] = __fmaf_rn(bytev[2 * i], (float)(1 << BITS), ra);
+          bytev[2 * i + 1] = __fmaf_rn(bytev[2 * i + 1], (float)(1 << BITS), rb);
+        }
+      }
+      if constexpr (!IS_V) {
+        if (valid[kk]) {
+          constexpr int wpc = D * BITS / 128;
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const uint32_t w = pack_bytes(bytev[4 * hh], bytev[4 * hh + 1], bytev[4 * hh + 2], bytev[4 * hh + 3]);
+            *reinterpret_cast<uint32_t*>(codes + (size_t)tau * K_ROW_BYTES + chunk_word_byte(2 * rh + hh, mw, wpc, 4)) = w;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) vbyte[kk][i] = bytev[i];
+      }
+    }
+    if constexpr (IS_V) {
+      const int cmb = pass * RS + rs;
+      uint8_t* wbase = codes + (size_t)(cmb >> 3) * (4 * D * BITS) + mw * 512 + (cmb & 3) * 16 +
+                       4 * (2 * rh + ((cmb >> 2) & 1));
+      if (FULLBLK || (valid[0] && valid[1] && valid[2] && valid[3])) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          *reinterpret_cast<uint32_t*>(wbase + 64 * i) = pack_bytes(vbyte[0][i], vbyte[1][i], vbyte[2][i], vbyte[3][i]);
+      } else if (valid[0] || valid[1] || valid[2] || valid[3]) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            if (valid[kk]) wbase[64 * i + kk] = (uint8_t)vbyte[kk][i];
+        }
+      }
+    }
+  }
+}
+
 // 16-bit passthrough of one side of a task: rows [lo, hi) copied to the page as they are.
 __device__ __forceinline__ void copy_task_side(const uint16_t* __restrict__ src, int64_t st, int D, int lo, int hi,
                                                uint16_t* __restrict__ dst_rows, int lane) {
@@ -286,8 +496,8 @@ __host__ __device__ __forceinline__ bool append_fits(int t0, int t_new, int capa
 
 // Token-wise quantization of V (blockIdx.z == 0) and of K (blockIdx.z == 1).  grid.y = stream, grid.x strides
 // over the warp tasks touched by this append.
-template <int D, int DTYPE>
-__global__ void __launch_bounds__(kThreads)
+template <int D, int DTYPE, bool ROT>
+__global__ void __launch_bounds__(kThreads, ROT ? 1 : 3)
 quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
                    int64_t sb, int64_t sh, int64_t st, int t_new) {
   const bool is_v = blockIdx.z == 0;
@@ -317,9 +527,17 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
       }
       uint8_t* vb = pg + g.v_codes_off + (size_t)(tp0 >> 5) * (4 * D * bits);
       uint32_t* vm = reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / gsz);
-      if (bits == 2) quantize_task<2, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane, nullptr);
-      else if (bits == 4) quantize_task<4, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane, nullptr);
-      else quantize_task<8, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane, nullptr);
+      const bool full = lo == 0 && hi == TT;
+      if (bits == 2) {
+        if (full) quantize_task_fast<2, true, D, DTYPE, true>(src, st, gsz, lo, hi, vb, vm, lane);
+        else quantize_task_fast<2, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane);
+      } else if (bits == 4) {
+        if (full) quantize_task_fast<4, true, D, DTYPE, true>(src, st, gsz, lo, hi, vb, vm, lane);
+        else quantize_task_fast<4, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane);
+      } else {
+        if (full) quantize_task_fast<8, true, D, DTYPE, true>(src, st, gsz, lo, hi, vb, vm, lane);
+        else quantize_task_fast<8, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane);
+      }
     } else {
       if (bits == 16) {
         copy_task_side(src, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg) + (size_t)tp0 * D, lane);
@@ -327,14 +545,22 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
       }
       uint8_t* kr = pg + (size_t)tp0 * (D * bits / 8);
       uint32_t* km = reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / gsz);
-      if (c.k_signs) {
+      if constexpr (ROT) {
         if (bits == 2) quantize_task<2, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
         else if (bits == 4) quantize_task<4, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
         else quantize_task<8, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
       } else {
-        if (bits == 2) quantize_task<2, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane, nullptr);
-        else if (bits == 4) quantize_task<4, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane, nullptr);
-        else quantize_task<8, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane, nullptr);
+        const bool full = lo == 0 && hi == TT;
+        if (bits == 2) {
+          if (full) quantize_task_fast<2, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane);
+          else quantize_task_fast<2, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane);
+        } else if (bits == 4) {
+          if (full) quantize_task_fast<4, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane);
+          else quantize_task_fast<4, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane);
+        } else {
+          if (full) quantize_task_fast<8, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane);
+          else quantize_task_fast<8, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane);
+        }
       }
     }
   }
@@ -475,14 +701,17 @@ int launch_quantize_append(const Geom& g, const CachePtrs& c, const void* k_new,
   const int want = (148 * 16 + streams - 1) / streams;       // enough CTAs to fill the GPU, not one per task
   if (gx > want) gx = want;
   dim3 grid1(gx, streams, g.k_axis == 0 ? 2 : 1);            // z = 0 values, z = 1 token-wise keys
-  if (g.D == 128 && g.in_dtype == KVQ_BF16)
-    quant_token_kernel<128, KVQ_BF16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
-  else if (g.D == 128)
-    quant_token_kernel<128, KVQ_FP16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
-  else if (g.in_dtype == KVQ_BF16)
-    quant_token_kernel<64, KVQ_BF16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
-  else
-    quant_token_kernel<64, KVQ_FP16><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
+  const bool rot = c.k_signs != nullptr && g.k_axis == 0;
+#define KVQ_QLAUNCH(D_, T_)                                                                                  \
+  do {                                                                                                       \
+    if (rot) quant_token_kernel<D_, T_, true><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new); \
+    else quant_token_kernel<D_, T_, false><<<grid1, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);    \
+  } while (0)
+  if (g.D == 128 && g.in_dtype == KVQ_BF16) KVQ_QLAUNCH(128, KVQ_BF16);
+  else if (g.D == 128) KVQ_QLAUNCH(128, KVQ_FP16);
+  else if (g.in_dtype == KVQ_BF16) KVQ_QLAUNCH(64, KVQ_BF16);
+  else KVQ_QLAUNCH(64, KVQ_FP16);
+#undef KVQ_QLAUNCH
   if (g.k_axis == 1) {
     size_t smem = (size_t)kPageTokens * g.D * 3;
     cudaFuncSetAttribute(quant_kchan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 3);

@@ -1,4 +1,4 @@
-"""Key-only randomized Hadamard rotation (Sec. 4.3) through the CUDA library: rotated keys are quantized bit for
+"""Key-only randomized Hadamard rotation (Sec. 4.4) through the CUDA library: rotated keys are quantized bit for
 bit like the oracle's, dequantize rotates back bit-exactly, decode rotates q and stays within tolerance."""
 import numpy as np
 import pytest
@@ -62,7 +62,7 @@ def test_rotated_keys_parity(kvq, name):
 
 def test_rotation_lowers_attention_error_on_outlier_keys(kvq):
     """Keys with 8 heavy channels per head: rotating them before 4-bit quantization lowers the error of the
-    attention output against exact attention on the unquantized cache (Sec. 4.3, key-only rotation)."""
+    attention output against exact attention on the unquantized cache (Sec. 4.4, key-only rotation)."""
     w = wl.LLAMA_8B.with_(n_kv_heads=2, n_q_heads=8)
     e_rot, e_plain = [], []
     for seed in range(4):

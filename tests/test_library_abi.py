@@ -36,7 +36,7 @@ def test_every_declared_symbol_is_exported(kvq):
     for n in names:
         assert hasattr(lib, n), f"{n} declared in include/ but not exported"
     assert set(kvq.EXPORTS) <= set(names)
-    assert kvq.kvq_layout_version() == 1
+    assert kvq.kvq_layout_version() == 2
 
 
 @pytest.mark.parametrize("D,kb,vb,gk,gv,k_axis", [

@@ -1,4 +1,4 @@
-"""Pins for the oracle's key rotation (randomized Hadamard transform before quantization, Sec. 4.3)."""
+"""Pins for the oracle's key rotation (randomized Hadamard transform before quantization, Sec. 4.4)."""
 import numpy as np
 import pytest
 import scipy.linalg
@@ -42,7 +42,7 @@ def test_rotation_is_orthogonal_and_its_own_inverse(D):
 
 
 def test_rotation_spreads_outlier_channels_and_lowers_key_error():
-    """Sec. 4.3: rotating the keys disperses outliers; with 8 heavy channels the 4-bit reconstruction error drops."""
+    """Sec. 4.4: rotating the keys disperses outliers; with 8 heavy channels the 4-bit reconstruction error drops."""
     w = wl.LLAMA_8B.with_(n_kv_heads=1, n_q_heads=4)
     k, _ = wl.make_kv(w, tokens=512, batch=1)
     x = k[0, 0].float().numpy()
