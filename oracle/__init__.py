@@ -16,4 +16,4 @@ forms, invariants, brute force or a library routine.  Parity unpinned: the
 paper's absolute MSE / accuracy table values (they need its models and
 datasets); nothing in this package claims to reproduce them.
 """
-from . import quantizer, layout, attention, cache  # noqa: F401
+from . import quantizer, layout, attention, cache, error  # noqa: F401

@@ -166,7 +166,7 @@ def quantize_symmetric(A: np.ndarray, bits: int):
 
 
 def mse(A: np.ndarray, Ahat: np.ndarray) -> float:
-    """MSE = ||A - Ahat||_F^2 / number of entries (App. B.3)."""
+    """MSE = ||A - Ahat||_F^2 / number of entries (App. B.4, Frobenius-norm perspective)."""
     d = np.asarray(A, np.float64) - np.asarray(Ahat, np.float64)
     return float(np.sum(d * d) / d.size)
 
