@@ -193,6 +193,29 @@ int kvq_decode_attention_static(const kvq_config* cfg, const kvq_cache* cache,
                                 const void* q, void* out, int32_t out_dtype, float softmax_scale,
                                 void* cuda_stream);
 
+/*
+ * Reconstruction-error analysis of the quantizer (Sec. 4.1, experiment (i); Table 1 reports
+ * MSE(A, A^) = ||A - A^||_F^2 / number of entries, App. B.4, of the dequantized K and V caches per head).
+ * One pass over n_tokens tokens of K and V quantizes every token row in registers exactly as
+ * kvq_quantize_append would (kb, vb, gk, gv of cfg; token-wise groups: k_axis must be 0), reconstructs
+ * x^ = fmaf(code, scale, zero) and ADDS, per (batch, kv-head), to
+ *   sums[b][h][0..3] = (sum k^2, sum (k - k^)^2, sum v^2, sum (v - v^)^2)      (device, double, 8-byte aligned).
+ * The caller zeroes sums before the first call; several calls (chunks of tokens, layers) accumulate.  The MSE
+ * of a head is sums[..][1] / (n_tokens * head_dim), its squared Frobenius norm sums[..][0].  k, v, strides: as
+ * in kvq_quantize_append.  Writes nothing but sums.  Asynchronous on cuda_stream.
+ */
+int kvq_quant_error(const kvq_config* cfg, const void* k, const void* v,
+                    int64_t stride_b, int64_t stride_h, int64_t stride_t, int32_t n_tokens,
+                    double* sums, void* cuda_stream);
+
+/*
+ * Host only.  The difference of bit widths that equalises the Frobenius error bounds of App. B.4,
+ * ||E||_F <~ sqrt(L d) / 2^b ||A||_F for keys and values:  b_K - b_V = log2(||K||_F / ||V||_F)
+ * = 0.5 log2(sum_k2 / sum_v2).  (App. B.4 prints the ratio inverted, which contradicts its own conclusion
+ * b_K > b_V; this is the form its preceding line implies.)  Both sums must be positive.
+ */
+int kvq_bit_balance(double sum_k2, double sum_v2, double* bk_minus_bv);
+
 /* Synchronises cuda_stream, reads *cache->status and returns KVQ_OK, KVQ_ERR_CAPACITY,
  * KVQ_ERR_DEVICE_TIMEOUT or KVQ_ERR_CUDA_LAUNCH (a CUDA error surfaced by the sync). */
 int kvq_check_status(const kvq_cache* cache, void* cuda_stream);

@@ -227,6 +227,27 @@ int kvq_dequantize(const kvq_config* cfg, const kvq_cache* cache, void* k_out, v
   return launch_dequantize(g, c, k_out, v_out, t_begin, t_end, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int kvq_quant_error(const kvq_config* cfg, const void* k, const void* v, int64_t stride_b, int64_t stride_h,
+                    int64_t stride_t, int32_t n_tokens, double* sums, void* cuda_stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != KVQ_OK) return rc;
+  if (g.k_axis != 0) return KVQ_ERR_UNSUPPORTED;          // token-wise groups only
+  if (!k || !v || !sums || n_tokens < 0) return KVQ_ERR_INVALID_ARG;
+  if (n_tokens == 0) return KVQ_OK;
+  if (stride_t < g.D || stride_h < 0 || stride_b < 0) return KVQ_ERR_INVALID_ARG;
+  if (!aligned16(k) || !aligned16(v) || (stride_b % 8) || (stride_h % 8) || (stride_t % 8) ||
+      (reinterpret_cast<uintptr_t>(sums) & 7u))
+    return KVQ_ERR_MISALIGNED;
+  return launch_quant_error(g, k, v, stride_b, stride_h, stride_t, n_tokens, sums, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int kvq_bit_balance(double sum_k2, double sum_v2, double* bk_minus_bv) {
+  if (!bk_minus_bv || !(sum_k2 > 0.0) || !(sum_v2 > 0.0)) return KVQ_ERR_INVALID_ARG;
+  *bk_minus_bv = 0.5 * log2(sum_k2 / sum_v2);
+  return KVQ_OK;
+}
+
 int kvq_check_status(const kvq_cache* cache, void* cuda_stream) {
   if (!cache || !cache->status) return KVQ_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

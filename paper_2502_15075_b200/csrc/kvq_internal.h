@@ -11,6 +11,9 @@ int launch_quantize_append(const Geom& g, const CachePtrs& c, const void* k_new,
 int launch_dequantize(const Geom& g, const CachePtrs& c, void* k_out, void* v_out, int t_begin, int t_end,
                       cudaStream_t stream);
 
+int launch_quant_error(const Geom& g, const void* k, const void* v, int64_t sb, int64_t sh, int64_t st, int n_tokens,
+                       double* sums, cudaStream_t stream);
+
 // Number of sequence splits the decode kernels use for this geometry (also sizes the workspace).
 int decode_num_splits(const Geom& g);
 size_t decode_workspace_bytes(const Geom& g);

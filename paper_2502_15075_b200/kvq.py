@@ -51,16 +51,20 @@ _lib.kvq_decode_attention_static.argtypes = [_P(kvq_config), _P(kvq_cache), ctyp
                                              ctypes.c_int32, ctypes.c_float, ctypes.c_void_p]
 _lib.kvq_dequantize.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
                                 ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
+_lib.kvq_quant_error.argtypes = [_P(kvq_config), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                 ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
+_lib.kvq_bit_balance.argtypes = [ctypes.c_double, ctypes.c_double, _P(ctypes.c_double)]
 _lib.kvq_check_status.argtypes = [_P(kvq_cache), ctypes.c_void_p]
 _lib.kvq_strerror.argtypes = [ctypes.c_int]
 _lib.kvq_strerror.restype = ctypes.c_char_p
 for _f in ("kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes", "kvq_quantize_append",
-           "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize", "kvq_check_status"):
+           "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize", "kvq_check_status",
+           "kvq_quant_error", "kvq_bit_balance"):
     getattr(_lib, _f).restype = ctypes.c_int
 
 EXPORTS = ("kvq_layout_version", "kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes",
            "kvq_quantize_append", "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize",
-           "kvq_check_status", "kvq_strerror")
+           "kvq_check_status", "kvq_strerror", "kvq_quant_error", "kvq_bit_balance")
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -194,6 +198,24 @@ def kvq_dequantize(cfg: kvq_config, cache: Cache, k_out: Optional[torch.Tensor],
                                k_out.data_ptr() if k_out is not None else None,
                                v_out.data_ptr() if v_out is not None else None,
                                t_begin, t_end, _stream_ptr(stream)), "kvq_dequantize")
+
+
+def kvq_quant_error(cfg: kvq_config, k: torch.Tensor, v: torch.Tensor, sums: torch.Tensor,
+                    stream: Optional[torch.cuda.Stream] = None):
+    """k, v: CUDA tensors [B, Hkv, T, D] of the config's dtype (last dim contiguous, identical strides);
+    sums: CUDA float64 [B, Hkv, 4], added to: (sum k^2, sum (k - k^)^2, sum v^2, sum (v - v^)^2)."""
+    assert k.is_cuda and v.is_cuda and k.shape == v.shape and k.dim() == 4 and k.stride() == v.stride()
+    assert k.stride(3) == 1 and _dtype_code(k.dtype) == cfg.in_dtype and v.dtype == k.dtype
+    assert sums.is_cuda and sums.dtype == torch.float64 and sums.is_contiguous()
+    assert tuple(sums.shape) == (cfg.batch, cfg.n_kv_heads, 4) and k.shape[0] == cfg.batch and k.shape[1] == cfg.n_kv_heads
+    _check(_lib.kvq_quant_error(ctypes.byref(cfg), k.data_ptr(), v.data_ptr(), k.stride(0), k.stride(1), k.stride(2),
+                                k.shape[2], sums.data_ptr(), _stream_ptr(stream)), "kvq_quant_error")
+
+
+def kvq_bit_balance(sum_k2: float, sum_v2: float) -> float:
+    out = ctypes.c_double()
+    _check(_lib.kvq_bit_balance(float(sum_k2), float(sum_v2), ctypes.byref(out)), "kvq_bit_balance")
+    return out.value
 
 
 def kvq_check_status(cache: Cache, stream: Optional[torch.cuda.Stream] = None) -> int:

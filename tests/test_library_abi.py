@@ -90,3 +90,11 @@ def test_null_and_misaligned_arguments_fail_before_any_launch(kvq):
     assert lib.kvq_quantize_append(ctypes.byref(cfg), ctypes.byref(ok), 4096, 4096, 0, 0, 128, 257, None) == -5  # > capacity
     assert lib.kvq_decode_attention(ctypes.byref(cfg), ctypes.byref(ok), 4096, 4096, 2, 0.0, 4096, 8, None) == -4
     assert lib.kvq_decode_attention(ctypes.byref(cfg), ctypes.byref(ok), 4096, 4096, 9, 0.0, 4096, 1 << 20, None) == -1
+
+
+def test_bit_balance_is_the_log_ratio_of_the_frobenius_norms(kvq):
+    assert kvq.kvq_bit_balance(16.0, 1.0) == 2.0          # ||K||_F = 4 ||V||_F -> two more bits for keys
+    assert kvq.kvq_bit_balance(1.0, 1.0) == 0.0
+    assert kvq.kvq_bit_balance(1.0, 4.0) == -1.0
+    with pytest.raises(kvq.KvqError):
+        kvq.kvq_bit_balance(0.0, 1.0)
