@@ -10,7 +10,8 @@ namespace mma {
 // Instantiation units (kvq_decode_mma_inst_*.cu).
 #define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB)                                                  \
   extern template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB>(                                   \
-      const Geom&, const CachePtrs&, const void*, float, float*, int, void*, int, unsigned long long, cudaStream_t);
+      const Geom&, const CachePtrs&, const void*, float, float*, int, void*, int, unsigned long long,              \
+      unsigned long long, long long, cudaStream_t);
 #include "kvq_decode_mma_list.inc"
 #undef KVQ_MMA_DECL
 
@@ -42,7 +43,7 @@ static unsigned long long next_call_id() {
 
 // Finds the instantiation for this geometry; launches it unless `probe`.  *grid = CTAs of the launch.
 static int pick(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap, void* out,
-                int out_dtype, cudaStream_t stream, bool probe, int* grid) {
+                int out_dtype, const DecodeDebug& dbg, cudaStream_t stream, bool probe, int* grid) {
   const int ngk = (g.k_axis == 1 || g.kb == 16) ? 1 : g.D / g.gk;
   const int ngv = (g.vb == 16) ? 1 : g.D / g.gv;
   const int nh = g.G <= 4 ? 1 : 2;                                         // query heads per lane
@@ -52,7 +53,8 @@ static int pick(const Geom& g, const CachePtrs& c, const void* q, float c1, floa
     *grid = 148 * MINB_;                                                                                      \
     if (probe) return KVQ_OK;                                                                                 \
     return mma::launch_mma_inst<D_, KB_, VB_, KAXIS_, NGK_, NGV_, NH_, NW_, MINB_>(                          \
-        g, c, q, c1, ws, s_cap, out, out_dtype, next_call_id(), stream);                                      \
+        g, c, q, c1, ws, s_cap, out, out_dtype, next_call_id(),                                               \
+        dbg.wait_us ? 1000ull * dbg.wait_us : mma::kWaitTimeoutNs, dbg.skip_page, stream);                    \
   }
 #include "kvq_decode_mma_list.inc"
 #undef KVQ_MMA_DECL
@@ -63,14 +65,14 @@ bool decode_mma_supported(const Geom& g) {
   if (g.B > mma::kMaxBatchFlat) return false;
   CachePtrs none{};
   int grid = 0;
-  return pick(g, none, nullptr, 0.f, nullptr, 0, nullptr, 0, nullptr, true, &grid) == KVQ_OK;
+  return pick(g, none, nullptr, 0.f, nullptr, 0, nullptr, 0, DecodeDebug{}, nullptr, true, &grid) == KVQ_OK;
 }
 
 int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype, float c1,
-                      float* ws, cudaStream_t stream) {
+                      float* ws, const DecodeDebug& dbg, cudaStream_t stream) {
   const int s_cap = flat_slot_cap(g);
   int grid = 0;
-  return pick(g, c, q, c1, ws, s_cap, out, out_dtype, stream, false, &grid);
+  return pick(g, c, q, c1, ws, s_cap, out, out_dtype, dbg, stream, false, &grid);
 }
 
 }  // namespace kvq

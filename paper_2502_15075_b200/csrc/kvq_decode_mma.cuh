@@ -29,7 +29,7 @@
 namespace kvq {
 namespace mma {
 
-constexpr unsigned long long kWaitTimeoutNs = 2000000000ull;   // 2 s
+constexpr unsigned long long kWaitTimeoutNs = 2000000000ull;   // default limit of a device-side wait: 2 s
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -67,18 +67,18 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Slow path of a wait: poll with a parking hint, give up after kWaitTimeoutNs.
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
+// Slow path of a wait: poll with a parking hint, give up after limit_ns.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
   const unsigned long long t0 = globaltimer_ns();
   while (true) {
     if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
-    if (globaltimer_ns() - t0 > kWaitTimeoutNs) return false;
+    if (globaltimer_ns() - t0 > limit_ns) return false;
   }
 }
 // Wait for the phase with the given parity; bounded in time (false = gave up).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity);
+  return mbar_wait_slow(bar, parity, limit_ns);
 }
 // One bulk copy global -> this CTA's shared memory, completion counted in bytes on `bar`.
 // dst, src and bytes are multiples of 16.

@@ -5,7 +5,8 @@ namespace kvq {
 namespace mma {
 #define KVQ_MMA_DECL(D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB)                                          \
   template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB>(                                          \
-      const Geom&, const CachePtrs&, const void*, float, float*, int, void*, int, unsigned long long, cudaStream_t);
+      const Geom&, const CachePtrs&, const void*, float, float*, int, void*, int, unsigned long long,              \
+      unsigned long long, long long, cudaStream_t);
 KVQ_MMA_DECL(128, 4, 2, 1, 1, 1, 1, 4, 3)
 KVQ_MMA_DECL(128, 8, 2, 1, 1, 1, 1, 4, 2)
 #undef KVQ_MMA_DECL

@@ -140,7 +140,8 @@ constexpr int kFlushBlocks = 512;          // fold the int32 value accumulators 
 template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NH, int NW, int MINB>
 __global__ void __launch_bounds__((NW + 1) * 32, MINB)
 decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1, float* __restrict__ ws,
-                  int s_cap, int stages, void* __restrict__ out, int out_dtype, unsigned long long call_id) {
+                  int s_cap, int stages, void* __restrict__ out, int out_dtype, unsigned long long call_id,
+                  unsigned long long wait_ns, long long skip_x) {
   constexpr int NR = D / 16;                // 16-channel register slots per key row
   constexpr int KS32 = D / 32;              // k-steps of an 8-bit MMA over the channels
   constexpr int MT = D / 16;                // m-tiles of PV (16 channels each)
@@ -248,13 +249,15 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       bool ok = true;
       for (long long x = x_lo; x < x_hi; ++x, ++it) {
         if (it >= stages) {
-          ok = mbar_wait(bar0 + 8 * (stages + stage), phase);
+          ok = mbar_wait(bar0 + 8 * (stages + stage), phase, wait_ns);
           if (!ok || *abort_flag) { ok = false; break; }
         }
         const uint8_t* src = c.pages + ((size_t)(b * Hkv + h) * g.n_pages + page) * (size_t)g.page_bytes;
         const uint32_t fb = bar0 + 8 * stage;
-        mbar_expect_tx(fb, (uint32_t)g.page_bytes);
-        bulk_load(ring + stage * sl.page_stride, src, (uint32_t)g.page_bytes, fb);
+        if (x != skip_x) {          // (skip_x: test hook - a page that never arrives makes the consumers' bounded wait expire)
+          mbar_expect_tx(fb, (uint32_t)g.page_bytes);
+          bulk_load(ring + stage * sl.page_stride, src, (uint32_t)g.page_bytes, fb);
+        }
         if (++stage == stages) { stage = 0; phase ^= 1; }
         if (++page == pages_b) {
           page = 0;
@@ -273,7 +276,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       // last copies issued, whether or not a consumer is still going to.
       for (int k = 1; k <= stages && k <= it; ++k) {
         const int j = it - k;
-        mbar_wait(bar0 + 8 * (j % stages), (j / stages) & 1);
+        mbar_wait(bar0 + 8 * (j % stages), (j / stages) & 1, wait_ns);
       }
     }
     return;
@@ -460,7 +463,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       const int nv = min(kPageTokens, n_tok - (page + pp) * kPageTokens);
       const bool tail_k = (KAXIS == 1) && (nv < kPageTokens);
       if (!aborted) {
-        const bool got = mbar_wait(bar0 + 8 * stage, phase);
+        const bool got = mbar_wait(bar0 + 8 * stage, phase, wait_ns);
         if (!__all_sync(FULL, got)) {
           aborted = true;
           *abort_flag = 1;
@@ -881,7 +884,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 // Launches one instantiation; defined per instantiation unit.
 template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NH, int NW, int MINB>
 int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap,
-                    void* out, int out_dtype, unsigned long long call_id, cudaStream_t stream) {
+                    void* out, int out_dtype, unsigned long long call_id, unsigned long long wait_ns, long long skip_x,
+                    cudaStream_t stream) {
   const int budget = (227 * 1024) / MINB - 1024;            // shared memory per CTA for MINB resident CTAs per SM
   int stages = (budget - smem_layout(0, 0, NW, g.B, D, NH, KAXIS == 1).total) / ((g.page_bytes + 127) & ~127);
   if (stages > 16) stages = 16;
@@ -891,7 +895,7 @@ int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, 
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
     return KVQ_ERR_CUDA_LAUNCH;
   kern<<<148 * MINB, (NW + 1) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap,
-                                                         stages, out, out_dtype, call_id);
+                                                         stages, out, out_dtype, call_id, wait_ns, skip_x);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
 

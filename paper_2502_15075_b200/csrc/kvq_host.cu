@@ -3,6 +3,7 @@
 #include <math.h>
 #include <stdlib.h>
 
+#include "kvq_debug.h"
 #include "kvq_internal.h"
 
 namespace kvq {
@@ -80,14 +81,12 @@ size_t decode_workspace_bytes(const Geom& g) {
 }
 
 int launch_decode_attention(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
-                            float softmax_scale, void* workspace, cudaStream_t stream) {
+                            float softmax_scale, void* workspace, cudaStream_t stream, const DecodeDebug& dbg) {
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)g.D);
   const float scale_log2e = scale * 1.4426950408889634f;
   float* ws = static_cast<float*>(workspace);
-  // KVQ_DECODE_GENERIC=1 (debugging aid) routes every configuration through the plain-ALU kernel.
-  const char* force_generic = getenv("KVQ_DECODE_GENERIC");
-  const bool use_mma = decode_mma_supported(g) && !(force_generic && force_generic[0] == '1');
-  if (use_mma) return launch_decode_mma(g, c, q, out, out_dtype, scale_log2e, ws, stream);
+  const bool use_mma = decode_mma_supported(g) && !dbg.force_generic;
+  if (use_mma) return launch_decode_mma(g, c, q, out, out_dtype, scale_log2e, ws, dbg, stream);
   const int n_split = decode_num_splits(g);
   int rc = launch_decode_generic(g, c, q, scale_log2e, ws, n_split, stream);
   if (rc != KVQ_OK) return rc;
@@ -211,6 +210,44 @@ int kvq_decode_attention_static(const kvq_config* cfg, const kvq_cache* cache, c
   if (rc != KVQ_OK) return rc;
   return launch_decode_attention(g, c, q, out, out_dtype, softmax_scale, scratch,
                                  static_cast<cudaStream_t>(cuda_stream));
+}
+
+// ---------------------------------------------------------------------------
+// Test hooks (kvq_debug.h): the same validation and launch path as kvq_decode_attention with one knob turned.
+// ---------------------------------------------------------------------------
+static int decode_with(const kvq_config* cfg, const kvq_cache* cache, const void* q, void* out, int32_t out_dtype,
+                       float softmax_scale, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                       const DecodeDebug& dbg) {
+  Geom g;
+  CachePtrs c;
+  int rc = make_geom(cfg, &g);
+  if (rc != KVQ_OK) return rc;
+  rc = make_cache(g, cache, &c);
+  if (rc != KVQ_OK) return rc;
+  if (!q || !out || !workspace) return KVQ_ERR_INVALID_ARG;
+  if (out_dtype != KVQ_FP16 && out_dtype != KVQ_BF16 && out_dtype != KVQ_FP32) return KVQ_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return KVQ_ERR_MISALIGNED;
+  if (workspace_bytes < decode_workspace_bytes(g)) return KVQ_ERR_WORKSPACE_TOO_SMALL;
+  return launch_decode_attention(g, c, q, out, out_dtype, softmax_scale, workspace,
+                                 static_cast<cudaStream_t>(cuda_stream), dbg);
+}
+
+int kvq_debug_decode_generic(const kvq_config* cfg, const kvq_cache* cache, const void* q, void* out,
+                             int32_t out_dtype, float softmax_scale, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
+  DecodeDebug dbg;
+  dbg.force_generic = true;
+  return decode_with(cfg, cache, q, out, out_dtype, softmax_scale, workspace, workspace_bytes, cuda_stream, dbg);
+}
+
+int kvq_debug_decode_stall(const kvq_config* cfg, const kvq_cache* cache, const void* q, void* out, int32_t out_dtype,
+                           float softmax_scale, void* workspace, size_t workspace_bytes, int64_t skip_page,
+                           uint32_t wait_us, void* cuda_stream) {
+  if (wait_us == 0 || wait_us > 100000u) return KVQ_ERR_INVALID_ARG;      // the hook never waits longer than 0.1 s
+  DecodeDebug dbg;
+  dbg.skip_page = skip_page;
+  dbg.wait_us = wait_us;
+  return decode_with(cfg, cache, q, out, out_dtype, softmax_scale, workspace, workspace_bytes, cuda_stream, dbg);
 }
 
 int kvq_dequantize(const kvq_config* cfg, const kvq_cache* cache, void* k_out, void* v_out, int32_t t_begin,

@@ -17,8 +17,15 @@ int launch_quant_error(const Geom& g, const void* k, const void* v, int64_t sb, 
 // Number of sequence splits the decode kernels use for this geometry (also sizes the workspace).
 int decode_num_splits(const Geom& g);
 size_t decode_workspace_bytes(const Geom& g);
+// Test hooks of a decode launch (all zero / -1 in the product path).
+struct DecodeDebug {
+  bool force_generic = false;    // run the plain-ALU kernel whatever the configuration
+  uint32_t wait_us = 0;          // limit of every device-side wait in microseconds (0: the default, 2 s)
+  long long skip_page = -1;      // flat page index whose copy is never issued (-1: none)
+};
 int launch_decode_attention(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
-                            float softmax_scale, void* workspace, cudaStream_t stream);
+                            float softmax_scale, void* workspace, cudaStream_t stream,
+                            const DecodeDebug& dbg = DecodeDebug{});
 
 }  // namespace kvq
 
@@ -34,5 +41,5 @@ namespace kvq {
 bool decode_mma_supported(const Geom& g);
 size_t flat_workspace_bytes(const Geom& g);
 int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
-                      float scale_log2e, float* ws, cudaStream_t stream);
+                      float scale_log2e, float* ws, const DecodeDebug& dbg, cudaStream_t stream);
 }  // namespace kvq

@@ -54,12 +54,16 @@ _lib.kvq_dequantize.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, 
 _lib.kvq_quant_error.argtypes = [_P(kvq_config), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                  ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
 _lib.kvq_bit_balance.argtypes = [ctypes.c_double, ctypes.c_double, _P(ctypes.c_double)]
+_lib.kvq_debug_decode_generic.argtypes = _lib.kvq_decode_attention.argtypes
+_lib.kvq_debug_decode_stall.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
+                                        ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
+                                        ctypes.c_int64, ctypes.c_uint32, ctypes.c_void_p]
 _lib.kvq_check_status.argtypes = [_P(kvq_cache), ctypes.c_void_p]
 _lib.kvq_strerror.argtypes = [ctypes.c_int]
 _lib.kvq_strerror.restype = ctypes.c_char_p
 for _f in ("kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes", "kvq_quantize_append",
            "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize", "kvq_check_status",
-           "kvq_quant_error", "kvq_bit_balance"):
+           "kvq_quant_error", "kvq_bit_balance", "kvq_debug_decode_generic", "kvq_debug_decode_stall"):
     getattr(_lib, _f).restype = ctypes.c_int
 
 EXPORTS = ("kvq_layout_version", "kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes",
@@ -216,6 +220,24 @@ def kvq_bit_balance(sum_k2: float, sum_v2: float) -> float:
     out = ctypes.c_double()
     _check(_lib.kvq_bit_balance(float(sum_k2), float(sum_v2), ctypes.byref(out)), "kvq_bit_balance")
     return out.value
+
+
+def kvq_debug_decode_generic(cfg: kvq_config, cache: Cache, q: torch.Tensor, out: torch.Tensor,
+                             workspace: torch.Tensor, softmax_scale: float = 0.0):
+    """Test hook: kvq_decode_attention through the plain-ALU kernel whatever the configuration."""
+    _check(_lib.kvq_debug_decode_generic(ctypes.byref(cfg), ctypes.byref(cache.c), q.data_ptr(), out.data_ptr(),
+                                         _dtype_code(out.dtype), float(softmax_scale), workspace.data_ptr(),
+                                         workspace.numel() * workspace.element_size(), _stream_ptr(None)),
+           "kvq_debug_decode_generic")
+
+
+def kvq_debug_decode_stall(cfg: kvq_config, cache: Cache, q: torch.Tensor, out: torch.Tensor,
+                           workspace: torch.Tensor, skip_page: int, wait_us: int):
+    """Test hook: decode with one page copy withheld and every device-side wait limited to wait_us."""
+    _check(_lib.kvq_debug_decode_stall(ctypes.byref(cfg), ctypes.byref(cache.c), q.data_ptr(), out.data_ptr(),
+                                       _dtype_code(out.dtype), 0.0, workspace.data_ptr(),
+                                       workspace.numel() * workspace.element_size(), int(skip_page), int(wait_us),
+                                       _stream_ptr(None)), "kvq_debug_decode_stall")
 
 
 def kvq_check_status(cache: Cache, stream: Optional[torch.cuda.Stream] = None) -> int:
