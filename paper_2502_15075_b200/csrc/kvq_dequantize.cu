@@ -13,6 +13,8 @@ namespace kvq {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kTilePad = 8;     // the shared [128][D + 8] tile: a row stride of D + 8 elements spreads the token rows
+                                // over the banks (a stride of D would put every row on the same banks)
 
 // All sizes that index arithmetic divides by are powers of two: use shifts.
 __device__ __forceinline__ int ilog2(int x) { return 31 - __clz(x); }
@@ -45,7 +47,7 @@ __device__ __forceinline__ void expand_keys(const uint8_t* spage, const Geom& g,
         const uint32_t m = meta[g.k_axis == 1 ? d0 + j : t * ngk + ((d0 + j) >> lgk)];
         o[j] = f32_to_bits16(fmaf(code, meta_scale(m), meta_zero(m)), g.in_dtype);
       }
-      *reinterpret_cast<uint2*>(tile + t * D + d0) =
+      *reinterpret_cast<uint2*>(tile + t * (D + kTilePad) + d0) =
           make_uint2((uint32_t)o[0] | ((uint32_t)o[1] << 16), (uint32_t)o[2] | ((uint32_t)o[3] << 16));
     }
   }
@@ -73,7 +75,7 @@ __device__ __forceinline__ void expand_values(const uint8_t* spage, const Geom& 
         const int t = blk * 32 + tau;
         const uint32_t m = meta[t * ngv + (d >> lgv)];
         const float code = (float)((word >> (8 * j + B * f)) & ((1u << B) - 1u));
-        tile[t * D + d] = f32_to_bits16(fmaf(code, meta_scale(m), meta_zero(m)), g.in_dtype);
+        tile[t * (D + kTilePad) + d] = f32_to_bits16(fmaf(code, meta_scale(m), meta_zero(m)), g.in_dtype);
       }
     }
   }
@@ -139,12 +141,12 @@ __device__ __forceinline__ void dequant_keys_rotated_d(const uint8_t* spage, con
   else dequant_keys_rotated<B, 64>(spage, g, tail, signs, out, lo, hi, tid);
 }
 
-// Copy token rows [lo, hi) of tile[128][D] to out rows (16-byte vectors).
-__device__ __forceinline__ void store_rows(const uint16_t* tile, uint16_t* out, int D, int lo, int hi, int tid) {
+// Copy token rows [lo, hi) of a tile with row stride `ts` elements to out rows (16-byte vectors).
+__device__ __forceinline__ void store_rows(const uint16_t* tile, int ts, uint16_t* out, int D, int lo, int hi, int tid) {
   const int vpr = D / 8, lv = ilog2(vpr);
   for (int idx = tid; idx < (hi - lo) * vpr; idx += kThreads) {
     const int t = lo + (idx >> lv), v = idx & (vpr - 1);
-    reinterpret_cast<uint4*>(out + (size_t)t * D)[v] = reinterpret_cast<const uint4*>(tile + t * D)[v];
+    reinterpret_cast<uint4*>(out + (size_t)t * D)[v] = reinterpret_cast<const uint4*>(tile + t * ts)[v];
   }
 }
 
@@ -177,13 +179,13 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
   if (blockIdx.z == 0) k_out = nullptr; else v_out = nullptr;
   if (v_out) {
     if (g.vb == 16) {
-      store_rows(reinterpret_cast<const uint16_t*>(spage + g.v_codes_off), v_out + out_base, D, lo, hi_l, tid);
+      store_rows(reinterpret_cast<const uint16_t*>(spage + g.v_codes_off), D, v_out + out_base, D, lo, hi_l, tid);
     } else {
       if (g.vb == 2) expand_values<2>(spage, g, tile, tid);
       else if (g.vb == 4) expand_values<4>(spage, g, tile, tid);
       else expand_values<8>(spage, g, tile, tid);
       __syncthreads();
-      store_rows(tile, v_out + out_base, D, lo, hi_l, tid);
+      store_rows(tile, D + kTilePad, v_out + out_base, D, lo, hi_l, tid);
     }
   }
   if (k_out) {
@@ -204,14 +206,14 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
             (g.in_dtype == KVQ_FP16) ? hbits : f32_to_bits16(bits16_to_f32(hbits, KVQ_FP16), KVQ_BF16);
       }
     } else if (g.kb == 16) {
-      store_rows(reinterpret_cast<const uint16_t*>(spage), k_out + out_base, D, lo, hi_l, tid);
+      store_rows(reinterpret_cast<const uint16_t*>(spage), D, k_out + out_base, D, lo, hi_l, tid);
     } else {
       __syncthreads();          // the value tile has been copied out
       if (g.kb == 2) expand_keys<2>(spage, g, tile, tid);
       else if (g.kb == 4) expand_keys<4>(spage, g, tile, tid);
       else expand_keys<8>(spage, g, tile, tid);
       __syncthreads();
-      store_rows(tile, k_out + out_base, D, lo, hi_l, tid);
+      store_rows(tile, D + kTilePad, k_out + out_base, D, lo, hi_l, tid);
     }
   }
 }
@@ -223,8 +225,9 @@ int launch_dequantize(const Geom& g, const CachePtrs& c, void* k_out, void* v_ou
   if (t_end <= t_begin) return KVQ_OK;
   const int page0 = t_begin / kPageTokens;
   const int page1 = (t_end + kPageTokens - 1) / kPageTokens;
-  const size_t smem = (size_t)((g.page_bytes + 15) & ~15) + (size_t)kPageTokens * g.D * 2;
-  cudaFuncSetAttribute(dequant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 4 + 128 * 128 * 2);
+  const size_t smem = (size_t)((g.page_bytes + 15) & ~15) + (size_t)kPageTokens * (g.D + kTilePad) * 2;
+  cudaFuncSetAttribute(dequant_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                       128 * 128 * 4 + 128 * (128 + kTilePad) * 2);
   dim3 grid(page1 - page0, g.B * g.Hkv, 2);
   dequant_kernel<<<grid, kThreads, smem, stream>>>(g, c, static_cast<uint16_t*>(k_out),
                                                    static_cast<uint16_t*>(v_out), t_begin, t_end, page0);
