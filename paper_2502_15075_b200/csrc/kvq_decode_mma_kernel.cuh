@@ -10,7 +10,7 @@ namespace mma {
 
 constexpr int kMaxBatchFlat = 1024;   // the flat partition keeps a per-batch prefix in shared memory
 
-// Flat split of all pages over the grid, identical in the decode and the merge kernel.
+// Flat split of all pages over the grid.
 struct FlatPlan {
   long long N;       // total pages over all streams
   int c_eff;         // CTAs that take part
@@ -134,7 +134,7 @@ constexpr int kFlushBlocks = 512;          // fold the int32 value accumulators 
 //
 // Both contractions run on integer tensor-core MMAs over the raw code bytes (m16n8k32, int32 accumulate).
 // The 8 columns of an MMA carry (head, limb) pairs: q as 16-bit fixed point in two signed bytes for QK^T, the
-// softmax weight times the value scale as 23-bit fixed point in three unsigned bytes for PV.  Lane (g, t) of a
+// softmax weight times the value scale as 31-bit (NH = 2: 24-bit) fixed point in unsigned bytes for PV.  Lane (g, t) of a
 // warp (g = lane / 4, t = lane % 4) owns query heads t (and t + 4 when NH = 2): its accumulator columns 2t, 2t+1
 // are the limbs of that head, so logits, softmax and the fixed-point weights need no exchange between lanes.
 template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NH, int NW, int MINB>
