@@ -7,7 +7,7 @@ namespace mma {
   template int launch_mma_inst<D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB>(                                          \
       const Geom&, const CachePtrs&, const void*, float, float*, int, void*, int, unsigned long long,              \
       unsigned long long, long long, cudaStream_t);
-KVQ_MMA_DECL(128, 4, 2, 1, 1, 1, 1, 4, 3)
+KVQ_MMA_DECL(128, 4, 2, 1, 1, 1, 1, 4, 2)
 KVQ_MMA_DECL(128, 8, 2, 1, 1, 1, 1, 4, 2)
 #undef KVQ_MMA_DECL
 }  // namespace mma

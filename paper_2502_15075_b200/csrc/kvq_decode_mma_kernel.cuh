@@ -104,21 +104,20 @@ __host__ __device__ inline size_t tag_offset_floats(int streams, int s_cap, int 
 constexpr float kQFix = 32512.0f;          // largest |Q| of the 16-bit fixed-point q (hi limb stays within +-127)
 constexpr float kQFix3 = 8300000.0f;       // ... of the 24-bit fixed-point q * s of channel-wise keys (three limbs)
 
-// Limb `which` (0 = lowest) of the balanced three-byte split Q = (l2 * 256 + l1) * 256 + l0 of four values times
-// `scale`, |Q| <= kQFix3, as one word of four signed bytes; which < 0 gives zero.
-__device__ __forceinline__ uint32_t fixed_point_limb3(const float (&t)[4], float scale, int which) {
-  uint32_t w = 0;
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int Q = __float2int_rn(t[j] * scale);
-    const int l0 = (int)(int8_t)(Q & 0xFF);
-    const int Q1 = (Q - l0) >> 8;
-    const int l1 = (int)(int8_t)(Q1 & 0xFF);
-    const int l2 = (Q1 - l1) >> 8;
-    const int v = which == 0 ? l0 : (which == 1 ? l1 : (which == 2 ? l2 : 0));
-    w |= (uint32_t)(v & 0xFF) << (8 * j);
-  }
-  return w;
+// Four values times `scale` rounded to integers |Q| <= kQFix3 and taken apart as two's-complement bytes,
+// Q = b2 * 65536 + b1 * 256 + b0 with b2 signed and b1, b0 unsigned.  Operand words of a lane: even operand
+// columns (odd = 0) carry b2 in n-tile 0 (signed bytes) and b1 in n-tile 1 (unsigned bytes), odd columns nothing in
+// n-tile 0 and b0 in n-tile 1.  Byte j of a word belongs to t[j].
+__device__ __forceinline__ void fixed_point_bytes3(const float (&t)[4], float scale, int odd, uint32_t& w_nt0,
+                                                   uint32_t& w_nt1) {
+  const uint32_t q0 = (uint32_t)__float2int_rn(t[0] * scale), q1 = (uint32_t)__float2int_rn(t[1] * scale);
+  const uint32_t q2 = (uint32_t)__float2int_rn(t[2] * scale), q3 = (uint32_t)__float2int_rn(t[3] * scale);
+  // byte k of each of the four integers -> one word: selectors pick byte k of (q0, q1) and of (q2, q3)
+  const uint32_t sel = odd ? 0x0040u : 0x0051u;                  // odd: byte 0; even: byte 1
+  const uint32_t lo01 = prmt(q0, q1, sel), lo23 = prmt(q2, q3, sel);
+  w_nt1 = prmt(lo01, lo23, 0x5410u);
+  const uint32_t hi01 = prmt(q0, q1, 0x0062u), hi23 = prmt(q2, q3, 0x0062u);   // byte 2 of each
+  w_nt0 = odd ? 0u : prmt(hi01, hi23, 0x5410u);
 }
 // The softmax weights enter PV as fixed point P = rint(p * s_V * 2^PBITS / s_lim), p = 2^(logit - reference) with the
 // reference kHeadroom bits above the largest logit seen so far, so that a larger logit rarely forces a rescale.
@@ -284,7 +283,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
   // =========================================================== consumer warps
   uint32_t qB[NH][NTK][NR];    // QK^T B operands: column gid = (head gid/2 + 4 nh, limb gid%2), channels 16 r + 4 tid + {0..3};
-                               // channel-wise keys: n-tile 0 carries limbs (2, 1), n-tile 1 limbs (0, none)
+                               // channel-wise keys: n-tile 0 carries (byte 2 signed, none), n-tile 1 (byte 1, byte 0) unsigned
   float hs[NH];                // c1 / fixed-point scale of q, own heads (tid + 4 nh)
   float qsum[NH][NGK];         // c1 * sum of q over each key group, own heads
   float zq[NH];                // channel-wise keys: c1 * sum_d q_d z_d of the current page, own heads
@@ -472,7 +471,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       }
       const uint8_t* sp = smem + stage * sl.page_stride;
 
-      // ---- channel-wise keys: per page, the operand of the integer MMAs is q_d * s_d in 16-bit fixed point
+      // ---- channel-wise keys: per page, the operand of the integer MMAs is q_d * s_d in 24-bit fixed point
       // (scale from max|q| of the head times the page's largest channel scale).  Each warp makes the operands of
       // its own slots, all warps exchange them through shared memory; sum_d q_d z_d is summed in fp32 the same way.
       if constexpr (KAXIS == 1) {
@@ -509,8 +508,10 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
                   t[j] = qa[j] * sz.x;
                   zsum = fmaf(qa[j], sz.y, zsum);
                 }
-                sB[(((buf * NH + nh) * 2 + 0) * NR + r) * 32 + lane] = fixed_point_limb3(t, scale, (gid & 1) ? 1 : 2);
-                sB[(((buf * NH + nh) * 2 + 1) * NR + r) * 32 + lane] = fixed_point_limb3(t, scale, (gid & 1) ? -1 : 0);
+                uint32_t w0, w1;
+                fixed_point_bytes3(t, scale, gid & 1, w0, w1);
+                sB[(((buf * NH + nh) * 2 + 0) * NR + r) * 32 + lane] = w0;
+                sB[(((buf * NH + nh) * 2 + 1) * NR + r) * 32 + lane] = w1;
               }
             }
             zsum += __shfl_xor_sync(FULL, zsum, 1);
@@ -601,17 +602,19 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
                 for (int nh = 0; nh < NH; ++nh) {
 #pragma unroll
-                  for (int nt = 0; nt < NTK; ++nt)
-                    mma16832_u8s8(S[j][nh][nt], a0, a1, a2, a3, qB[nh][nt][2 * s], qB[nh][nt][2 * s + 1]);
+                  for (int nt = 0; nt < NTK; ++nt) {
+                    if (nt == 0) mma16832_u8s8(S[j][nh][nt], a0, a1, a2, a3, qB[nh][nt][2 * s], qB[nh][nt][2 * s + 1]);
+                    else mma16832_u8u8(S[j][nh][nt], a0, a1, a2, a3, qB[nh][nt][2 * s], qB[nh][nt][2 * s + 1]);
+                  }
                 }
               }
               // accumulator columns 2 tid, 2 tid + 1 = (hi, lo) limbs of head tid + 4 nh: sum_d code_d Q_d = 256 hi + lo
-              // (channel-wise keys: limbs (2, 1) in n-tile 0 and limb 0 in n-tile 1, combined in fp32)
+              // (channel-wise keys: the signed top byte in n-tile 0, the two unsigned lower bytes in n-tile 1, combined in fp32)
               if constexpr (KAXIS == 1) {
 #pragma unroll
                 for (int nh = 0; nh < NH; ++nh) {
-                  const float t0 = fmaf((float)S[0][nh][0][0], 65536.f, (float)(S[0][nh][0][1] * 256 + S[0][nh][NTK - 1][0]));
-                  const float t1 = fmaf((float)S[0][nh][0][2], 65536.f, (float)(S[0][nh][0][3] * 256 + S[0][nh][NTK - 1][2]));
+                  const float t0 = fmaf((float)S[0][nh][0][0], 65536.f, fmaf((float)S[0][nh][NTK - 1][0], 256.f, (float)S[0][nh][NTK - 1][1]));
+                  const float t1 = fmaf((float)S[0][nh][0][2], 65536.f, fmaf((float)S[0][nh][NTK - 1][2], 256.f, (float)S[0][nh][NTK - 1][3]));
                   L[u][0][nh] = fmaf(t0, hs[nh], zq[nh]);
                   L[u][1][nh] = fmaf(t1, hs[nh], zq[nh]);
                 }
