@@ -63,3 +63,25 @@ def lse_merge(parts):
     num = sum(np.exp(m - mstar) * o for m, _, o in parts)
     den = sum(np.exp(m - mstar) * l for m, l, _ in parts)
     return num / den
+
+
+def decode_attention_rows(q: np.ndarray, K: np.ndarray, V: np.ndarray, seq_len, scale=None) -> np.ndarray:
+    """Several query rows per head (App. A.1: Q has one row per position, S = Q K^T / sqrt(d)), for the last R
+    positions of each sequence, with the causal mask of a decoder (reading: the paper writes no mask; its models
+    are causal language models): row r belongs to the token at position seq_len - R + r and attends to the
+    tokens at positions <= its own, i.e. to the first seq_len - (R - 1 - r) tokens.
+
+    q (B, R, Hq, D); K, V (B, Hkv, T, D) fp64; returns (B, R, Hq, D) fp64.  A row whose token does not exist
+    (seq_len < R - r) gives zeros."""
+    B, R, Hq, D = q.shape
+    G = Hq // K.shape[1]
+    if scale is None or scale <= 0:
+        scale = 1.0 / math.sqrt(D)
+    out = np.zeros((B, R, Hq, D), np.float64)
+    for b in range(B):
+        for r in range(R):
+            n = max(0, int(seq_len[b]) - (R - 1 - r))
+            for h in range(Hq):
+                kv = h // G
+                out[b, r, h] = attend_one(q[b, r, h].astype(np.float64), K[b, kv, :n], V[b, kv, :n], scale)
+    return out

@@ -167,6 +167,14 @@ class OracleCache:
         K, V = self.values_f64()
         return attention.decode_attention(q, K, V, self.seq_len, scale)
 
+    def decode_rows(self, q_bits: np.ndarray, scale=None) -> np.ndarray:
+        """q_bits uint16 [B, R, Hq, D]: R causal query rows for the last R cached tokens -> fp64 [B, R, Hq, D]."""
+        q = quantizer.bits_to_f32(q_bits, self.dtype).astype(np.float64)
+        if self.k_signs is not None:
+            q = quantizer.hadamard_rotate_f64(q, self.k_signs)
+        K, V = self.values_f64()
+        return attention.decode_attention_rows(q, K, V, self.seq_len, scale)
+
     def decode_streams(self, q_bits: np.ndarray, streams, scale=None):
         """Same as decode but only for the listed (b, kv_head) streams; returns
         {(b, kv_head): fp64 (G, D)} (used to sample full-size workloads)."""

@@ -333,3 +333,30 @@ def test_k4v2_beats_k2v4_when_key_norm_exceeds_value_norm():
                 c.append(bits_of(k), bits_of(v))
                 acc.append(np.linalg.norm(c.decode(bits_of(q)) - exact) / np.linalg.norm(exact))
         assert np.mean(e42) < np.mean(e24), (base.name, np.mean(e42), np.mean(e24))
+
+
+def test_multi_row_attention_matches_library_causal_sdpa():
+    """Several query rows with a decoder's causal mask against torch's scaled_dot_product_attention in fp64:
+    the R rows are the last R positions of a T-token sequence."""
+    B, Hq, Hkv, T, D, R = 2, 4, 2, 37, 16, 3
+    q = RNG.normal(size=(B, R, Hq, D))
+    K = RNG.normal(size=(B, Hkv, T, D))
+    V = RNG.normal(size=(B, Hkv, T, D))
+    got = oa.decode_attention_rows(q, K, V, [T, T])
+    G = Hq // Hkv
+    mask = torch.zeros((R, T), dtype=torch.bool)
+    for r in range(R):
+        mask[r, : T - (R - 1 - r)] = True
+    qt = torch.from_numpy(q).permute(0, 2, 1, 3)                              # (B, Hq, R, D)
+    kt = torch.from_numpy(K).repeat_interleave(G, 1)
+    vt = torch.from_numpy(V).repeat_interleave(G, 1)
+    want = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, attn_mask=mask).permute(0, 2, 1, 3).numpy()
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-13)
+    # one row is the plain decode step; the last row of several sees the whole cache
+    one = oa.decode_attention_rows(q[:, -1:], K, V, [T, T])
+    assert np.array_equal(one[:, 0], oa.decode_attention(q[:, -1], K, V, [T, T]))
+    assert np.array_equal(got[:, -1], one[:, 0])
+    # ragged: a sequence shorter than the number of rows leaves the rows without a token at zero
+    short = oa.decode_attention_rows(q, K, V, [2, T])
+    assert not short[0, 0].any() and short[0, 1].any() and short[0, 2].any()
+    assert np.array_equal(short[0, 1, 0], V[0, 0, 0])                          # row 1 sees exactly token 0
