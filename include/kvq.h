@@ -154,6 +154,24 @@ int kvq_decode_attention(const kvq_config* cfg, const kvq_cache* cache,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Decode with several query rows per head (App. A.1: Q has one row per position, S = Q K^T / sqrt(d)), the shape
+ * of speculative decoding and chunked prefill.  The n_rows rows are the queries of the LAST n_rows cached tokens of
+ * each sequence (append their keys and values first), under a decoder's causal mask: row r attends to the tokens
+ * t < seq_len[b] - (n_rows - 1 - r); a row whose token does not exist (seq_len[b] < n_rows - r) gives zeros.
+ * n_rows = 1 is kvq_decode_attention.
+ *   q, out: device, [batch][n_rows][n_q_heads][head_dim] contiguous (q in_dtype, out out_dtype).
+ *   The (row, head) pairs of a KV head share its stream like query heads do: n_rows * (n_q_heads / n_kv_heads)
+ *   may be up to 4 for every configuration the tensor-core path serves (2/4/8-bit codes, token-wise or
+ *   channel-wise keys, head_dim 128, or head_dim 64 with K4V2 and groups of 64) and up to 8 for token-wise K4V2
+ *   at head_dim 128; otherwise KVQ_ERR_UNSUPPORTED.  workspace: at least kvq_workspace_bytes_rows(cfg, n_rows).
+ * Everything else as kvq_decode_attention.
+ */
+int kvq_workspace_bytes_rows(const kvq_config* cfg, int32_t n_rows, size_t* out);
+int kvq_decode_attention_rows(const kvq_config* cfg, const kvq_cache* cache,
+                              const void* q, int32_t n_rows, void* out, int32_t out_dtype, float softmax_scale,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Reconstruct tokens t_begin <= t < min(t_end, seq_len[b]) as x^ = fmaf(code, s, z) rounded to
  * in_dtype (App. B.1: A^ = scale * Q); tail keys are converted from fp16.
  *   k_out, v_out: device, in_dtype, [batch][n_kv_heads][capacity_tokens][head_dim] contiguous;

@@ -23,6 +23,7 @@ struct Geom {
   int k_codes_bytes, k_meta_off, k_meta_bytes;
   int v_codes_off, v_codes_bytes, v_meta_off, v_meta_bytes;
   int page_bytes;
+  int rows;          // query rows per head of a decode call (1 = a plain decode step)
 };
 
 // Pointers of one cache (device memory).

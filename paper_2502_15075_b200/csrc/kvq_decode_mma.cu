@@ -29,7 +29,7 @@ int flat_slot_cap(const Geom& g) {
 // Partials [streams][slots][G][D + 2] floats, then one 64-bit count word per stream.
 size_t flat_workspace_bytes(const Geom& g) {
   const int s_cap = flat_slot_cap(g);
-  return mma::tag_offset_floats(g.B * g.Hkv, s_cap, g.G, g.D) * sizeof(float) + (size_t)g.B * g.Hkv * 8;
+  return mma::tag_offset_floats(g.B * g.Hkv, s_cap, g.G * g.rows, g.D) * sizeof(float) + (size_t)g.B * g.Hkv * 8;
 }
 
 // Id of a launch: the words that count a stream's finished partials carry it, so that neither stale workspace
@@ -46,7 +46,7 @@ static int pick(const Geom& g, const CachePtrs& c, const void* q, float c1, floa
                 int out_dtype, const DecodeDebug& dbg, cudaStream_t stream, bool probe, int* grid) {
   const int ngk = (g.k_axis == 1 || g.kb == 16) ? 1 : g.D / g.gk;
   const int ngv = (g.vb == 16) ? 1 : g.D / g.gv;
-  const int nh = g.G <= 4 ? 1 : 2;                                         // query heads per lane
+  const int nh = g.G * g.rows <= 4 ? 1 : 2;                                // (virtual) query heads per lane
 #define KVQ_MMA_DECL(D_, KB_, VB_, KAXIS_, NGK_, NGV_, NH_, NW_, MINB_)                                      \
   if (g.D == D_ && g.kb == KB_ && g.vb == VB_ && g.k_axis == KAXIS_ && ngk == NGK_ && ngv == NGV_ &&          \
       NH_ == nh) {                                                                                            \

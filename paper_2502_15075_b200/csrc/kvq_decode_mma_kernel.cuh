@@ -174,7 +174,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
   const int tid_ = threadIdx.x, lane = tid_ & 31, warp = tid_ >> 5;
   const int gid = lane >> 2, tid = lane & 3;
-  const int B = g.B, Hkv = g.Hkv, G = g.G;
+  // Several query rows per head (g.rows > 1) are served as virtual heads: row r of head j is virtual head
+  // r * Gq + j, with its own causal limit on the tokens it may see.
+  const int B = g.B, Hkv = g.Hkv, Gq = g.G, G = g.G * g.rows;
 
   // ---- plan: pages per sequence, prefix over the batch
   if (tid_ == 0) { sPref[0] = 0; sMisc[0] = 0; sMisc[1] = 0; }
@@ -209,8 +211,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   // an empty sequence has no page and therefore no CTA of its own: its output rows are zero
   for (int bb = blockIdx.x; bb < B; bb += gridDim.x) {
     if (sPref[bb + 1] == sPref[bb]) {
-      for (int i = tid_; i < g.Hq * D; i += blockDim.x) {
-        const size_t oi = (size_t)bb * g.Hq * D + i;
+      for (int i = tid_; i < g.rows * g.Hq * D; i += blockDim.x) {
+        const size_t oi = (size_t)bb * g.rows * g.Hq * D + i;
         if (out_dtype == KVQ_FP32) static_cast<float*>(out)[oi] = 0.f;
         else static_cast<uint16_t*>(out)[oi] = 0;
       }
@@ -342,6 +344,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     const int seg_pages = (int)min((long long)(pages_b - page), x_hi - x);
     const int n_tok = clamped_len(c.seq_len, b, g.capacity);
     const int stream = b * Hkv + h;
+    int limh[NH];                          // tokens the lane's heads may attend to (causal limit of their query row)
+#pragma unroll
+    for (int nh = 0; nh < NH; ++nh) limh[nh] = n_tok - (g.rows - 1 - min((tid + 4 * nh) / Gq, g.rows - 1));
 
     // ---- segment start: q operands, group sums and a clean state for this stream's heads
     {
@@ -350,7 +355,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       for (int nh = 0; nh < NH; ++nh) {
         const int hb = (gid >> 1) + 4 * nh;                          // head of this lane's operand column
         float qv[NR][4];
-        const uint16_t* qrow = q + ((size_t)b * g.Hq + (size_t)h * G + hb) * D;
+        const uint16_t* qrow = q + (((size_t)b * g.rows + hb / Gq) * g.Hq + (size_t)h * Gq + hb % Gq) * D;
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
           uint2 raw = make_uint2(0u, 0u);
@@ -637,10 +642,11 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               }
             }
             if (MASKED) {
+              const int tokg = (page + pp) * kPageTokens + tok0;        // position of row tok0 in the sequence
 #pragma unroll
               for (int nh = 0; nh < NH; ++nh) {
-                if (!vld[u][0]) L[u][0][nh] = -INFINITY;
-                if (!vld[u][1]) L[u][1][nh] = -INFINITY;
+                if (!vld[u][0] || tokg >= limh[nh]) L[u][0][nh] = -INFINITY;
+                if (!vld[u][1] || tokg + 8 >= limh[nh]) L[u][1][nh] = -INFINITY;
               }
             }
           }
@@ -710,6 +716,10 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             for (int nh = 0; nh < NH; ++nh) {
               p[0][nh] = ex2(L[u][0][nh] - m_ref[nh]);
               p[1][nh] = ex2(L[u][1][nh] - m_ref[nh]);
+              if (MASKED) {       // a head that has seen no token yet has no reference: its weights are zero
+                if (L[u][0][nh] == -INFINITY) p[0][nh] = 0.f;
+                if (L[u][1][nh] == -INFINITY) p[1][nh] = 0.f;
+              }
               l[nh] += p[0][nh] + p[1][nh];
             }
 #pragma unroll
@@ -756,7 +766,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           }
         };
 
-        if (nv - wq * 32 >= 32) do_block(std::false_type{});
+        // the masked variant also serves the last tokens when several causal query rows see different prefixes
+        if (nv - wq * 32 >= 32 && (page + pp) * kPageTokens + wq * 32 + 32 <= n_tok - (g.rows - 1)) do_block(std::false_type{});
         else do_block(std::true_type{});
       }
       __syncwarp();
@@ -812,7 +823,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           }
           if (n_part == 1) {
             const float r = lsum > 0.f ? o / lsum : 0.f;
-            const size_t oi = ((size_t)b * g.Hq + (size_t)h * G + head) * D + d;
+            const size_t oi = (((size_t)b * g.rows + head / Gq) * g.Hq + (size_t)h * Gq + head % Gq) * D + d;
             if (out_dtype == KVQ_FP32) static_cast<float*>(out)[oi] = r;
             else static_cast<uint16_t*>(out)[oi] = f32_to_bits16(r, out_dtype);
           } else {
@@ -859,7 +870,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
                 mstar = mb;
               }
               const float r = den > 0.f ? num / den : 0.f;
-              const size_t oi = ((size_t)b * g.Hq + (size_t)h * G + head) * D + d;
+              const size_t oi = (((size_t)b * g.rows + head / Gq) * g.Hq + (size_t)h * Gq + head % Gq) * D + d;
               if (out_dtype == KVQ_FP32) static_cast<float*>(out)[oi] = r;
               else static_cast<uint16_t*>(out)[oi] = f32_to_bits16(r, out_dtype);
             }

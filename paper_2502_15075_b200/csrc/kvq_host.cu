@@ -42,6 +42,7 @@ int make_geom(const kvq_config* cfg, Geom* out) {
   g.v_meta_off = g.v_codes_off + g.v_codes_bytes;
   g.v_meta_bytes = (g.vb == 16) ? 0 : kPageTokens * (g.D / g.gv) * 4;
   g.page_bytes = g.v_meta_off + g.v_meta_bytes;
+  g.rows = 1;
   *out = g;
   return KVQ_OK;
 }
@@ -75,7 +76,7 @@ int decode_num_splits(const Geom& g) {
 }
 
 size_t decode_workspace_bytes(const Geom& g) {
-  size_t generic = (size_t)g.B * g.Hq * decode_num_splits(g) * (g.D + 2) * sizeof(float);
+  size_t generic = (size_t)g.B * g.Hq * g.rows * decode_num_splits(g) * (g.D + 2) * sizeof(float);
   size_t flat = flat_workspace_bytes(g);
   return generic > flat ? generic : flat;
 }
@@ -209,6 +210,37 @@ int kvq_decode_attention_static(const kvq_config* cfg, const kvq_cache* cache, c
   rc = static_scratch_ptr(&scratch);
   if (rc != KVQ_OK) return rc;
   return launch_decode_attention(g, c, q, out, out_dtype, softmax_scale, scratch,
+                                 static_cast<cudaStream_t>(cuda_stream));
+}
+
+int kvq_workspace_bytes_rows(const kvq_config* cfg, int32_t n_rows, size_t* out) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != KVQ_OK) return rc;
+  if (!out || n_rows < 1) return KVQ_ERR_INVALID_ARG;
+  if (n_rows * g.G > kMaxGroupHeads) return KVQ_ERR_UNSUPPORTED;
+  g.rows = n_rows;
+  *out = decode_workspace_bytes(g);
+  return KVQ_OK;
+}
+
+int kvq_decode_attention_rows(const kvq_config* cfg, const kvq_cache* cache, const void* q, int32_t n_rows,
+                              void* out, int32_t out_dtype, float softmax_scale, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+  Geom g;
+  CachePtrs c;
+  int rc = make_geom(cfg, &g);
+  if (rc != KVQ_OK) return rc;
+  rc = make_cache(g, cache, &c);
+  if (rc != KVQ_OK) return rc;
+  if (!q || !out || !workspace || n_rows < 1) return KVQ_ERR_INVALID_ARG;
+  if (out_dtype != KVQ_FP16 && out_dtype != KVQ_BF16 && out_dtype != KVQ_FP32) return KVQ_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return KVQ_ERR_MISALIGNED;
+  if (n_rows * g.G > kMaxGroupHeads) return KVQ_ERR_UNSUPPORTED;
+  g.rows = n_rows;
+  if (n_rows > 1 && !decode_mma_supported(g)) return KVQ_ERR_UNSUPPORTED;      // only the fast path serves several rows
+  if (workspace_bytes < decode_workspace_bytes(g)) return KVQ_ERR_WORKSPACE_TOO_SMALL;
+  return launch_decode_attention(g, c, q, out, out_dtype, softmax_scale, workspace,
                                  static_cast<cudaStream_t>(cuda_stream));
 }
 

@@ -54,6 +54,10 @@ _lib.kvq_dequantize.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, 
 _lib.kvq_quant_error.argtypes = [_P(kvq_config), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                  ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
 _lib.kvq_bit_balance.argtypes = [ctypes.c_double, ctypes.c_double, _P(ctypes.c_double)]
+_lib.kvq_workspace_bytes_rows.argtypes = [_P(kvq_config), ctypes.c_int32, _P(ctypes.c_size_t)]
+_lib.kvq_decode_attention_rows.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_int32,
+                                           ctypes.c_void_p, ctypes.c_int32, ctypes.c_float, ctypes.c_void_p,
+                                           ctypes.c_size_t, ctypes.c_void_p]
 _lib.kvq_debug_decode_generic.argtypes = _lib.kvq_decode_attention.argtypes
 _lib.kvq_debug_decode_stall.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
                                         ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
@@ -63,12 +67,14 @@ _lib.kvq_strerror.argtypes = [ctypes.c_int]
 _lib.kvq_strerror.restype = ctypes.c_char_p
 for _f in ("kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes", "kvq_quantize_append",
            "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize", "kvq_check_status",
-           "kvq_quant_error", "kvq_bit_balance", "kvq_debug_decode_generic", "kvq_debug_decode_stall"):
+           "kvq_quant_error", "kvq_bit_balance", "kvq_debug_decode_generic", "kvq_debug_decode_stall",
+           "kvq_workspace_bytes_rows", "kvq_decode_attention_rows"):
     getattr(_lib, _f).restype = ctypes.c_int
 
 EXPORTS = ("kvq_layout_version", "kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes",
            "kvq_quantize_append", "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize",
-           "kvq_check_status", "kvq_strerror", "kvq_quant_error", "kvq_bit_balance")
+           "kvq_check_status", "kvq_strerror", "kvq_quant_error", "kvq_bit_balance", "kvq_workspace_bytes_rows",
+           "kvq_decode_attention_rows")
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -220,6 +226,25 @@ def kvq_bit_balance(sum_k2: float, sum_v2: float) -> float:
     out = ctypes.c_double()
     _check(_lib.kvq_bit_balance(float(sum_k2), float(sum_v2), ctypes.byref(out)), "kvq_bit_balance")
     return out.value
+
+
+def kvq_workspace_bytes_rows(cfg: kvq_config, n_rows: int) -> int:
+    out = ctypes.c_size_t()
+    _check(_lib.kvq_workspace_bytes_rows(ctypes.byref(cfg), int(n_rows), ctypes.byref(out)), "kvq_workspace_bytes_rows")
+    return out.value
+
+
+def kvq_decode_attention_rows(cfg: kvq_config, cache: Cache, q: torch.Tensor, out: torch.Tensor,
+                              workspace: torch.Tensor, softmax_scale: float = 0.0,
+                              stream: Optional[torch.cuda.Stream] = None):
+    """q, out [B, R, Hq, D]: R causal query rows for the last R cached tokens of every sequence."""
+    assert q.is_cuda and out.is_cuda and q.is_contiguous() and out.is_contiguous() and q.dim() == 4
+    assert (q.shape[0], q.shape[2], q.shape[3]) == (cfg.batch, cfg.n_q_heads, cfg.head_dim) and out.shape == q.shape
+    assert _dtype_code(q.dtype) == cfg.in_dtype
+    _check(_lib.kvq_decode_attention_rows(ctypes.byref(cfg), ctypes.byref(cache.c), q.data_ptr(), q.shape[1],
+                                          out.data_ptr(), _dtype_code(out.dtype), float(softmax_scale),
+                                          workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                          _stream_ptr(stream)), "kvq_decode_attention_rows")
 
 
 def kvq_debug_decode_generic(cfg: kvq_config, cache: Cache, q: torch.Tensor, out: torch.Tensor,
