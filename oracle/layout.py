@@ -37,6 +37,10 @@ kept in quads of qw = min(wpc, 4) words, quad-major:
     byte   = (word // 4)*(nchunks*4*qw) + chunk*(4*qw) + (word % 4)*4
 (for wpc <= 4 this is simply chunk-major).
 b = 16 (either side): plain rows [token][D] of the input's 16-bit patterns.
+b in {1, 3, 6}: bit planes.  A 3-bit code is stored as a 2-bit plane (code >> 1) followed by a 1-bit plane
+(code & 1), a 6-bit code as a 4-bit plane (code >> 2) followed by a 2-bit plane (code & 3), a 1-bit code as one
+1-bit plane; every plane is a code region of its own width laid out as above (the high plane first), so the
+region still holds 128*D*b/8 bytes.  1-bit planes need head_dim 128.
 
 Meta: (scale fp16, zero fp16) pairs, 4 bytes each.  Per-token axis:
 [128 tokens][D/g groups]; per-channel K: [D channels] (one group per channel
@@ -49,6 +53,11 @@ import dataclasses
 import numpy as np
 
 PAGE_TOKENS = 128
+
+
+def planes(b: int):
+    """Bit planes of a b-bit code, high plane first: [(plane bits, right shift of the code)]."""
+    return {1: [(1, 0)], 2: [(2, 0)], 3: [(2, 1), (1, 0)], 4: [(4, 0)], 6: [(4, 2), (2, 0)], 8: [(8, 0)]}[b]
 
 
 @dataclasses.dataclass(frozen=True)
@@ -142,11 +151,16 @@ def _put_codes(region: np.ndarray, pos_fn, tokens: np.ndarray, codes: np.ndarray
         region[tt * 2 * D + 2 * dd] = (u & 0xFF).astype(np.uint8)
         region[tt * 2 * D + 2 * dd + 1] = (u >> 8).astype(np.uint8)
         return
-    byte, shift = pos_fn(tt, dd, D, b)
-    mask = (1 << b) - 1
-    # clear, then set (fields never straddle bytes because b divides 8)
-    np.bitwise_and.at(region, byte.ravel(), (~(mask << shift.ravel()) & 0xFF).astype(np.uint8))
-    np.bitwise_or.at(region, byte.ravel(), ((codes.astype(np.uint32).ravel() & mask) << shift.ravel()).astype(np.uint8))
+    off = 0
+    for pb, sh in planes(b):
+        byte, shift = pos_fn(tt, dd, D, pb)
+        byte = byte + off
+        mask = (1 << pb) - 1
+        part = (codes.astype(np.uint32).ravel() >> sh) & mask
+        # clear, then set (fields never straddle bytes because the plane width divides 8)
+        np.bitwise_and.at(region, byte.ravel(), (~(mask << shift.ravel()) & 0xFF).astype(np.uint8))
+        np.bitwise_or.at(region, byte.ravel(), (part << shift.ravel()).astype(np.uint8))
+        off += PAGE_TOKENS * D * pb // 8
 
 
 def _get_codes(region: np.ndarray, pos_fn, D, b) -> np.ndarray:
@@ -155,8 +169,13 @@ def _get_codes(region: np.ndarray, pos_fn, D, b) -> np.ndarray:
         lo = region[tt * 2 * D + 2 * dd].astype(np.uint16)
         hi = region[tt * 2 * D + 2 * dd + 1].astype(np.uint16)
         return lo | (hi << 8)
-    byte, shift = pos_fn(tt, dd, D, b)
-    return ((region[byte] >> shift.astype(np.uint8)) & ((1 << b) - 1)).astype(np.uint8)
+    out = np.zeros(tt.shape, np.uint8)
+    off = 0
+    for pb, sh in planes(b):
+        byte, shift = pos_fn(tt, dd, D, pb)
+        out |= (((region[byte + off] >> shift.astype(np.uint8)) & ((1 << pb) - 1)) << sh).astype(np.uint8)
+        off += PAGE_TOKENS * D * pb // 8
+    return out
 
 
 def put_k_codes(page: np.ndarray, L: Layout, tokens, codes):

@@ -79,7 +79,7 @@ def quantize_groups(x32: np.ndarray, bits: int):
     Returns (codes uint8 (..., g), s16 uint16 (...), z16 uint16 (...)):
     the b-bit codes and the fp16 bit patterns of scale and zero-point.
     """
-    assert bits in (2, 4, 8)
+    assert bits in (1, 2, 3, 4, 6, 8)
     x = np.asarray(x32, dtype=np.float32)
     assert np.all(np.isfinite(x)), "precondition: finite inputs"
     qmax = F32(2 ** bits - 1)

@@ -360,3 +360,29 @@ def test_multi_row_attention_matches_library_causal_sdpa():
     short = oa.decode_attention_rows(q, K, V, [2, T])
     assert not short[0, 0].any() and short[0, 1].any() and short[0, 2].any()
     assert np.array_equal(short[0, 1, 0], V[0, 0, 0])                          # row 1 sees exactly token 0
+
+
+@pytest.mark.parametrize("D,b", [(128, 1), (128, 3), (128, 6), (64, 6)])
+def test_bit_plane_widths_tile_the_region_and_keep_their_planes_apart(D, b):
+    """1-, 3- and 6-bit codes are stored as planes of 1, 2 or 4 bits (high plane first): every code bit of every
+    (token, channel) owns one distinct bit of the region, the region is exactly 128*D*b/8 bytes, and the high
+    plane of a code sits in the first part of the region."""
+    L = ol.Layout(D, b, b, 64, 64, 0)
+    assert L.k_codes_bytes == 128 * D * b // 8 and L.v_codes_bytes == 128 * D * b // 8
+    for put, get, off in ((ol.put_k_codes, ol.get_k_codes, 0), (ol.put_v_codes, ol.get_v_codes, L.v_codes_off)):
+        seen = np.zeros(L.page_bytes, np.uint16)
+        for bit in range(b):                                   # one code bit at a time: count the region bits it sets
+            page = np.zeros(L.page_bytes, np.uint8)
+            put(page, L, np.arange(128), np.full((128, D), 1 << bit, np.uint16))
+            ones = np.unpackbits(page[off: off + 128 * D * b // 8]).sum()
+            assert ones == 128 * D and not page[:off].any() and not page[off + 128 * D * b // 8:].any()
+            assert not (seen[: L.page_bytes] & page).any()     # no region bit serves two code bits
+            seen |= page
+            assert np.array_equal(get(page, L), np.full((128, D), 1 << bit, np.uint8))
+        assert np.all(seen[off: off + 128 * D * b // 8] == 0xFF)
+    # hand-computed: 3-bit key code 5 = (2-bit plane 2, 1-bit plane 1) of token 0, channel 0
+    if b == 3:
+        page = np.zeros(L.page_bytes, np.uint8)
+        codes = np.zeros((1, D), np.uint16); codes[0, 0] = 5
+        ol.put_k_codes(page, L, np.array([0]), codes)
+        assert page[0] == 2 and page[128 * D * 2 // 8] == 1 and page.sum() == 3

@@ -269,3 +269,29 @@ def test_symmetric_quantizer_bounds(bits):
     # the entry of largest magnitude is reproduced exactly
     i = np.unravel_index(np.abs(A).argmax(), A.shape)
     assert abs(Ah[i] - A[i]) < 1e-12
+
+
+@pytest.mark.parametrize("bits", [1, 3, 6])
+def test_odd_widths_follow_the_same_formula(bits):
+    """1, 3 and 6 bits (Table 1's 3-bit column, Sec. 4.1's 1- and 6-bit settings): an integer ladder 0..qmax is
+    reproduced exactly, the error stays within half a step, and brute force over all code vectors of a tiny group
+    finds nothing better."""
+    qmax = 2 ** bits - 1
+    ladder = np.arange(qmax + 1, dtype=np.float32)[None]
+    c, s16, z16 = oq.quantize_groups(ladder, bits)
+    assert np.array_equal(c[0], np.arange(qmax + 1)) and oq.bits_to_f32(s16, "fp16")[0] == 1.0
+    rng = np.random.default_rng(bits)
+    x = rng.normal(size=(50, 32)).astype(np.float16).astype(np.float32)
+    c, s16, z16 = oq.quantize_groups(x, bits)
+    s = oq.bits_to_f32(s16, "fp16").astype(np.float64)
+    xh = oq.dequantize_groups_f64(c, s16, z16)
+    z_exact = oq.bits_to_f32(z16, "fp16") == x.min(axis=1)
+    assert c.max() <= qmax and np.all(np.abs(x - xh)[z_exact] <= (0.5 * s[:, None] * (1 + 1e-3) * np.ones_like(xh))[z_exact])
+    if bits <= 3:
+        import itertools
+        g = x[0, :3][None]
+        c3, s3, z3 = oq.quantize_groups(g, bits)
+        sc = float(oq.bits_to_f32(s3, "fp16")[0]); z = float(oq.bits_to_f32(z3, "fp16")[0])
+        best = min(sum((g[0, i] - (z + sc * cv[i])) ** 2 for i in range(3)) for cv in itertools.product(range(qmax + 1), repeat=3))
+        mine = sum((g[0, i] - (z + sc * int(c3[0, i]))) ** 2 for i in range(3))
+        assert mine <= best * (1 + 1e-9) + 1e-18
