@@ -44,6 +44,12 @@
  *     byte = block*(4*D*b) + mw*512 + (4*g + t)*16 + 4*(2*rh + kh) + j,  bit = b*f
  *     (the bytes of a word are tokens 2t, 2t+8, 2t+1, 2t+9 of one half of the block).
  *   b = 16: rows [token][D] of the input's 16-bit patterns, no meta.
+ *   b in {1, 3, 6} (Table 1's 3-bit column; Sec. 4.1's 1- and 6-bit settings): bit planes.  A 3-bit code is a
+ *     2-bit plane (code >> 1) followed by a 1-bit plane (code & 1), a 6-bit code a 4-bit plane (code >> 2)
+ *     followed by a 2-bit plane (code & 3), a 1-bit code one 1-bit plane; every plane is a code region of its
+ *     own width laid out as above, the high plane first (the region still holds 128*D*b/8 bytes).  Widths 1 and
+ *     3 need head_dim 128; plane widths are token-wise only, are not combined with key rotation, and decode
+ *     serves them through the plain-ALU kernel.
  *   Meta: (scale fp16, zero fp16) per group; per-token axis [128][D/g],
  *     per-channel K [D].
  * pages: [batch][n_kv_heads][capacity_tokens/128][page_bytes].
@@ -90,7 +96,7 @@ typedef struct {
                               group size n_q_heads/n_kv_heads <= 8 */
   int32_t n_kv_heads;
   int32_t head_dim;        /* 64 or 128 */
-  int32_t kb, vb;          /* 2, 4, 8 quantized; 16 = unquantized passthrough */
+  int32_t kb, vb;          /* 1, 2, 3, 4, 6, 8 quantized; 16 = unquantized passthrough */
   int32_t gk, gv;          /* group size along head_dim: 32, 64 or 128, dividing head_dim (per-token axis) */
   int32_t k_axis;          /* 0: keys token-wise; 1: keys channel-wise over 128-token blocks (needs kb != 16) */
   int32_t in_dtype;        /* KVQ_FP16 or KVQ_BF16: type of k_new, v_new, q and of dequantize's outputs */

@@ -186,6 +186,38 @@ __device__ __forceinline__ void v_field_pos(int w, int j, int f, int b, int& tau
   d = 16 * (fpb * mw + f) + 8 * rh + gq;
 }
 
+// Code widths 1, 3 and 6 are stored as bit planes: a high plane of 2 (4) bits followed by a low plane of 1 (2)
+// bits, each a code region of its own width; 1-bit codes are one 1-bit plane.  planes_of: (high plane bits, low
+// plane bits or 0).
+__host__ __device__ __forceinline__ bool is_plane_width(int b) { return b == 1 || b == 3 || b == 6; }
+__host__ __device__ __forceinline__ void planes_of(int b, int& hi, int& lo) {
+  if (b == 3) { hi = 2; lo = 1; } else if (b == 6) { hi = 4; lo = 2; } else { hi = b; lo = 0; }
+}
+
+// Position of one plane's field of (token t, channel d) in a key (is_v = false) or value code region of a page:
+// byte offset of the 32-bit word (from the region's start) and the field's bit offset.  plane 0 = high plane.
+__device__ __forceinline__ void plane_pos(bool is_v, int t, int d, int D, int b, int plane, int& word_byte, int& bit,
+                                          int& pbits) {
+  int hi, lo;
+  planes_of(b, hi, lo);
+  pbits = plane == 0 ? hi : lo;
+  if (is_v) v_code_pos(t, d, D, pbits, word_byte, bit); else k_code_pos(t, d, D, pbits, word_byte, bit);
+  if (plane == 1) word_byte += kPageTokens * D * hi / 8;
+}
+
+// A code of any supported width from a code region.
+__device__ __forceinline__ uint32_t load_code_any(const uint8_t* region, bool is_v, int t, int d, int D, int b) {
+  int hi, lo, wb, bit, pb;
+  planes_of(b, hi, lo);
+  plane_pos(is_v, t, d, D, b, 0, wb, bit, pb);
+  uint32_t c = (*reinterpret_cast<const uint32_t*>(region + wb) >> bit) & ((1u << hi) - 1u);
+  if (lo) {
+    plane_pos(is_v, t, d, D, b, 1, wb, bit, pb);
+    c = (c << lo) | ((*reinterpret_cast<const uint32_t*>(region + wb) >> bit) & ((1u << lo) - 1u));
+  }
+  return c;
+}
+
 __device__ __forceinline__ uint32_t load_code(const uint8_t* region, int word_byte, int bit, int b) {
   uint32_t w = *reinterpret_cast<const uint32_t*>(region + word_byte);
   return (w >> bit) & ((1u << b) - 1u);

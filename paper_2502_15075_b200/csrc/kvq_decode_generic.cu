@@ -87,6 +87,13 @@ decode_generic_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float
             float kv = bits16_to_f32(row[d], dt);
             KVQ_FOR_HEADS(gh) acc[gh] = fmaf(sq[gh * D + d], kv, acc[gh]);
           }
+        } else if (is_plane_width(g.kb)) {
+          const uint32_t* meta = reinterpret_cast<const uint32_t*>(spage + g.k_meta_off);
+          for (int d = 0; d < D; ++d) {
+            uint32_t mm = meta[tp * (D / g.gk) + d / g.gk];
+            float kv = fmaf((float)load_code_any(spage, false, tp, d, D, g.kb), meta_scale(mm), meta_zero(mm));
+            KVQ_FOR_HEADS(gh) acc[gh] = fmaf(sq[gh * D + d], kv, acc[gh]);
+          }
         } else {
           const int bk = g.kb, nf = 32 / bk, wpr = D * bk / 32, wpc = wpr / 4;
           const uint32_t* roww = reinterpret_cast<const uint32_t*>(spage + (size_t)tp * (D * bk / 8));
@@ -131,10 +138,8 @@ decode_generic_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float
         if (g.vb == 16) {
           vv = bits16_to_f32(reinterpret_cast<const uint16_t*>(spage + g.v_codes_off)[tp * D + my_d], g.in_dtype);
         } else {
-          int wb, bit;
-          v_code_pos(tp, my_d, D, g.vb, wb, bit);
           uint32_t mm = vmeta[tp * (D / g.gv) + my_d / g.gv];
-          vv = fmaf((float)load_code(spage + g.v_codes_off, wb, bit, g.vb), meta_scale(mm), meta_zero(mm));
+          vv = fmaf((float)load_code_any(spage + g.v_codes_off, true, tp, my_d, D, g.vb), meta_scale(mm), meta_zero(mm));
         }
         KVQ_FOR_HEADS(gh) {
           float pr = sp[gh * kPageTokens + tp];

@@ -81,6 +81,20 @@ __device__ __forceinline__ void expand_values(const uint8_t* spage, const Geom& 
   }
 }
 
+// Expand a code region of a bit-plane width (1, 3, 6 bits) into tile[t][d], element by element.
+__device__ __forceinline__ void expand_planes(const uint8_t* spage, const Geom& g, bool is_v, uint16_t* tile, int tid) {
+  const int D = g.D, b = is_v ? g.vb : g.kb, gs = is_v ? g.gv : g.gk;
+  const uint8_t* region = spage + (is_v ? g.v_codes_off : 0);
+  const uint32_t* meta = reinterpret_cast<const uint32_t*>(spage + (is_v ? g.v_meta_off : g.k_meta_off));
+  const int lD = ilog2(D), lgs = ilog2(gs), ng = D >> lgs;
+  for (int idx = tid; idx < kPageTokens * D; idx += kThreads) {
+    const int t = idx >> lD, d = idx & (D - 1);
+    const uint32_t m = meta[t * ng + (d >> lgs)];
+    const float code = (float)load_code_any(region, is_v, t, d, D, b);
+    tile[t * (D + kTilePad) + d] = f32_to_bits16(fmaf(code, meta_scale(m), meta_zero(m)), g.in_dtype);
+  }
+}
+
 // Rotated keys: reconstruct rows [lo, hi) in fp32, rotate back (x = signs * H y / sqrt(D)) and store 16-bit rows.
 // A row is handled by D/8 consecutive lanes, lane l owning channels 8l..8l+7 (two code words of 4 channels each).
 template <int B, int D>
@@ -181,7 +195,8 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
     if (g.vb == 16) {
       store_rows(reinterpret_cast<const uint16_t*>(spage + g.v_codes_off), D, v_out + out_base, D, lo, hi_l, tid);
     } else {
-      if (g.vb == 2) expand_values<2>(spage, g, tile, tid);
+      if (is_plane_width(g.vb)) expand_planes(spage, g, true, tile, tid);
+      else if (g.vb == 2) expand_values<2>(spage, g, tile, tid);
       else if (g.vb == 4) expand_values<4>(spage, g, tile, tid);
       else expand_values<8>(spage, g, tile, tid);
       __syncthreads();
@@ -209,7 +224,8 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
       store_rows(reinterpret_cast<const uint16_t*>(spage), D, k_out + out_base, D, lo, hi_l, tid);
     } else {
       __syncthreads();          // the value tile has been copied out
-      if (g.kb == 2) expand_keys<2>(spage, g, tile, tid);
+      if (is_plane_width(g.kb)) expand_planes(spage, g, false, tile, tid);
+      else if (g.kb == 2) expand_keys<2>(spage, g, tile, tid);
       else if (g.kb == 4) expand_keys<4>(spage, g, tile, tid);
       else expand_keys<8>(spage, g, tile, tid);
       __syncthreads();

@@ -10,7 +10,7 @@ namespace kvq {
 
 namespace {
 
-bool is_bits(int b) { return b == 2 || b == 4 || b == 8 || b == 16; }
+bool is_bits(int b) { return b == 1 || b == 2 || b == 3 || b == 4 || b == 6 || b == 8 || b == 16; }
 bool is_group(int g) { return g == 32 || g == 64 || g == 128; }
 
 int make_geom(const kvq_config* cfg, Geom* out) {
@@ -22,6 +22,9 @@ int make_geom(const kvq_config* cfg, Geom* out) {
   if (cfg->k_axis != 0 && cfg->k_axis != 1) return KVQ_ERR_INVALID_ARG;
   if (!is_bits(cfg->kb) || !is_bits(cfg->vb)) return KVQ_ERR_UNSUPPORTED;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return KVQ_ERR_UNSUPPORTED;
+  // 1-bit planes (widths 1 and 3) fill whole bytes only at head_dim 128; plane widths are token-wise only
+  if (cfg->head_dim != 128 && (cfg->kb == 1 || cfg->kb == 3 || cfg->vb == 1 || cfg->vb == 3)) return KVQ_ERR_UNSUPPORTED;
+  if (cfg->k_axis == 1 && is_plane_width(cfg->kb)) return KVQ_ERR_UNSUPPORTED;
   if (cfg->n_q_heads / cfg->n_kv_heads > kMaxGroupHeads) return KVQ_ERR_UNSUPPORTED;
   if (cfg->kb != 16 && cfg->k_axis == 0 && (!is_group(cfg->gk) || cfg->head_dim % cfg->gk)) return KVQ_ERR_UNSUPPORTED;
   if (cfg->vb != 16 && (!is_group(cfg->gv) || cfg->head_dim % cfg->gv)) return KVQ_ERR_UNSUPPORTED;
@@ -58,7 +61,7 @@ int make_cache(const Geom& g, const kvq_cache* cache, CachePtrs* out) {
   out->seq_len = cache->seq_len;
   out->status = reinterpret_cast<uint32_t*>(cache->status);
   out->k_signs = cache->k_signs;
-  if (cache->k_signs && g.kb == 16) return KVQ_ERR_UNSUPPORTED;   // rotation applies to quantized keys only
+  if (cache->k_signs && (g.kb == 16 || is_plane_width(g.kb))) return KVQ_ERR_UNSUPPORTED;   // rotation: 2/4/8-bit keys only
   return KVQ_OK;
 }
 

@@ -480,6 +480,63 @@ __device__ __forceinline__ void quantize_task_fast(const uint16_t* __restrict__ 
   }
 }
 
+// Bit-plane widths (1, 3, 6 bits): a plain variant, one token row per warp step.  A lane holds 8 consecutive
+// channels of a row, groups reduce by butterflies, and every code's plane fields are cleared and set with atomic
+// AND / OR on the 32-bit words of the page (several lanes share a word).  Not tuned: these widths are served for
+// the paper's 1-, 3- and 6-bit settings, the 2/4/8-bit path above is the fast one.
+template <int D, int DTYPE>
+__device__ __forceinline__ void quantize_task_planes(const uint16_t* __restrict__ src, int64_t st, int gsz, int bits,
+                                                     bool is_v, int lo, int hi, int tp0, uint8_t* __restrict__ region,
+                                                     uint32_t* __restrict__ meta_out, int lane) {
+  constexpr int LPR = D / 8, RPW = 32 / LPR;           // lanes per row, rows per warp step
+  const int l = lane % LPR, r0 = lane / LPR;
+  const int lpg = gsz >> 3, ng = D / gsz;
+  const float qmax = (float)((1 << bits) - 1);
+  for (int base = lo; base < hi; base += RPW) {
+    const int tau = base + r0;                         // task-local token
+    const bool valid = tau < hi;
+    uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+    if (valid) raw = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + 8 * l);
+    const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
+    float x[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[2 * i] = bits16_to_f32((uint16_t)(rw[i] & 0xFFFF), DTYPE);
+      x[2 * i + 1] = bits16_to_f32((uint16_t)(rw[i] >> 16), DTYPE);
+    }
+    float mn = x[0], mx = x[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) { mn = fminf(mn, x[i]); mx = fmaxf(mx, x[i]); }
+#pragma unroll
+    for (int off = 1; off < 16; off <<= 1) {
+      if (off < lpg) {
+        mn = fminf(mn, __shfl_xor_sync(FULL, mn, off));
+        mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, off));
+      }
+    }
+    const GroupParams p = group_params(mn, mx, qmax);
+    if (!valid) continue;
+    const int t = tp0 + tau;                           // page-local token
+    if ((l & (lpg - 1)) == 0) meta_out[tau * ng + (8 * l) / gsz] = p.meta;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const uint32_t code = code_of(x[i], p, qmax);
+      int hb, lb;
+      planes_of(bits, hb, lb);
+#pragma unroll
+      for (int plane = 0; plane < 2; ++plane) {
+        if (plane == 1 && lb == 0) break;
+        int wb, bit, pb;
+        plane_pos(is_v, t, 8 * l + i, D, bits, plane, wb, bit, pb);
+        const uint32_t field = (plane == 0 ? (code >> lb) : code) & ((1u << pb) - 1u);
+        uint32_t* w = reinterpret_cast<uint32_t*>(region + wb);
+        atomicAnd(w, ~(((1u << pb) - 1u) << bit));
+        atomicOr(w, field << bit);
+      }
+    }
+  }
+}
+
 // 16-bit passthrough of one side of a task: rows [lo, hi) copied to the page as they are.
 __device__ __forceinline__ void copy_task_side(const uint16_t* __restrict__ src, int64_t st, int D, int lo, int hi,
                                                uint16_t* __restrict__ dst_rows, int lane) {
@@ -507,7 +564,7 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
   if (!append_fits(t0, t_new, g.capacity)) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int bits = is_v ? g.vb : g.kb;
-  const int TT = bits == 16 ? 32 : task_tokens(D, bits);
+  const int TT = (bits == 16 || is_plane_width(bits)) ? 32 : task_tokens(D, bits);
   const int first_task = t0 / TT;
   const int n_tasks = (t0 + t_new + TT - 1) / TT - first_task;
   const uint16_t* in = is_v ? v_new : k_new;
@@ -523,6 +580,11 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
     if (is_v) {
       if (bits == 16) {
         copy_task_side(src, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg + g.v_codes_off) + (size_t)tp0 * D, lane);
+        continue;
+      }
+      if (is_plane_width(bits)) {
+        quantize_task_planes<D, DTYPE>(src, st, gsz, bits, true, lo, hi, tp0, pg + g.v_codes_off,
+                                       reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / gsz), lane);
         continue;
       }
       uint8_t* vb = pg + g.v_codes_off + (size_t)(tp0 >> 5) * (4 * D * bits);
@@ -541,6 +603,11 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
     } else {
       if (bits == 16) {
         copy_task_side(src, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg) + (size_t)tp0 * D, lane);
+        continue;
+      }
+      if (is_plane_width(bits)) {
+        quantize_task_planes<D, DTYPE>(src, st, gsz, bits, false, lo, hi, tp0, pg,
+                                       reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / gsz), lane);
         continue;
       }
       uint8_t* kr = pg + (size_t)tp0 * (D * bits / 8);

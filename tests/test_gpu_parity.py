@@ -33,6 +33,13 @@ SMALL = {
     "14b-k4v2": (wl.SHAPED_14B, 2, 128 * 3 + 63, [128 * 3 + 63]),
     "14b-k8v2": (wl.SHAPED_14B.with_(kb=8), 1, 128 * 2 + 127, [100, 155, 128]),
     "70b": (wl.LLAMA_70B, 1, 1000, [1000]),
+    # bit-plane widths (Table 1's 3-bit column, Sec. 4.1's 1- and 6-bit settings), alone and mixed with 2/4/8 bits
+    "8b-k3v3": (wl.LLAMA_8B.with_(kb=3, vb=3), 2, 300, [171, 1, 128]),
+    "8b-k6v1": (wl.LLAMA_8B.with_(kb=6, vb=1, gk=32, gv=64), 1, 260, [260]),
+    "8b-k1v6": (wl.LLAMA_8B.with_(kb=1, vb=6), 1, 200, [77, 123]),
+    "8b-k3v2": (wl.LLAMA_8B.with_(kb=3, vb=2), 1, 300, [300]),
+    "8b-k4v3": (wl.LLAMA_8B.with_(kb=4, vb=3), 1, 300, [299, 1]),
+    "1b-k6v6": (wl.LLAMA_1B.with_(kb=6, vb=6), 2, 200, [200]),
 }
 
 
@@ -126,6 +133,30 @@ def test_ragged_sequences_and_empty_and_single_token(kvq):
     ko_ref = np.zeros((B, 2, cap, 128), np.uint16)
     oc.dequantize(ko_ref, np.zeros_like(ko_ref), 100, 300)
     assert np.array_equal(tl.bits_of(ko), ko_ref)
+
+
+def test_rewound_append_overwrites_bit_plane_codes(kvq):
+    """Appending again after seq_len was moved back replaces the codes (the plane fields are cleared, then set)."""
+    w = wl.LLAMA_8B.with_(n_kv_heads=2, n_q_heads=8, kb=3, vb=6)
+    k, v = wl.make_kv(w, tokens=100, batch=1)
+    k2, v2 = wl.make_kv(w, layer=3, tokens=100, batch=1)
+    cfg = tl.gpu_config_for(kvq, w, 1, 128)
+    gc = kvq.Cache(cfg)
+    kvq.kvq_quantize_append(cfg, gc, k.cuda(), v.cuda())
+    gc.seq_len.zero_()
+    kvq.kvq_quantize_append(cfg, gc, k2.cuda(), v2.cuda())
+    oc = tl.oracle_cache_for(w, 1, 128)
+    oc.append(tl.bits_of(k2), tl.bits_of(v2))
+    tl.assert_caches_equal(gc, oc)
+
+
+def test_odd_widths_that_do_not_fill_bytes_are_rejected(kvq):
+    for kb, vb, D in ((3, 2, 64), (4, 1, 64)):
+        with pytest.raises(kvq.KvqError) as e:
+            kvq.kvq_page_bytes(kvq.make_config(1, 8, 2, D, kb, vb, 64, 64, 0, "fp16", 128))
+        assert e.value.code == -2
+    with pytest.raises(kvq.KvqError):       # channel-wise keys keep to 2/4/8 bits
+        kvq.kvq_page_bytes(kvq.make_config(1, 8, 2, 128, 3, 2, 128, 128, 1, "bf16", 128))
 
 
 def test_capacity_overflow_sets_status_and_skips_sequence(kvq):

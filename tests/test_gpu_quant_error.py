@@ -29,6 +29,8 @@ CASES = {
     "14b-tokenwise": (wl.SHAPED_14B.with_(k_axis=0), 1, 257),
     "70b": (wl.LLAMA_70B, 1, 400),
     "16bit-keys": (wl.LLAMA_8B.with_(kb=16), 1, 100),
+    "8b-k3v3": (wl.LLAMA_8B.with_(kb=3, vb=3), 1, 200),        # Table 1's middle column
+    "8b-k6v1": (wl.LLAMA_8B.with_(kb=6, vb=1), 1, 200),
 }
 
 

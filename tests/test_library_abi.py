@@ -61,7 +61,7 @@ def test_k4v2_page_is_104_bytes_per_token(kvq):
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(head_dim=96), -2), (dict(kb=3), -2), (dict(vb=5), -2), (dict(gk=16), -2), (dict(gv=256), -2),
+    (dict(head_dim=96), -2), (dict(kb=7), -2), (dict(vb=5), -2), (dict(gk=16), -2), (dict(gv=256), -2),
     (dict(capacity_tokens=100), -1), (dict(n_q_heads=9), -1), (dict(batch=0), -1), (dict(in_dtype=7), -1),
     (dict(k_axis=1, kb=16), -2), (dict(n_q_heads=32, n_kv_heads=2), -2), (dict(k_axis=2), -1)])
 def test_invalid_configs_are_rejected_on_the_host(kvq, kw, code):
