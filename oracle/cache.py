@@ -8,6 +8,11 @@ tests can compare bytes and values one by one:
   an fp16 residual tail (Sec. 4.1: recent tokens stay in full precision and are
   flushed periodically); when the block is complete it is quantized with one
   group per channel and written to its page.
+* residual window (Sec. 4.1: "a 64-token residual buffer, which stores the most recent tokens in full precision
+  before being periodically flushed"; token-wise keys only): with residual = R > 0 the newest seq_len mod R tokens
+  of K and V stay as their 16-bit inputs in a ring of R slots (token t in slot t mod R); whenever R of them are
+  complete they are quantized as a block and move to the pages.  Reading: the flush is block-aligned, so the
+  window holds 0 .. R-1 tokens.
 * dequantize: xhat = fmaf(code, scale, zero) rounded to the 16-bit input type.
 * decode: fp64 attention (App. A.1) over z + s*code exactly, the tail as stored.
 """
@@ -22,7 +27,8 @@ ERR_CAPACITY_BIT = 1
 
 
 class OracleCache:
-    def __init__(self, batch, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, dtype, capacity_tokens, k_signs=None):
+    def __init__(self, batch, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, dtype, capacity_tokens, k_signs=None,
+                 residual=0):
         """k_signs: None, or +-1 per channel: keys are rotated by the randomized Hadamard transform
         y = H (signs * x) / sqrt(D) before quantization (Sec. 4.4, key-only rotation); queries get the same
         rotation at decode time and dequantize rotates back."""
@@ -38,15 +44,53 @@ class OracleCache:
         self.k_tail = np.zeros((batch, n_kv_heads, PAGE_TOKENS, head_dim), np.uint16) if k_axis == 1 else None
         self.seq_len = np.zeros(batch, np.int32)
         self.status = 0
+        assert residual == 0 or (k_axis == 0 and residual > 0)
+        self.R = residual
+        # [B, H, R, 2, D]: 16-bit patterns of (key row, value row) of the tokens not yet quantized
+        self.kv_win = np.zeros((batch, n_kv_heads, residual, 2, head_dim), np.uint16) if residual else None
+
+    def flushed(self, b) -> int:
+        """Tokens of sequence b that live in the pages (the rest is in the residual window)."""
+        n = int(self.seq_len[b])
+        return n if not self.R else (n // self.R) * self.R
 
     # ------------------------------------------------------------------ append
     def append(self, k_bits: np.ndarray, v_bits: np.ndarray):
         """k_bits, v_bits: uint16 [B, Hkv, t_new, D] patterns of the input dtype."""
-        L = self.L
-        t_new = k_bits.shape[2]
+        if self.R:
+            return self._append_residual(k_bits, v_bits)
+        return self._append_at(k_bits, v_bits, None)
+
+    def _append_residual(self, k_bits, v_bits):
+        R, t_new = self.R, k_bits.shape[2]
         for b in range(self.B):
             t0 = int(self.seq_len[b])
             if t0 + t_new > self.capacity:
+                self.status |= ERR_CAPACITY_BIT
+                continue
+            f0, f1 = (t0 // R) * R, ((t0 + t_new) // R) * R
+            if f1 > f0:
+                # tokens f0 .. f1-1 are complete blocks: the old window's tokens followed by new ones
+                kq = np.concatenate([self.kv_win[b, :, :t0 - f0, 0], k_bits[b, :, :f1 - t0]], axis=1)
+                vq = np.concatenate([self.kv_win[b, :, :t0 - f0, 1], v_bits[b, :, :f1 - t0]], axis=1)
+                self._append_at(kq[None], vq[None], (b, f0))
+            for t in range(max(t0, f1), t0 + t_new):
+                self.kv_win[b, :, t % R, 0] = k_bits[b, :, t - t0]
+                self.kv_win[b, :, t % R, 1] = v_bits[b, :, t - t0]
+            self.seq_len[b] = t0 + t_new
+
+    def _append_at(self, k_bits, v_bits, where):
+        """Quantize and store tokens; where = None: every sequence at its seq_len (which is advanced), or
+        (b, position): one sequence's tokens at a given position (seq_len untouched)."""
+        L = self.L
+        t_new = k_bits.shape[2]
+        for b in (range(self.B) if where is None else [where[0]]):
+            t0 = int(self.seq_len[b]) if where is None else where[1]
+            if where is not None:
+                k_bits_b, v_bits_b = k_bits[0], v_bits[0]
+            else:
+                k_bits_b, v_bits_b = k_bits[b], v_bits[b]
+            if where is None and t0 + t_new > self.capacity:
                 self.status |= ERR_CAPACITY_BIT
                 continue
             for h in range(self.H):
@@ -57,8 +101,8 @@ class OracleCache:
                     n = min(PAGE_TOKENS - slot, t_new - done)
                     slots = np.arange(slot, slot + n)
                     page = self.pages[b, h, p]
-                    kx = k_bits[b, h, done:done + n]
-                    vx = v_bits[b, h, done:done + n]
+                    kx = k_bits_b[h, done:done + n]
+                    vx = v_bits_b[h, done:done + n]
                     # values: always token-wise
                     if L.vb == 16:
                         layout.put_v_codes(page, L, slots, vx)
@@ -90,7 +134,8 @@ class OracleCache:
                             layout.put_k_codes(page, L, np.arange(PAGE_TOKENS), c)
                             layout.put_k_meta_channels(page, L, s, z)
                     done += n
-            self.seq_len[b] = t0 + t_new
+            if where is None:
+                self.seq_len[b] = t0 + t_new
 
     # ------------------------------------------------------- page -> values
     def _page_values(self, b, h, p, n_valid, exact: bool):
@@ -126,6 +171,12 @@ class OracleCache:
             V = V.astype(np.float64)
         return K[:n_valid], V[:n_valid]
 
+    def _window_values(self, b, h, t_lo, t_hi):
+        """fp32 values (K, V) of the window tokens t_lo <= t < t_hi of stream (b, h): the 16-bit inputs, exactly."""
+        slots = np.arange(t_lo, t_hi) % self.R
+        return (quantizer.bits_to_f32(self.kv_win[b, h, slots, 0], self.dtype),
+                quantizer.bits_to_f32(self.kv_win[b, h, slots, 1], self.dtype))
+
     def values_f64(self):
         """K-hat, V-hat as fp64 [B, Hkv, capacity, D]; zeros beyond seq_len."""
         K = np.zeros((self.B, self.H, self.capacity, self.D), np.float64)
@@ -138,6 +189,8 @@ class OracleCache:
                     k, v = self._page_values(b, h, p, nv, exact=True)
                     K[b, h, p * PAGE_TOKENS: p * PAGE_TOKENS + nv] = k
                     V[b, h, p * PAGE_TOKENS: p * PAGE_TOKENS + nv] = v
+                if self.R and self.flushed(b) < n:
+                    K[b, h, self.flushed(b):n], V[b, h, self.flushed(b):n] = self._window_values(b, h, self.flushed(b), n)
         return K, V
 
     # -------------------------------------------------------------- dequantize
@@ -157,6 +210,12 @@ class OracleCache:
                     ks = k[sl] if self.k_signs is None else quantizer.unrotate_f32(k[sl], self.k_signs)
                     k_out[b, h, lo_t:hi_t] = quantizer.f32_to_bits(ks, self.dtype)
                     v_out[b, h, lo_t:hi_t] = quantizer.f32_to_bits(v[sl], self.dtype)
+                if self.R:                       # tokens still in the residual window come back as they went in
+                    w_lo, w_hi = max(t_begin, self.flushed(b)), hi
+                    if w_lo < w_hi:
+                        slots = np.arange(w_lo, w_hi) % self.R
+                        k_out[b, h, w_lo:w_hi] = self.kv_win[b, h, slots, 0]
+                        v_out[b, h, w_lo:w_hi] = self.kv_win[b, h, slots, 1]
 
     # ------------------------------------------------------------------ decode
     def decode(self, q_bits: np.ndarray, scale=None) -> np.ndarray:
@@ -195,5 +254,8 @@ class OracleCache:
                 Vs.append(v)
             K = np.concatenate(Ks) if Ks else np.zeros((0, self.D))
             V = np.concatenate(Vs) if Vs else np.zeros((0, self.D))
+            if self.R and self.flushed(b) < n:
+                kw, vw = self._window_values(b, h, self.flushed(b), n)
+                K[self.flushed(b):n], V[self.flushed(b):n] = kw, vw
             res[(b, h)] = np.stack([attention.attend_one(q[b, h * G + j], K, V, sc) for j in range(G)])
         return res

@@ -386,3 +386,44 @@ def test_bit_plane_widths_tile_the_region_and_keep_their_planes_apart(D, b):
         codes = np.zeros((1, D), np.uint16); codes[0, 0] = 5
         ol.put_k_codes(page, L, np.array([0]), codes)
         assert page[0] == 2 and page[128 * D * 2 // 8] == 1 and page.sum() == 3
+
+
+def test_residual_window_keeps_recent_tokens_exact_and_flushes_whole_blocks():
+    """Sec. 4.1's residual buffer: with R = 64 the newest seq_len mod 64 tokens of K and V are the 16-bit inputs
+    themselves; the tokens behind them carry exactly the codes a cache without a window would have; any chunking
+    of the appends gives the same state."""
+    w = wl.LLAMA_8B.with_(n_kv_heads=2, n_q_heads=8)
+    T, R = 64 * 3 + 21, 64
+    k, v = wl.make_kv(w, tokens=T, batch=2)
+    kb_, vb_ = bits_of(k), bits_of(v)
+    def build(chunks, residual):
+        oc = OracleCache(2, 2, 128, 4, 2, 128, 128, 0, "bf16", 256, residual=residual)
+        t = 0
+        for n in chunks:
+            oc.append(kb_[:, :, t:t + n], vb_[:, :, t:t + n]); t += n
+        return oc
+    a = build([T], R)
+    for chunks in ([1] * T, [63, 1, 1, 64, 70, T - 199], [130, T - 130]):
+        c = build(chunks, R)
+        assert np.array_equal(a.pages, c.pages) and np.array_equal(a.seq_len, c.seq_len)
+        n = T % R
+        slots = np.arange(T - n, T) % R
+        assert np.array_equal(a.kv_win[:, :, slots], c.kv_win[:, :, slots])
+    plain = build([192], 0)                                     # the flushed part = a cache of the first 192 tokens
+    assert np.array_equal(a.pages[:, :, :1], plain.pages[:, :, :1])
+    assert np.array_equal(a.pages[:, :, 1, : ], plain.pages[:, :, 1])
+    K, V = a.values_f64()
+    assert np.array_equal(K[:, :, 192:T], oq.bits_to_f32(kb_[:, :, 192:T], "bf16").astype(np.float64))
+    assert np.array_equal(V[:, :, 192:T], oq.bits_to_f32(vb_[:, :, 192:T], "bf16").astype(np.float64))
+    Kp, _ = plain.values_f64()
+    assert np.array_equal(K[:, :, :192], Kp[:, :, :192])
+    # dequantize returns the window tokens bit for bit
+    ko = np.zeros((2, 2, 256, 128), np.uint16); vo = np.zeros_like(ko)
+    a.dequantize(ko, vo, 0, 256)
+    assert np.array_equal(ko[:, :, 192:T], kb_[:, :, 192:T]) and np.array_equal(vo[:, :, 192:T], vb_[:, :, 192:T])
+    # attention with a window is closer to exact attention than without (recent tokens carry no error)
+    q = wl.make_q(w, batch=2)
+    exact = oa.decode_attention(q.double().numpy(), k.double().numpy(), v.double().numpy(), [T, T])
+    e_win = np.linalg.norm(a.decode(bits_of(q)) - exact)
+    e_plain = np.linalg.norm(build([T], 0).decode(bits_of(q)) - exact)
+    assert e_win < e_plain
