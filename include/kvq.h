@@ -101,6 +101,9 @@ typedef struct {
   int32_t k_axis;          /* 0: keys token-wise; 1: keys channel-wise over 128-token blocks (needs kb != 16) */
   int32_t in_dtype;        /* KVQ_FP16 or KVQ_BF16: type of k_new, v_new, q and of dequantize's outputs */
   int32_t capacity_tokens; /* per sequence; multiple of 128 */
+  int32_t residual_tokens; /* 0, or R = 64 or 128: the newest seq_len % R tokens of K and V stay in 16 bits in
+                              kvq_cache.kv_win and are quantized as a block when R of them are complete (Sec. 4.1:
+                              "a 64-token residual buffer ... periodically flushed").  Needs k_axis == 0. */
 } kvq_config;
 
 typedef struct {
@@ -114,6 +117,8 @@ typedef struct {
                             same rotation to q, dequantize rotates back.  Needs kb != 16.  The transform is
                             computed in fp32 with butterfly stages h = 1, 2, 4, ... in this order, (a, b) ->
                             (a + b, a - b), then one multiplication by (float)(1/sqrt(head_dim)). */
+  void* kv_win;     /* device, in_dtype [batch][n_kv_heads][residual_tokens][2][head_dim] (key row, value row of
+                       token t in slot t % residual_tokens), 16-byte aligned; NULL when residual_tokens == 0 */
 } kvq_cache;        /* one per layer.  The caller zeroes seq_len and status for a fresh cache;
                        pages must be zero-filled once before the first append. */
 
@@ -122,6 +127,7 @@ typedef struct {
 int kvq_layout_version(void);
 int kvq_page_bytes(const kvq_config* cfg, size_t* out);
 int kvq_cache_bytes(const kvq_config* cfg, size_t* pages_bytes, size_t* k_tail_bytes);
+int kvq_window_bytes(const kvq_config* cfg, size_t* kv_win_bytes);   /* 0 when residual_tokens == 0 */
 /* Scratch needed by kvq_decode_attention for its split partial results. */
 int kvq_workspace_bytes(const kvq_config* cfg, size_t* out);
 

@@ -172,10 +172,14 @@ class OracleCache:
         return K[:n_valid], V[:n_valid]
 
     def _window_values(self, b, h, t_lo, t_hi):
-        """fp32 values (K, V) of the window tokens t_lo <= t < t_hi of stream (b, h): the 16-bit inputs, exactly."""
+        """Values (K, V) of the window tokens t_lo <= t < t_hi of stream (b, h) for attention: the 16-bit inputs,
+        exactly.  With rotated keys the queries are rotated too, so the window's keys are given the same (exact,
+        fp64) rotation: (H k) . (H q) = k . q."""
         slots = np.arange(t_lo, t_hi) % self.R
-        return (quantizer.bits_to_f32(self.kv_win[b, h, slots, 0], self.dtype),
-                quantizer.bits_to_f32(self.kv_win[b, h, slots, 1], self.dtype))
+        kw = quantizer.bits_to_f32(self.kv_win[b, h, slots, 0], self.dtype).astype(np.float64)
+        if self.k_signs is not None:
+            kw = quantizer.hadamard_rotate_f64(kw, self.k_signs)
+        return kw, quantizer.bits_to_f32(self.kv_win[b, h, slots, 1], self.dtype)
 
     def values_f64(self):
         """K-hat, V-hat as fp64 [B, Hkv, capacity, D]; zeros beyond seq_len."""

@@ -24,6 +24,7 @@ struct Geom {
   int v_codes_off, v_codes_bytes, v_meta_off, v_meta_bytes;
   int page_bytes;
   int rows;          // query rows per head of a decode call (1 = a plain decode step)
+  int R;             // residual window: the newest seq_len % R tokens are not in the pages (0: no window)
 };
 
 // Pointers of one cache (device memory).
@@ -33,11 +34,18 @@ struct CachePtrs {
   int32_t* seq_len;
   uint32_t* status;
   const int8_t* k_signs;   // NULL: keys are not rotated
+  uint16_t* kv_win;        // residual window [B][Hkv][R][2][D], or NULL
 };
 
 // Sequence length as the kernels use it: a corrupt value can never index outside the cache.
 __device__ __forceinline__ int clamped_len(const int32_t* seq_len, int b, int capacity) {
   return min(max(seq_len[b], 0), capacity);
+}
+
+// Tokens of a sequence that live in the pages: all of them, or whole blocks of R when a residual window is kept.
+__device__ __forceinline__ int paged_len(const int32_t* seq_len, int b, int capacity, int R) {
+  const int n = clamped_len(seq_len, b, capacity);
+  return R ? (n / R) * R : n;
 }
 
 // ---------------------------------------------------------------- conversions

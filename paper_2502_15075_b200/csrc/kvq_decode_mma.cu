@@ -23,6 +23,7 @@ int flat_slot_cap(const Geom& g) {
   const int streams = g.B * g.Hkv;
   int s = (2 * kFlatGrid + streams - 1) / streams + 2;
   if (s > g.n_pages + 1) s = g.n_pages + 1;
+  if (g.R) s += 1;                           // one more slot per stream: the partial of the residual window
   return s;
 }
 
@@ -72,6 +73,11 @@ int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* ou
                       float* ws, const DecodeDebug& dbg, cudaStream_t stream) {
   const int s_cap = flat_slot_cap(g);
   int grid = 0;
+  if (g.R) {      // the residual window first: its partial (or, for sequences without pages, the output) is ready
+                  // when the main kernel's last finisher merges
+    int rc = launch_decode_window(g, c, q, out, out_dtype, c1, ws, s_cap, stream);
+    if (rc != KVQ_OK) return rc;
+  }
   return pick(g, c, q, c1, ws, s_cap, out, out_dtype, dbg, stream, false, &grid);
 }
 

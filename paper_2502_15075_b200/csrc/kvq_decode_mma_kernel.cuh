@@ -182,7 +182,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   if (tid_ == 0) { sPref[0] = 0; sMisc[0] = 0; sMisc[1] = 0; }
   __syncthreads();
   for (int b = tid_; b < B; b += blockDim.x) {
-    int pages = (clamped_len(c.seq_len, b, g.capacity) + kPageTokens - 1) >> 7;
+    int pages = (paged_len(c.seq_len, b, g.capacity, g.R) + kPageTokens - 1) >> 7;
     sPref[b + 1] = pages * Hkv;
     atomicMax(&sMisc[0], pages);
   }
@@ -208,8 +208,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  // an empty sequence has no page and therefore no CTA of its own: its output rows are zero
-  for (int bb = blockIdx.x; bb < B; bb += gridDim.x) {
+  // an empty sequence has no page and therefore no CTA of its own: its output rows are zero (with a residual
+  // window the window kernel, which runs first, has written the rows of sequences without pages)
+  for (int bb = blockIdx.x; bb < B && g.R == 0; bb += gridDim.x) {
     if (sPref[bb + 1] == sPref[bb]) {
       for (int i = tid_; i < g.rows * g.Hq * D; i += blockDim.x) {
         const size_t oi = (size_t)bb * g.rows * g.Hq * D + i;
@@ -218,7 +219,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       }
     }
   }
-  const FlatPlan plan = make_plan(sPref[B], sMisc[0], gridDim.x, s_cap);
+  const int s_plan = s_cap - (g.R ? 1 : 0);       // the last partial slot of a stream belongs to its residual window
+  const FlatPlan plan = make_plan(sPref[B], sMisc[0], gridDim.x, s_plan);
   if (plan.N == 0 || (int)blockIdx.x >= plan.c_eff) return;
   unsigned long long* counts = reinterpret_cast<unsigned long long*>(ws + tag_offset_floats(B * Hkv, s_cap, G, D));
   const long long x_lo = plan.lo(blockIdx.x), x_hi = plan.lo(blockIdx.x + 1);
@@ -342,11 +344,13 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
   for (long long x = x_lo; x < x_hi;) {
     const int seg_pages = (int)min((long long)(pages_b - page), x_hi - x);
-    const int n_tok = clamped_len(c.seq_len, b, g.capacity);
+    const int n_all = clamped_len(c.seq_len, b, g.capacity);      // tokens of the sequence
+    const int n_tok = g.R ? (n_all / g.R) * g.R : n_all;          // ... of which in the pages
+    const bool has_win = n_all > n_tok;                           // the window kernel left a partial in slot s_cap - 1
     const int stream = b * Hkv + h;
     int limh[NH];                          // tokens the lane's heads may attend to (causal limit of their query row)
 #pragma unroll
-    for (int nh = 0; nh < NH; ++nh) limh[nh] = n_tok - (g.rows - 1 - min((tid + 4 * nh) / Gq, g.rows - 1));
+    for (int nh = 0; nh < NH; ++nh) limh[nh] = n_all - (g.rows - 1 - min((tid + 4 * nh) / Gq, g.rows - 1));
 
     // ---- segment start: q operands, group sums and a clean state for this stream's heads
     {
@@ -767,7 +771,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         };
 
         // the masked variant also serves the last tokens when several causal query rows see different prefixes
-        if (nv - wq * 32 >= 32 && (page + pp) * kPageTokens + wq * 32 + 32 <= n_tok - (g.rows - 1)) do_block(std::false_type{});
+        if (nv - wq * 32 >= 32 && (page + pp) * kPageTokens + wq * 32 + 32 <= n_all - (g.rows - 1)) do_block(std::false_type{});
         else do_block(std::true_type{});
       }
       __syncwarp();
@@ -807,7 +811,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       const int c_first = plan.cta_of(xs);
       const int slot = (int)blockIdx.x - c_first;
       const int n_part = plan.cta_of(xs + pages_b - 1) - c_first + 1;        // partials of this stream
-      if (slot >= 0 && slot < s_cap) {
+      if (slot >= 0 && slot < s_plan) {
         for (int idx = tid_; idx < G * D; idx += NCONS) {
           const int head = idx / D, d = idx % D;
           float mstar = -INFINITY;
@@ -821,7 +825,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             o = fmaf(f, sMaster[(w * NHEADS + head) * MSTRIDE + d], o);
             lsum = fmaf(f, sML[(w * NHEADS + head) * 2 + 1], lsum);
           }
-          if (n_part == 1) {
+          if (n_part == 1 && !has_win) {
             const float r = lsum > 0.f ? o / lsum : 0.f;
             const size_t oi = (((size_t)b * g.rows + head / Gq) * g.Hq + (size_t)h * Gq + head % Gq) * D + d;
             if (out_dtype == KVQ_FP32) static_cast<float*>(out)[oi] = r;
@@ -832,7 +836,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             dst[2 + d] = o;
           }
         }
-        if (n_part > 1) {
+        if (n_part > 1 || has_win) {
           __threadfence();
           named_bar_sync(1, NCONS);
           if (tid_ == 0) *n_published = (int)tagged_count(counts + stream, id40);
@@ -844,12 +848,14 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
               const float* base = ws + (((size_t)stream * s_cap) * G + head) * (D + 2);
               const size_t slot_stride = (size_t)G * (D + 2);
               float mstar = -INFINITY, num = 0.f, den = 0.f;
-              for (int j0 = 0; j0 < n_part; j0 += 4) {
+              const int n_merge = n_part + (has_win ? 1 : 0);
+              for (int j0 = 0; j0 < n_merge; j0 += 4) {
                 float mj[4], lj[4], oj[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {                   // issue the loads of a batch before using any
-                  const bool on = j0 + u < n_part;
-                  const float* pj = base + (size_t)(on ? j0 + u : 0) * slot_stride;
+                  const bool on = j0 + u < n_merge;
+                  const int sj = (j0 + u < n_part) ? j0 + u : s_cap - 1;      // the window's partial comes last
+                  const float* pj = base + (size_t)(on ? sj : 0) * slot_stride;
                   mj[u] = on ? __ldcg(pj) : -INFINITY;
                   lj[u] = on ? __ldcg(pj + 1) : 0.f;
                   oj[u] = on ? __ldcg(pj + 2 + d) : 0.f;

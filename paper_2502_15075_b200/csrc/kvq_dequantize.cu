@@ -173,7 +173,7 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
   uint16_t* tile = reinterpret_cast<uint16_t*>(smem + ((g.page_bytes + 15) & ~15));   // [128][D]
   const int bh = blockIdx.y;
   const int b = bh / g.Hkv;
-  const int n = clamped_len(c.seq_len, b, g.capacity);
+  const int n = paged_len(c.seq_len, b, g.capacity, g.R);      // tokens behind a residual window are in the pages
   const int hi = min(t_end, n);
   const int page = page0 + blockIdx.x;
   const int lo_t = max(t_begin, page * kPageTokens), hi_t = min(hi, page * kPageTokens + kPageTokens);
@@ -234,6 +234,22 @@ dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out,
   }
 }
 
+// Tokens still in the residual window are the 16-bit inputs themselves: copy their rows out.
+__global__ void __launch_bounds__(kThreads)
+window_dequant_kernel(Geom g, CachePtrs c, uint16_t* k_out, uint16_t* v_out, int t_begin, int t_end) {
+  const int bh = blockIdx.x, b = bh / g.Hkv;
+  const int D = g.D, R = g.R, vpr = D / 8;
+  const int n = clamped_len(c.seq_len, b, g.capacity);
+  const int lo = max(t_begin, (n / R) * R), hi = min(t_end, n);
+  for (int idx = threadIdx.x; idx < (hi - lo) * 2 * vpr; idx += kThreads) {
+    const int t = lo + idx / (2 * vpr), side = (idx / vpr) & 1, v = idx % vpr;
+    uint16_t* dst = side ? v_out : k_out;
+    if (!dst) continue;
+    reinterpret_cast<uint4*>(dst + ((size_t)bh * g.capacity + t) * D)[v] =
+        reinterpret_cast<const uint4*>(c.kv_win + (((size_t)bh * R + (t % R)) * 2 + side) * D)[v];
+  }
+}
+
 }  // namespace
 
 int launch_dequantize(const Geom& g, const CachePtrs& c, void* k_out, void* v_out, int t_begin, int t_end,
@@ -247,6 +263,9 @@ int launch_dequantize(const Geom& g, const CachePtrs& c, void* k_out, void* v_ou
   dim3 grid(page1 - page0, g.B * g.Hkv, 2);
   dequant_kernel<<<grid, kThreads, smem, stream>>>(g, c, static_cast<uint16_t*>(k_out),
                                                    static_cast<uint16_t*>(v_out), t_begin, t_end, page0);
+  if (g.R)
+    window_dequant_kernel<<<g.B * g.Hkv, kThreads, 0, stream>>>(g, c, static_cast<uint16_t*>(k_out),
+                                                                static_cast<uint16_t*>(v_out), t_begin, t_end);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
 

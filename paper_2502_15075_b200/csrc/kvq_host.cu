@@ -46,6 +46,9 @@ int make_geom(const kvq_config* cfg, Geom* out) {
   g.v_meta_bytes = (g.vb == 16) ? 0 : kPageTokens * (g.D / g.gv) * 4;
   g.page_bytes = g.v_meta_off + g.v_meta_bytes;
   g.rows = 1;
+  g.R = cfg->residual_tokens;
+  if (g.R != 0 && g.R != 64 && g.R != 128) return KVQ_ERR_UNSUPPORTED;
+  if (g.R != 0 && g.k_axis != 0) return KVQ_ERR_UNSUPPORTED;
   *out = g;
   return KVQ_OK;
 }
@@ -61,6 +64,9 @@ int make_cache(const Geom& g, const kvq_cache* cache, CachePtrs* out) {
   out->seq_len = cache->seq_len;
   out->status = reinterpret_cast<uint32_t*>(cache->status);
   out->k_signs = cache->k_signs;
+  out->kv_win = static_cast<uint16_t*>(cache->kv_win);
+  if (g.R != 0 && !cache->kv_win) return KVQ_ERR_INVALID_ARG;
+  if (!aligned16(cache->kv_win)) return KVQ_ERR_MISALIGNED;
   if (cache->k_signs && (g.kb == 16 || is_plane_width(g.kb))) return KVQ_ERR_UNSUPPORTED;   // rotation: 2/4/8-bit keys only
   return KVQ_OK;
 }
@@ -90,6 +96,7 @@ int launch_decode_attention(const Geom& g, const CachePtrs& c, const void* q, vo
   const float scale_log2e = scale * 1.4426950408889634f;
   float* ws = static_cast<float*>(workspace);
   const bool use_mma = decode_mma_supported(g) && !dbg.force_generic;
+  if (g.R != 0 && !use_mma) return KVQ_ERR_UNSUPPORTED;      // only the tensor-core path merges the residual window
   if (use_mma) return launch_decode_mma(g, c, q, out, out_dtype, scale_log2e, ws, dbg, stream);
   const int n_split = decode_num_splits(g);
   int rc = launch_decode_generic(g, c, q, scale_log2e, ws, n_split, stream);
@@ -120,6 +127,15 @@ int kvq_cache_bytes(const kvq_config* cfg, size_t* pages_bytes, size_t* k_tail_b
   if (rc != KVQ_OK) return rc;
   if (pages_bytes) *pages_bytes = (size_t)g.B * g.Hkv * g.n_pages * g.page_bytes;
   if (k_tail_bytes) *k_tail_bytes = g.k_axis == 1 ? (size_t)g.B * g.Hkv * kPageTokens * g.D * 2 : 0;
+  return KVQ_OK;
+}
+
+int kvq_window_bytes(const kvq_config* cfg, size_t* kv_win_bytes) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != KVQ_OK) return rc;
+  if (!kv_win_bytes) return KVQ_ERR_INVALID_ARG;
+  *kv_win_bytes = (size_t)g.B * g.Hkv * g.R * 2 * g.D * 2;
   return KVQ_OK;
 }
 

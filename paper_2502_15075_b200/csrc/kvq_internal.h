@@ -40,6 +40,9 @@ namespace kvq {
 // fast (tensor-core) decode path: flat split over the grid
 bool decode_mma_supported(const Geom& g);
 size_t flat_workspace_bytes(const Geom& g);
+// attention over the residual window's tokens: one partial per stream in slot s_cap - 1 of the flat workspace
+int launch_decode_window(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
+                         float scale_log2e, float* ws, int s_cap, cudaStream_t stream);
 int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
                       float scale_log2e, float* ws, const DecodeDebug& dbg, cudaStream_t stream);
 }  // namespace kvq

@@ -22,6 +22,19 @@ constexpr int kWarps = kThreads / 32;
 constexpr uint32_t FULL = 0xffffffffu;
 constexpr float kRoundMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to nearest-even at integer precision
 
+// Where the 16-bit row of a task-local token comes from: the call's input, or - for the first n_win tokens of a task
+// when a residual window is kept - the window's ring of rows (token t in slot t % R; a task never wraps the ring).
+struct RowSrc {
+  const uint16_t* in;     // row of task-local token 0 in the input (never dereferenced before the first new token)
+  int64_t st;             // input row stride in elements
+  const uint16_t* win;    // window row of task-local token 0 (this side), or nullptr
+  int n_win;              // task-local tokens [0, n_win) are read from the window
+  int wst;                // window row stride in elements (2 D: key row, value row)
+  __device__ __forceinline__ const uint16_t* row(int tau) const {
+    return (tau < n_win) ? win + (size_t)tau * wst : in + (int64_t)tau * st;
+  }
+};
+
 // Tokens handled by one warp task: 32, or 64 where 32 tokens would leave a lane fewer than the four tokens
 // that make up a word of value codes.
 __host__ __device__ constexpr int task_tokens(int D, int bits) { return (D == 64 && bits == 2) ? 64 : 32; }
@@ -45,7 +58,7 @@ __device__ __forceinline__ uint32_t pack_bytes(float b0, float b1, float b2, flo
 // Lane = (row slot rs, word column mw, row half rh): it owns, for each of its tokens, the FPB pieces of
 // 8 channels 16 (FPB mw + f) + 8 rh + {0..7}, f < FPB, whose codes share bytes.
 template <int BITS, bool IS_V, int D, int DTYPE, bool ROT>
-__device__ __forceinline__ void quantize_task(const uint16_t* __restrict__ src, int64_t st, int gsz, int lo, int hi,
+__device__ __forceinline__ void quantize_task(const RowSrc& rsrc, int gsz, int lo, int hi,
                                               uint8_t* __restrict__ codes, uint32_t* __restrict__ meta_out,
                                               int lane, const int8_t* __restrict__ signs) {
   constexpr int FPB = 8 / BITS;
@@ -82,7 +95,7 @@ __device__ __forceinline__ void quantize_task(const uint16_t* __restrict__ src, 
 #pragma unroll
     for (int f = 0; f < FPB; ++f) {
       raw[k][f] = make_uint4(0u, 0u, 0u, 0u);
-      if (valid) raw[k][f] = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + 16 * (FPB * mw + f) + 8 * rh);
+      if (valid) raw[k][f] = *reinterpret_cast<const uint4*>(rsrc.row(tau) + 16 * (FPB * mw + f) + 8 * rh);
     }
   }
 
@@ -294,7 +307,7 @@ __device__ __forceinline__ void minmax8(const uint4& r, float& mn, float& mx) {
 // group rather than once per lane, and are then broadcast to the lanes of the group.  FULLBLK: every token of
 // the task is new (no predicates).  Same results as quantize_task, bit for bit.
 template <int BITS, bool IS_V, int D, int DTYPE, bool FULLBLK>
-__device__ __forceinline__ void quantize_task_fast(const uint16_t* __restrict__ src, int64_t st, int gsz, int lo,
+__device__ __forceinline__ void quantize_task_fast(const RowSrc& rsrc, int gsz, int lo,
                                                    int hi, uint8_t* __restrict__ codes,
                                                    uint32_t* __restrict__ meta_out, int lane) {
   constexpr int FPB = 8 / BITS;
@@ -334,7 +347,7 @@ __device__ __forceinline__ void quantize_task_fast(const uint16_t* __restrict__ 
 #pragma unroll
       for (int f = 0; f < FPB; ++f) {
         raw[kk][f] = make_uint4(0u, 0u, 0u, 0u);
-        if (valid[kk]) raw[kk][f] = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + 16 * (FPB * mw + f) + 8 * rh);
+        if (valid[kk]) raw[kk][f] = *reinterpret_cast<const uint4*>(rsrc.row(tau) + 16 * (FPB * mw + f) + 8 * rh);
       }
     }
     // ---- phase 1: minima / maxima of the lane's fields, per token and per set
@@ -485,7 +498,7 @@ __device__ __forceinline__ void quantize_task_fast(const uint16_t* __restrict__ 
 // AND / OR on the 32-bit words of the page (several lanes share a word).  Not tuned: these widths are served for
 // the paper's 1-, 3- and 6-bit settings, the 2/4/8-bit path above is the fast one.
 template <int D, int DTYPE>
-__device__ __forceinline__ void quantize_task_planes(const uint16_t* __restrict__ src, int64_t st, int gsz, int bits,
+__device__ __forceinline__ void quantize_task_planes(const RowSrc& rsrc, int gsz, int bits,
                                                      bool is_v, int lo, int hi, int tp0, uint8_t* __restrict__ region,
                                                      uint32_t* __restrict__ meta_out, int lane) {
   constexpr int LPR = D / 8, RPW = 32 / LPR;           // lanes per row, rows per warp step
@@ -496,7 +509,7 @@ __device__ __forceinline__ void quantize_task_planes(const uint16_t* __restrict_
     const int tau = base + r0;                         // task-local token
     const bool valid = tau < hi;
     uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-    if (valid) raw = *reinterpret_cast<const uint4*>(src + (int64_t)tau * st + 8 * l);
+    if (valid) raw = *reinterpret_cast<const uint4*>(rsrc.row(tau) + 8 * l);
     const uint32_t rw[4] = {raw.x, raw.y, raw.z, raw.w};
     float x[8];
 #pragma unroll
@@ -538,12 +551,12 @@ __device__ __forceinline__ void quantize_task_planes(const uint16_t* __restrict_
 }
 
 // 16-bit passthrough of one side of a task: rows [lo, hi) copied to the page as they are.
-__device__ __forceinline__ void copy_task_side(const uint16_t* __restrict__ src, int64_t st, int D, int lo, int hi,
+__device__ __forceinline__ void copy_task_side(const RowSrc& rsrc, int D, int lo, int hi,
                                                uint16_t* __restrict__ dst_rows, int lane) {
   const int lpr = D >> 3, rps = 32 / lpr, l = lane & (lpr - 1);
   for (int row = lo + lane / lpr; row < hi; row += rps)
     *reinterpret_cast<uint4*>(dst_rows + (size_t)row * D + l * 8) =
-        *reinterpret_cast<const uint4*>(src + (int64_t)row * st + l * 8);
+        *reinterpret_cast<const uint4*>(rsrc.row(row) + l * 8);
 }
 
 // An append of t_new tokens at position t0 fits the cache; written without a sum that could overflow.
@@ -565,25 +578,35 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int bits = is_v ? g.vb : g.kb;
   const int TT = (bits == 16 || is_plane_width(bits)) ? 32 : task_tokens(D, bits);
-  const int first_task = t0 / TT;
-  const int n_tasks = (t0 + t_new + TT - 1) / TT - first_task;
+  // tokens to quantize: the new ones, or - with a residual window of R tokens - the blocks of R that this append
+  // completes (their first tokens may come from the window, the rest from the input)
+  const int R = g.R;
+  const int qa = R ? (t0 / R) * R : t0, qb = R ? ((t0 + t_new) / R) * R : t0 + t_new;
+  if (qb <= qa) return;
+  const int first_task = qa / TT;
+  const int n_tasks = (qb + TT - 1) / TT - first_task;
   const uint16_t* in = is_v ? v_new : k_new;
   const int gsz = is_v ? g.gv : g.gk;
 
   for (int j = blockIdx.x * kWarps + warp; j < n_tasks; j += gridDim.x * kWarps) {
     const int tk0 = (first_task + j) * TT;                     // first token of the task
-    const int lo = max(t0, tk0) - tk0, hi = min(t0 + t_new, tk0 + TT) - tk0;
+    const int lo = max(qa, tk0) - tk0, hi = min(qb, tk0 + TT) - tk0;
     const int page = tk0 >> 7, tp0 = tk0 & 127;                // page-local token of the task's first row
     uint8_t* pg = c.pages + ((size_t)bh * g.n_pages + page) * g.page_bytes;
     // row 0 of the task in the input (may lie before the first new token; never dereferenced there)
-    const uint16_t* src = in + (int64_t)b * sb + (int64_t)h * sh + (int64_t)(tk0 - t0) * st;
+    RowSrc rs;
+    rs.in = in + (int64_t)b * sb + (int64_t)h * sh + (int64_t)(tk0 - t0) * st;
+    rs.st = st;
+    rs.n_win = R ? max(0, min(TT, t0 - tk0)) : 0;
+    rs.wst = 2 * D;
+    rs.win = R ? c.kv_win + ((size_t)bh * R + (tk0 % R)) * (2 * D) + (is_v ? D : 0) : nullptr;
     if (is_v) {
       if (bits == 16) {
-        copy_task_side(src, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg + g.v_codes_off) + (size_t)tp0 * D, lane);
+        copy_task_side(rs, D, lo, hi, reinterpret_cast<uint16_t*>(pg + g.v_codes_off) + (size_t)tp0 * D, lane);
         continue;
       }
       if (is_plane_width(bits)) {
-        quantize_task_planes<D, DTYPE>(src, st, gsz, bits, true, lo, hi, tp0, pg + g.v_codes_off,
+        quantize_task_planes<D, DTYPE>(rs, gsz, bits, true, lo, hi, tp0, pg + g.v_codes_off,
                                        reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / gsz), lane);
         continue;
       }
@@ -591,42 +614,42 @@ quant_token_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, cons
       uint32_t* vm = reinterpret_cast<uint32_t*>(pg + g.v_meta_off) + tp0 * (D / gsz);
       const bool full = lo == 0 && hi == TT;
       if (bits == 2) {
-        if (full) quantize_task_fast<2, true, D, DTYPE, true>(src, st, gsz, lo, hi, vb, vm, lane);
-        else quantize_task_fast<2, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane);
+        if (full) quantize_task_fast<2, true, D, DTYPE, true>(rs, gsz, lo, hi, vb, vm, lane);
+        else quantize_task_fast<2, true, D, DTYPE, false>(rs, gsz, lo, hi, vb, vm, lane);
       } else if (bits == 4) {
-        if (full) quantize_task_fast<4, true, D, DTYPE, true>(src, st, gsz, lo, hi, vb, vm, lane);
-        else quantize_task_fast<4, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane);
+        if (full) quantize_task_fast<4, true, D, DTYPE, true>(rs, gsz, lo, hi, vb, vm, lane);
+        else quantize_task_fast<4, true, D, DTYPE, false>(rs, gsz, lo, hi, vb, vm, lane);
       } else {
-        if (full) quantize_task_fast<8, true, D, DTYPE, true>(src, st, gsz, lo, hi, vb, vm, lane);
-        else quantize_task_fast<8, true, D, DTYPE, false>(src, st, gsz, lo, hi, vb, vm, lane);
+        if (full) quantize_task_fast<8, true, D, DTYPE, true>(rs, gsz, lo, hi, vb, vm, lane);
+        else quantize_task_fast<8, true, D, DTYPE, false>(rs, gsz, lo, hi, vb, vm, lane);
       }
     } else {
       if (bits == 16) {
-        copy_task_side(src, st, D, lo, hi, reinterpret_cast<uint16_t*>(pg) + (size_t)tp0 * D, lane);
+        copy_task_side(rs, D, lo, hi, reinterpret_cast<uint16_t*>(pg) + (size_t)tp0 * D, lane);
         continue;
       }
       if (is_plane_width(bits)) {
-        quantize_task_planes<D, DTYPE>(src, st, gsz, bits, false, lo, hi, tp0, pg,
+        quantize_task_planes<D, DTYPE>(rs, gsz, bits, false, lo, hi, tp0, pg,
                                        reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / gsz), lane);
         continue;
       }
       uint8_t* kr = pg + (size_t)tp0 * (D * bits / 8);
       uint32_t* km = reinterpret_cast<uint32_t*>(pg + g.k_meta_off) + tp0 * (D / gsz);
       if constexpr (ROT) {
-        if (bits == 2) quantize_task<2, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
-        else if (bits == 4) quantize_task<4, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
-        else quantize_task<8, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane, c.k_signs);
+        if (bits == 2) quantize_task<2, false, D, DTYPE, true>(rs, gsz, lo, hi, kr, km, lane, c.k_signs);
+        else if (bits == 4) quantize_task<4, false, D, DTYPE, true>(rs, gsz, lo, hi, kr, km, lane, c.k_signs);
+        else quantize_task<8, false, D, DTYPE, true>(rs, gsz, lo, hi, kr, km, lane, c.k_signs);
       } else {
         const bool full = lo == 0 && hi == TT;
         if (bits == 2) {
-          if (full) quantize_task_fast<2, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane);
-          else quantize_task_fast<2, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane);
+          if (full) quantize_task_fast<2, false, D, DTYPE, true>(rs, gsz, lo, hi, kr, km, lane);
+          else quantize_task_fast<2, false, D, DTYPE, false>(rs, gsz, lo, hi, kr, km, lane);
         } else if (bits == 4) {
-          if (full) quantize_task_fast<4, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane);
-          else quantize_task_fast<4, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane);
+          if (full) quantize_task_fast<4, false, D, DTYPE, true>(rs, gsz, lo, hi, kr, km, lane);
+          else quantize_task_fast<4, false, D, DTYPE, false>(rs, gsz, lo, hi, kr, km, lane);
         } else {
-          if (full) quantize_task_fast<8, false, D, DTYPE, true>(src, st, gsz, lo, hi, kr, km, lane);
-          else quantize_task_fast<8, false, D, DTYPE, false>(src, st, gsz, lo, hi, kr, km, lane);
+          if (full) quantize_task_fast<8, false, D, DTYPE, true>(rs, gsz, lo, hi, kr, km, lane);
+          else quantize_task_fast<8, false, D, DTYPE, false>(rs, gsz, lo, hi, kr, km, lane);
         }
       }
     }
@@ -744,6 +767,25 @@ quant_kchan_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new,
   }
 }
 
+// Residual window: the new tokens that stay unquantized (positions >= the last complete block of R) are copied to
+// the ring, key row and value row of token t in slot t % R.  Runs after the quantize kernel, which may still read
+// the slots being replaced.
+__global__ void __launch_bounds__(kThreads)
+window_store_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new, const uint16_t* __restrict__ v_new,
+                    int64_t sb, int64_t sh, int64_t st, int t_new) {
+  const int bh = blockIdx.y, b = bh / g.Hkv, h = bh % g.Hkv;
+  const int t0 = c.seq_len[b];
+  if (!append_fits(t0, t_new, g.capacity)) return;
+  const int R = g.R, D = g.D, vpr = D / 8;
+  const int first = max(t0, ((t0 + t_new) / R) * R), n = t0 + t_new - first;     // tokens first .. first + n - 1 stay
+  for (int idx = blockIdx.x * kThreads + threadIdx.x; idx < n * 2 * vpr; idx += gridDim.x * kThreads) {
+    const int t = first + idx / (2 * vpr), side = (idx / vpr) & 1, vcol = idx % vpr;
+    const uint16_t* src = (side ? v_new : k_new) + (int64_t)b * sb + (int64_t)h * sh + (int64_t)(t - t0) * st + 8 * vcol;
+    uint16_t* dst = c.kv_win + (((size_t)bh * R + (t % R)) * 2 + side) * D + 8 * vcol;
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+  }
+}
+
 __global__ void bump_seq_len_kernel(Geom g, CachePtrs c, int t_new) {
   int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= g.B) return;
@@ -784,6 +826,10 @@ int launch_quantize_append(const Geom& g, const CachePtrs& c, const void* k_new,
     cudaFuncSetAttribute(quant_kchan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 128 * 3);
     dim3 grid2((t_new + 127) / 128 + 1, streams);
     quant_kchan_kernel<<<grid2, kThreads, smem, stream>>>(g, c, k, sb, sh, st, t_new);
+  }
+  if (g.R) {
+    dim3 grid3(1, streams);
+    window_store_kernel<<<grid3, kThreads, 0, stream>>>(g, c, k, v, sb, sh, st, t_new);
   }
   bump_seq_len_kernel<<<(g.B + 127) / 128, 128, 0, stream>>>(g, c, t_new);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;

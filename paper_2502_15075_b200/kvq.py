@@ -29,12 +29,13 @@ STATUS_CAPACITY, STATUS_DEVICE_TIMEOUT = 1, 2
 class kvq_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in (
         "batch", "n_q_heads", "n_kv_heads", "head_dim", "kb", "vb", "gk", "gv", "k_axis", "in_dtype",
-        "capacity_tokens")]
+        "capacity_tokens", "residual_tokens")]
 
 
 class kvq_cache(ctypes.Structure):
     _fields_ = [("pages", ctypes.c_void_p), ("k_tail", ctypes.c_void_p),
-                ("seq_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("k_signs", ctypes.c_void_p)]
+                ("seq_len", ctypes.c_void_p), ("status", ctypes.c_void_p), ("k_signs", ctypes.c_void_p),
+                ("kv_win", ctypes.c_void_p)]
 
 
 _P = ctypes.POINTER
@@ -42,6 +43,8 @@ _lib.kvq_layout_version.restype = ctypes.c_int
 _lib.kvq_page_bytes.argtypes = [_P(kvq_config), _P(ctypes.c_size_t)]
 _lib.kvq_cache_bytes.argtypes = [_P(kvq_config), _P(ctypes.c_size_t), _P(ctypes.c_size_t)]
 _lib.kvq_workspace_bytes.argtypes = [_P(kvq_config), _P(ctypes.c_size_t)]
+_lib.kvq_window_bytes.argtypes = [_P(kvq_config), _P(ctypes.c_size_t)]
+_lib.kvq_window_bytes.restype = ctypes.c_int
 _lib.kvq_quantize_append.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
                                      ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p]
 _lib.kvq_decode_attention.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
@@ -74,7 +77,7 @@ for _f in ("kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes", "kvq_quan
 EXPORTS = ("kvq_layout_version", "kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes",
            "kvq_quantize_append", "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize",
            "kvq_check_status", "kvq_strerror", "kvq_quant_error", "kvq_bit_balance", "kvq_workspace_bytes_rows",
-           "kvq_decode_attention_rows")
+           "kvq_decode_attention_rows", "kvq_window_bytes")
 STATIC_SCRATCH_BYTES = 8 << 20
 
 
@@ -106,9 +109,17 @@ def kvq_layout_version() -> int:
     return _lib.kvq_layout_version()
 
 
-def make_config(batch, n_q_heads, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, dtype, capacity_tokens) -> kvq_config:
+def make_config(batch, n_q_heads, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, dtype, capacity_tokens,
+                residual_tokens=0) -> kvq_config:
     code = _dtype_code(dtype) if isinstance(dtype, torch.dtype) else {"fp16": 0, "bf16": 1}[dtype]
-    return kvq_config(batch, n_q_heads, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, code, capacity_tokens)
+    return kvq_config(batch, n_q_heads, n_kv_heads, head_dim, kb, vb, gk, gv, k_axis, code, capacity_tokens,
+                      residual_tokens)
+
+
+def kvq_window_bytes(cfg: kvq_config) -> int:
+    out = ctypes.c_size_t()
+    _check(_lib.kvq_window_bytes(ctypes.byref(cfg), ctypes.byref(out)), "kvq_window_bytes")
+    return out.value
 
 
 def kvq_page_bytes(cfg: kvq_config) -> int:
@@ -142,13 +153,21 @@ class Cache:
         self.k_tail = torch.zeros(tail_bytes // 2, dtype=torch.float16, device=device) if tail_bytes else None
         self.seq_len = torch.zeros(cfg.batch, dtype=torch.int32, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
+        win_bytes = kvq_window_bytes(cfg)
+        self.kv_win = torch.zeros(win_bytes // 2, dtype=torch.int16, device=device) if win_bytes else None
         self.c = kvq_cache(self.pages.data_ptr(), self.k_tail.data_ptr() if self.k_tail is not None else None,
                            self.seq_len.data_ptr(), self.status.data_ptr(),
-                           self.k_signs.data_ptr() if self.k_signs is not None else None)
+                           self.k_signs.data_ptr() if self.k_signs is not None else None,
+                           self.kv_win.data_ptr() if self.kv_win is not None else None)
 
     def pages_view(self) -> torch.Tensor:
         c = self.cfg
         return self.pages.view(c.batch, c.n_kv_heads, c.capacity_tokens // PAGE_TOKENS, -1)
+
+    def window_view(self) -> Optional[torch.Tensor]:
+        """int16 [B, Hkv, R, 2, D] bit patterns of the residual window, or None."""
+        c = self.cfg
+        return None if self.kv_win is None else self.kv_win.view(c.batch, c.n_kv_heads, c.residual_tokens, 2, c.head_dim)
 
     def tail_view(self) -> Optional[torch.Tensor]:
         c = self.cfg

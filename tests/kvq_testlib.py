@@ -16,23 +16,24 @@ def bits_of(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-def oracle_cache_for(w: wl.Workload, batch: int, capacity: int, k_signs=None) -> OracleCache:
+def oracle_cache_for(w: wl.Workload, batch: int, capacity: int, k_signs=None, residual=0) -> OracleCache:
     return OracleCache(batch, w.n_kv_heads, w.head_dim, w.kb, w.vb, w.gk, w.gv, w.k_axis, w.dtype, capacity,
-                       k_signs=k_signs)
+                       k_signs=k_signs, residual=residual)
 
 
-def gpu_config_for(kvq, w: wl.Workload, batch: int, capacity: int):
+def gpu_config_for(kvq, w: wl.Workload, batch: int, capacity: int, residual=0):
     return kvq.make_config(batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.kb, w.vb, w.gk, w.gv, w.k_axis,
-                           w.torch_dtype, capacity)
+                           w.torch_dtype, capacity, residual)
 
 
-def build_both(kvq, w: wl.Workload, k: torch.Tensor, v: torch.Tensor, chunks, capacity: int, k_signs=None):
+def build_both(kvq, w: wl.Workload, k: torch.Tensor, v: torch.Tensor, chunks, capacity: int, k_signs=None,
+               residual=0):
     """Append k, v ([B,Hkv,T,D] CPU tensors) in the given chunk sizes through both paths.
     k_signs: optional +-1 per channel (numpy int8): rotate the keys on both sides."""
     B = k.shape[0]
-    cfg = gpu_config_for(kvq, w, B, capacity)
+    cfg = gpu_config_for(kvq, w, B, capacity, residual)
     gc = kvq.Cache(cfg, k_signs=None if k_signs is None else torch.from_numpy(k_signs))
-    oc = oracle_cache_for(w, B, capacity, k_signs)
+    oc = oracle_cache_for(w, B, capacity, k_signs, residual)
     kd, vd = k.cuda(), v.cuda()
     kb_, vb_ = bits_of(k), bits_of(v)
     t = 0
@@ -57,6 +58,12 @@ def assert_caches_equal(gc, oc: OracleCache):
         for b in range(oc.B):
             r = int(oc.seq_len[b]) % 128
             assert np.array_equal(gt[b, :, :r], oc.k_tail[b, :, :r]), "fp16 tail differs"
+    if oc.R:
+        gw = gc.window_view().cpu().numpy().view(np.uint16)
+        for b in range(oc.B):
+            n = int(oc.seq_len[b])
+            slots = np.arange(oc.flushed(b), n) % oc.R
+            assert np.array_equal(gw[b][:, slots], oc.kv_win[b][:, slots]), "residual window differs"
 
 
 def oracle_on_gpu_codes(gc, w: wl.Workload) -> OracleCache:
@@ -64,8 +71,10 @@ def oracle_on_gpu_codes(gc, w: wl.Workload) -> OracleCache:
     same codes)."""
     cfg = gc.cfg
     oc = oracle_cache_for(w, cfg.batch, cfg.capacity_tokens,
-                          None if gc.k_signs is None else gc.k_signs.cpu().numpy())
+                          None if gc.k_signs is None else gc.k_signs.cpu().numpy(), cfg.residual_tokens)
     oc.pages = gc.pages_view().cpu().numpy().copy()
+    if oc.R:
+        oc.kv_win = gc.window_view().cpu().numpy().view(np.uint16).copy()
     if oc.k_tail is not None:
         oc.k_tail = gc.tail_view().cpu().view(torch.int16).numpy().view(np.uint16).copy()
     oc.seq_len = gc.seq_len.cpu().numpy().copy()
