@@ -137,6 +137,8 @@ int kvq_workspace_bytes(const kvq_config* cfg, size_t* out);
  *   k_new, v_new: device, in_dtype, logical shape [batch][n_kv_heads][t_new][head_dim];
  *     element (b,h,t,d) at offset b*stride_b + h*stride_h + t*stride_t + d (in elements);
  *     head_dim contiguous, base pointers and strides such that every row is 16-byte aligned.
+ * With residual_tokens = R > 0 the new tokens first live in kv_win; the blocks of R tokens that this call completes
+ * are quantized (their first tokens read from kv_win) and the tokens behind the last complete block are stored there.
  * Asynchronous on cuda_stream.  seq_len[b] += t_new for every sequence that fits; a sequence
  * with seq_len[b] + t_new > capacity_tokens is left untouched and KVQ_STATUS_CAPACITY is set.
  * Returns KVQ_OK or a host-detected argument / launch error (then nothing was launched).
@@ -152,7 +154,8 @@ int kvq_quantize_append(const kvq_config* cfg, const kvq_cache* cache,
  * over t < seq_len[b] (App. A.1: S = Q K^T / sqrt(d), A = softmax(S), A V), streaming the
  * packed pages and reconstructing K^, V^ on the fly; tokens of an incomplete channel-wise
  * key block are read from the fp16 tail.  Split over the sequence, partial results merged by
- * log-sum-exp.  seq_len[b] == 0 gives zeros.
+ * log-sum-exp.  seq_len[b] == 0 gives zeros.  Tokens of a residual window (residual_tokens > 0) are attended in
+ * full precision; that needs a configuration the tensor-core path serves (otherwise KVQ_ERR_UNSUPPORTED).
  *   q: device, in_dtype, [batch][n_q_heads][head_dim] contiguous.
  *   out: device, [batch][n_q_heads][head_dim] contiguous, out_dtype (KVQ_FP16/BF16/FP32).
  *   softmax_scale <= 0 selects 1/sqrt(head_dim).
@@ -185,7 +188,8 @@ int kvq_decode_attention_rows(const kvq_config* cfg, const kvq_cache* cache,
 
 /*
  * Reconstruct tokens t_begin <= t < min(t_end, seq_len[b]) as x^ = fmaf(code, s, z) rounded to
- * in_dtype (App. B.1: A^ = scale * Q); tail keys are converted from fp16.
+ * in_dtype (App. B.1: A^ = scale * Q); tail keys are converted from fp16, tokens of a residual window are returned
+ * as they were appended.
  *   k_out, v_out: device, in_dtype, [batch][n_kv_heads][capacity_tokens][head_dim] contiguous;
  *     either may be NULL to skip it.  Elements outside the token range are not written.
  * Asynchronous on cuda_stream; reads the cache only.

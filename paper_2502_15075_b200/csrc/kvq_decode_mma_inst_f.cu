@@ -9,6 +9,7 @@ namespace mma {
       unsigned long long, long long, cudaStream_t);
 KVQ_MMA_DECL(128, 4, 2, 0, 4, 1, 2, 4, 2)
 KVQ_MMA_DECL(128, 4, 2, 0, 2, 2, 2, 4, 2)
+KVQ_MMA_DECL(64, 4, 2, 0, 2, 2, 1, 4, 3)
 #undef KVQ_MMA_DECL
 }  // namespace mma
 }  // namespace kvq
