@@ -344,13 +344,11 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
   for (long long x = x_lo; x < x_hi;) {
     const int seg_pages = (int)min((long long)(pages_b - page), x_hi - x);
-    const int n_all = clamped_len(c.seq_len, b, g.capacity);      // tokens of the sequence
-    const int n_tok = g.R ? (n_all / g.R) * g.R : n_all;          // ... of which in the pages
-    const bool has_win = n_all > n_tok;                           // the window kernel left a partial in slot s_cap - 1
+    const int n_tok = paged_len(c.seq_len, b, g.capacity, g.R);   // tokens of the sequence that are in the pages
+    // a block is unmasked when all of its 32 tokens exist and every query row may see them (several causal rows:
+    // row r sees the first n - (rows - 1 - r) tokens of the n the sequence holds, window included)
+    const int n_unmasked = min(n_tok, clamped_len(c.seq_len, b, g.capacity) - (g.rows - 1));
     const int stream = b * Hkv + h;
-    int limh[NH];                          // tokens the lane's heads may attend to (causal limit of their query row)
-#pragma unroll
-    for (int nh = 0; nh < NH; ++nh) limh[nh] = n_all - (g.rows - 1 - min((tid + 4 * nh) / Gq, g.rows - 1));
 
     // ---- segment start: q operands, group sums and a clean state for this stream's heads
     {
@@ -647,10 +645,13 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             }
             if (MASKED) {
               const int tokg = (page + pp) * kPageTokens + tok0;        // position of row tok0 in the sequence
+              const int n_all = clamped_len(c.seq_len, b, g.capacity);
 #pragma unroll
               for (int nh = 0; nh < NH; ++nh) {
-                if (!vld[u][0] || tokg >= limh[nh]) L[u][0][nh] = -INFINITY;
-                if (!vld[u][1] || tokg + 8 >= limh[nh]) L[u][1][nh] = -INFINITY;
+                // tokens the lane's head may attend to: the causal limit of its query row
+                const int lim = n_all - (g.rows - 1 - min((tid + 4 * nh) / Gq, g.rows - 1));
+                if (!vld[u][0] || tokg >= lim) L[u][0][nh] = -INFINITY;
+                if (!vld[u][1] || tokg + 8 >= lim) L[u][1][nh] = -INFINITY;
               }
             }
           }
@@ -771,7 +772,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         };
 
         // the masked variant also serves the last tokens when several causal query rows see different prefixes
-        if (nv - wq * 32 >= 32 && (page + pp) * kPageTokens + wq * 32 + 32 <= n_all - (g.rows - 1)) do_block(std::false_type{});
+        if ((page + pp) * kPageTokens + wq * 32 + 32 <= n_unmasked) do_block(std::false_type{});
         else do_block(std::true_type{});
       }
       __syncwarp();
@@ -811,6 +812,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       const int c_first = plan.cta_of(xs);
       const int slot = (int)blockIdx.x - c_first;
       const int n_part = plan.cta_of(xs + pages_b - 1) - c_first + 1;        // partials of this stream
+      const bool has_win = clamped_len(c.seq_len, b, g.capacity) > n_tok;    // the window kernel left a partial in slot s_cap - 1
       if (slot >= 0 && slot < s_plan) {
         for (int idx = tid_; idx < G * D; idx += NCONS) {
           const int head = idx / D, d = idx % D;
