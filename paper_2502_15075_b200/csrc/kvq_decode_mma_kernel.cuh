@@ -34,22 +34,21 @@ struct SmemLayout {
   int page_stride, ring_bytes, bar_off, pref_off, misc_off, master_off, ml_off, chan_off, total;
 };
 // master: per consumer warp, 4 NH heads x (D + 8) floats (the row padding keeps a warp's accesses conflict-free).
-// chan: channel-wise keys need, per group of four warps, two buffers of per-page q operands (NH x 2 x D/16 x 32 words),
-// the partial zero-point sums (2 x 8 heads x 8 floats) and the page's fixed-point scale per head (2 x 8), and once
-// the stream's q in fp32 (8 x D).
+// chan: channel-wise keys keep, per ring stage, the page's q operands made by the preparation warp
+// (NH x 2 x D/16 x 32 words) followed by 8 zero-point sums and 8 fixed-point scales (one per head).
+__host__ __device__ inline int chan_stage_bytes(int D, int nh) { return nh * 2 * (D / 16) * 32 * 4 + 64; }
 __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, int nw, int batch, int D, int nh,
                                                   bool chan) {
   SmemLayout s;
   s.page_stride = (page_bytes + 127) & ~127;
   s.ring_bytes = s.page_stride * stages;
   s.bar_off = s.ring_bytes;
-  s.pref_off = s.bar_off + 16 * 8 * 2;                      // up to 16 stages x (full, empty)
+  s.pref_off = s.bar_off + 16 * 8 * 2;                      // up to 32 barriers: (full, empty[, ready]) per stage
   s.misc_off = (s.pref_off + (batch + 1) * 4 + 15) & ~15;
   s.master_off = s.misc_off + 64;
   s.ml_off = s.master_off + nw * 4 * nh * (D + 8) * 4;
   s.chan_off = s.ml_off + nw * 4 * nh * 2 * 4;
-  const int ng = nw / 4;
-  s.total = s.chan_off + (chan ? (2 * ng * nh * 2 * (D / 16) * 32 * 4 + 2 * ng * 64 * 4 + 2 * ng * 8 * 4 + 8 * D * 4) : 0);
+  s.total = s.chan_off + (chan ? stages * chan_stage_bytes(D, nh) : 0);
   return s;
 }
 
@@ -127,6 +126,73 @@ template <int NH> constexpr int kPBits = NH == 1 ? 31 : 24;
 template <int NH> constexpr float kHeadroom = NH == 1 ? 6.0f : 1.0f;
 constexpr int kFlushBlocks = 512;          // fold the int32 value accumulators at least this often (no overflow)
 
+// The query values a lane needs as MMA operand: head hb (a (row, head) pair when several rows are served), channels
+// 16 r + 4 tid + {0..3} for every slot r, in fp32, rotated like the keys if the cache rotates them; heads >= G are
+// zero.  Returns max |q| over the lane's values (the caller reduces over the quad).
+template <int D>
+__device__ __forceinline__ float load_q_lane(const Geom& g, const CachePtrs& c, const uint16_t* __restrict__ q, int b,
+                                             int h, int hb, int tid, float (&qv)[D / 16][4]) {
+  constexpr int NR = D / 16;
+  constexpr uint32_t FULL = 0xffffffffu;
+  const int Gq = g.G, G = g.G * g.rows;
+        const uint16_t* qrow = q + (((size_t)b * g.rows + hb / Gq) * g.Hq + (size_t)h * Gq + hb % Gq) * D;
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+          uint2 raw = make_uint2(0u, 0u);
+          if (hb < G) raw = *reinterpret_cast<const uint2*>(qrow + 16 * r + 4 * tid);
+          qv[r][0] = bits16_to_f32((uint16_t)(raw.x & 0xFFFF), g.in_dtype);
+          qv[r][1] = bits16_to_f32((uint16_t)(raw.x >> 16), g.in_dtype);
+          qv[r][2] = bits16_to_f32((uint16_t)(raw.y & 0xFFFF), g.in_dtype);
+          qv[r][3] = bits16_to_f32((uint16_t)(raw.y >> 16), g.in_dtype);
+        }
+        if (c.k_signs != nullptr) {
+          // rotated keys: give q the same rotation, q' = H (signs * q) / sqrt(D); channel 16 r + 4 tid + j,
+          // so the butterflies run over j inside the lane, over tid across lanes, over r inside the lane
+#pragma unroll
+          for (int r = 0; r < NR; ++r) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) qv[r][j] *= (float)c.k_signs[16 * r + 4 * tid + j];
+            float a = qv[r][0], bq = qv[r][1], cq = qv[r][2], dq = qv[r][3];
+            qv[r][0] = (a + bq) + (cq + dq); qv[r][1] = (a - bq) + (cq - dq);
+            qv[r][2] = (a + bq) - (cq + dq); qv[r][3] = (a - bq) - (cq - dq);
+#pragma unroll
+            for (int m = 1; m < 4; m <<= 1) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float o = __shfl_xor_sync(FULL, qv[r][j], m);
+                qv[r][j] = (tid & m) ? o - qv[r][j] : qv[r][j] + o;
+              }
+            }
+          }
+#pragma unroll
+          for (int hh = 1; hh < NR; hh <<= 1) {
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+              if ((r & hh) == 0) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  const float a = qv[r][j], bq = qv[r + hh][j];
+                  qv[r][j] = a + bq;
+                  qv[r + hh][j] = a - bq;
+                }
+              }
+            }
+          }
+#pragma unroll
+          for (int r = 0; r < NR; ++r) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) qv[r][j] *= inv_sqrt_dim<D>();
+          }
+        }
+        float amax = 0.f;
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) amax = fmaxf(amax, fabsf(qv[r][j]));
+        }
+  return amax;
+}
+
 // Template parameters: head_dim, key bits, value bits, key axis (0 token-wise, 1 channel-wise), key / value groups
 // per row, NH = query heads per lane (1: up to 4 heads per KV head, 2: up to 8), consumer warps (4: one per
 // 32-token block of a page), resident CTAs per SM.
@@ -137,7 +203,7 @@ constexpr int kFlushBlocks = 512;          // fold the int32 value accumulators 
 // warp (g = lane / 4, t = lane % 4) owns query heads t (and t + 4 when NH = 2): its accumulator columns 2t, 2t+1
 // are the limbs of that head, so logits, softmax and the fixed-point weights need no exchange between lanes.
 template <int D, int KB, int VB, int KAXIS, int NGK, int NGV, int NH, int NW, int MINB>
-__global__ void __launch_bounds__((NW + 1) * 32, MINB)
+__global__ void __launch_bounds__((NW + 1 + (KAXIS == 1 ? 1 : 0)) * 32, MINB)
 decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1, float* __restrict__ ws,
                   int s_cap, int stages, void* __restrict__ out, int out_dtype, unsigned long long call_id,
                   unsigned long long wait_ns, long long skip_x) {
@@ -204,6 +270,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     for (int s = 0; s < stages; ++s) {
       mbar_init(smem_u32(&bars[s]), 1);
       mbar_init(smem_u32(&bars[stages + s]), 4);
+      if constexpr (KAXIS == 1) mbar_init(smem_u32(&bars[2 * stages + s]), 1);     // ready: operands of the page made
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -285,23 +352,120 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     return;
   }
 
+  // =========================================================== preparation warp (channel-wise keys)
+  // Per page, the operand of the integer QK^T MMAs is q_d * s_d in 24-bit fixed point (scale from max|q| of the head
+  // times the page's largest channel scale), and sum_d q_d z_d is one fp32 scalar per head.  One warp makes both for
+  // every page, in the lane arrangement the consumers' B fragments have, leaves them in the stage's operand buffer
+  // and signals the stage's `ready` barrier; for the incomplete last block it leaves q split into fp16 high and
+  // low parts instead (operands of the fp16 MMAs on the tail keys).
+  if constexpr (KAXIS == 1) {
+    if (warp == NW + 1) {
+      constexpr int CSB = NH * 2 * NR * 32 * 4 + 64;
+      int stage = 0;
+      uint32_t phase = 0;
+      float qv[NH][NR][4];
+      float amaxB[NH];
+      int cur_b = -1, cur_h = -1;
+      for (long long x = x_lo; x < x_hi; ++x) {
+        if (b != cur_b || h != cur_h) {          // a new stream: its queries
+          cur_b = b; cur_h = h;
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) {
+            float am = load_q_lane<D>(g, c, q, b, h, (gid >> 1) + 4 * nh, tid, qv[nh]);
+            am = fmaxf(am, __shfl_xor_sync(FULL, am, 1));
+            amaxB[nh] = fmaxf(am, __shfl_xor_sync(FULL, am, 2));
+          }
+        }
+        const int n_tok = paged_len(c.seq_len, b, g.capacity, g.R);
+        const bool tail_pg = n_tok - page * kPageTokens < kPageTokens;
+        const bool got = mbar_wait(bar0 + 8 * stage, phase, wait_ns);
+        if (!__all_sync(FULL, got) || *abort_flag) {
+          *abort_flag = 1;
+          if (lane == 0) atomicOr(c.status, KVQ_STATUS_DEVICE_TIMEOUT);
+          return;
+        }
+        const uint8_t* sp = smem + stage * sl.page_stride;
+        uint32_t* ops = reinterpret_cast<uint32_t*>(smem + sl.chan_off + stage * CSB);     // [NH][2][NR][32]
+        float* opf = reinterpret_cast<float*>(ops + NH * 2 * NR * 32);                      // zq[8], hs[8]
+        if (tail_pg) {
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) {
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+              uint32_t h0, l0_, h1, l1_;
+              split_h2(qv[nh][r][0], qv[nh][r][2], h0, l0_);
+              split_h2(qv[nh][r][1], qv[nh][r][3], h1, l1_);
+              ops[((nh * 2 + 0) * NR + r) * 32 + lane] = (gid & 1) ? l0_ : h0;
+              ops[((nh * 2 + 1) * NR + r) * 32 + lane] = (gid & 1) ? l1_ : h1;
+            }
+          }
+        } else {
+          const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + K_META_OFF);
+          float smax = 0.f;
+          if (4 * lane < D) {
+            const uint4 mm = *reinterpret_cast<const uint4*>(km + 4 * lane);
+            smax = fmaxf(fmaxf(meta_s(mm.x), meta_s(mm.y)), fmaxf(meta_s(mm.z), meta_s(mm.w)));
+          }
+#pragma unroll
+          for (int off = 1; off < 32; off <<= 1) smax = fmaxf(smax, __shfl_xor_sync(FULL, smax, off));
+#pragma unroll
+          for (int nh = 0; nh < NH; ++nh) {
+            const int hb = (gid >> 1) + 4 * nh;
+            const float am = amaxB[nh] * smax;
+            const float scale = am > 0.f ? kQFix3 / am : 0.f;
+            float zsum = 0.f;
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+              const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);     // (s, z) of 4 channels
+              const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
+              float t[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 sz = __half22float2(as_h2(mw[j]));
+                t[j] = qv[nh][r][j] * sz.x;
+                zsum = fmaf(qv[nh][r][j], sz.y, zsum);
+              }
+              uint32_t w0, w1;
+              fixed_point_bytes3(t, scale, gid & 1, w0, w1);
+              ops[((nh * 2 + 0) * NR + r) * 32 + lane] = w0;
+              ops[((nh * 2 + 1) * NR + r) * 32 + lane] = w1;
+            }
+            zsum += __shfl_xor_sync(FULL, zsum, 1);
+            zsum += __shfl_xor_sync(FULL, zsum, 2);
+            if (tid == 0 && (gid & 1) == 0) {
+              opf[hb] = c1 * zsum;
+              opf[8 + hb] = am > 0.f ? c1 / scale : 0.f;
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar0 + 8 * (2 * stages + stage));
+        if (++stage == stages) { stage = 0; phase ^= 1; }
+        if (++page == pages_b) {
+          page = 0;
+          if (++h == Hkv) {
+            h = 0;
+            do { ++b; } while (b < B && sPref[b + 1] == sPref[b]);
+            if (b < B) pages_b = (sPref[b + 1] - sPref[b]) / Hkv;
+          }
+        }
+      }
+      return;
+    }
+  }
+
   // =========================================================== consumer warps
   uint32_t qB[NH][NTK][NR];    // QK^T B operands: column gid = (head gid/2 + 4 nh, limb gid%2), channels 16 r + 4 tid + {0..3};
                                // channel-wise keys: n-tile 0 carries (byte 2 signed, none), n-tile 1 (byte 1, byte 0) unsigned
   float hs[NH];                // c1 / fixed-point scale of q, own heads (tid + 4 nh)
   float qsum[NH][NGK];         // c1 * sum of q over each key group, own heads
   float zq[NH];                // channel-wise keys: c1 * sum_d q_d z_d of the current page, own heads
-  float amaxB[NH];             // channel-wise keys: max |q| of the operand heads (gid/2 + 4 nh)
   float m_ref[NH], l[NH], zacc[NH][NGV];
   int Oi[NTV][MT][4];          // PV accumulators: NH = 1: n-tiles (limb 3, 2 | limb 1, 0) of head tid; NH = 2: (head tid:
                                // limb 2, 1 | head tid + 4: limb 2, 1 | limb 0 of both)
   constexpr float PONE = (float)(1u << (kPBits<NH> - 1)) * 2.0f;     // 2^PBITS
   // sscale = 2^PBITS / s_lim, s_lim a power of two above every value scale folded into the weights so far (2^-40 at first)
   float sscale = PONE / 9.094947e-13f;
-  uint32_t* sB = reinterpret_cast<uint32_t*>(smem + sl.chan_off);                                  // [2 NG][NH][2][NR][32]
-  float* sZ = reinterpret_cast<float*>(smem + sl.chan_off + 2 * NG * NH * 2 * NR * 32 * 4);        // [2 NG][8 heads][8]
-  float* sHS = sZ + 2 * NG * 64;                                                                   // [2 NG][8 heads]
-  float* sQ = sHS + 2 * NG * 8;                                                                         // [8 heads][D]
   float* myM = sMaster + warp * NHEADS * MSTRIDE;
   const int grp = warp >> 2, wq = warp & 3;       // page group of this warp, and its 32-token block inside a page
   int page_no = 0;
@@ -352,76 +516,16 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 
     // ---- segment start: q operands, group sums and a clean state for this stream's heads
     {
-      if constexpr (KAXIS == 1) named_bar_sync(1, NCONS);            // nobody still reads the previous stream's q
 #pragma unroll
       for (int nh = 0; nh < NH; ++nh) {
         const int hb = (gid >> 1) + 4 * nh;                          // head of this lane's operand column
         float qv[NR][4];
-        const uint16_t* qrow = q + (((size_t)b * g.rows + hb / Gq) * g.Hq + (size_t)h * Gq + hb % Gq) * D;
-#pragma unroll
-        for (int r = 0; r < NR; ++r) {
-          uint2 raw = make_uint2(0u, 0u);
-          if (hb < G) raw = *reinterpret_cast<const uint2*>(qrow + 16 * r + 4 * tid);
-          qv[r][0] = bits16_to_f32((uint16_t)(raw.x & 0xFFFF), g.in_dtype);
-          qv[r][1] = bits16_to_f32((uint16_t)(raw.x >> 16), g.in_dtype);
-          qv[r][2] = bits16_to_f32((uint16_t)(raw.y & 0xFFFF), g.in_dtype);
-          qv[r][3] = bits16_to_f32((uint16_t)(raw.y >> 16), g.in_dtype);
-        }
-        if (c.k_signs != nullptr) {
-          // rotated keys: give q the same rotation, q' = H (signs * q) / sqrt(D); channel 16 r + 4 tid + j,
-          // so the butterflies run over j inside the lane, over tid across lanes, over r inside the lane
-#pragma unroll
-          for (int r = 0; r < NR; ++r) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) qv[r][j] *= (float)c.k_signs[16 * r + 4 * tid + j];
-            float a = qv[r][0], bq = qv[r][1], cq = qv[r][2], dq = qv[r][3];
-            qv[r][0] = (a + bq) + (cq + dq); qv[r][1] = (a - bq) + (cq - dq);
-            qv[r][2] = (a + bq) - (cq + dq); qv[r][3] = (a - bq) - (cq - dq);
-#pragma unroll
-            for (int m = 1; m < 4; m <<= 1) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float o = __shfl_xor_sync(FULL, qv[r][j], m);
-                qv[r][j] = (tid & m) ? o - qv[r][j] : qv[r][j] + o;
-              }
-            }
-          }
-#pragma unroll
-          for (int hh = 1; hh < NR; hh <<= 1) {
-#pragma unroll
-            for (int r = 0; r < NR; ++r) {
-              if ((r & hh) == 0) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const float a = qv[r][j], bq = qv[r + hh][j];
-                  qv[r][j] = a + bq;
-                  qv[r + hh][j] = a - bq;
-                }
-              }
-            }
-          }
-#pragma unroll
-          for (int r = 0; r < NR; ++r) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) qv[r][j] *= inv_sqrt_dim<D>();
-          }
-        }
         float amax = 0.f;
-#pragma unroll
-        for (int r = 0; r < NR; ++r) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) amax = fmaxf(amax, fabsf(qv[r][j]));
-        }
+        if constexpr (KAXIS == 0) amax = load_q_lane<D>(g, c, q, b, h, hb, tid, qv);
         amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 1));
         amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, 2));
         if constexpr (KAXIS == 1) {
-          // channel-wise keys: the operands depend on the page's scales and are made per page from the stream's q
-          amaxB[nh] = amax;
-          if ((gid & 1) == 0) {
-#pragma unroll
-            for (int r = 0; r < NR; ++r)
-              *reinterpret_cast<float4*>(sQ + hb * D + 16 * r + 4 * tid) = make_float4(qv[r][0], qv[r][1], qv[r][2], qv[r][3]);
-          }
+          // channel-wise keys: the operands depend on the page's scales; the preparation warp makes them per page
           hs[nh] = 0.f;
         } else {
           // 16-bit fixed point relative to the head's largest entry: Q = rint(q * scale), |Q| <= 32512
@@ -449,7 +553,6 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
 #pragma unroll
         for (int j = 0; j < NGV; ++j) zacc[nh][j] = 0.f;
       }
-      if constexpr (KAXIS == 1) named_bar_sync(1, NCONS);
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
@@ -478,70 +581,29 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       }
       const uint8_t* sp = smem + stage * sl.page_stride;
 
-      // ---- channel-wise keys: per page, the operand of the integer MMAs is q_d * s_d in 24-bit fixed point
-      // (scale from max|q| of the head times the page's largest channel scale).  Each warp makes the operands of
-      // its own slots, all warps exchange them through shared memory; sum_d q_d z_d is summed in fp32 the same way.
+      // ---- channel-wise keys: the page's operands come from the preparation warp (stage buffer, `ready` barrier)
       if constexpr (KAXIS == 1) {
-        constexpr int OWN = NR / 4 > 0 ? NR / 4 : 1;
-        const int buf = 2 * grp + (page_no & 1);
-        if (!aborted && !tail_k) {
-          const uint32_t* km = reinterpret_cast<const uint32_t*>(sp + K_META_OFF);
-          float smax = 0.f;
-          if (4 * lane < D) {
-            const uint4 mm = *reinterpret_cast<const uint4*>(km + 4 * lane);
-            smax = fmaxf(fmaxf(meta_s(mm.x), meta_s(mm.y)), fmaxf(meta_s(mm.z), meta_s(mm.w)));
-          }
-#pragma unroll
-          for (int off = 1; off < 32; off <<= 1) smax = fmaxf(smax, __shfl_xor_sync(FULL, smax, off));
-#pragma unroll
-          for (int nh = 0; nh < NH; ++nh) {
-            const int hb = (gid >> 1) + 4 * nh;
-            const float am = amaxB[nh] * smax;
-            const float scale = am > 0.f ? kQFix3 / am : 0.f;
-            if (wq == 0 && tid == 0 && (gid & 1) == 0) sHS[buf * 8 + hb] = am > 0.f ? c1 / scale : 0.f;
-            float zsum = 0.f;
-#pragma unroll
-            for (int i = 0; i < OWN; ++i) {
-              const int r = wq * OWN + i;
-              if (r < NR) {
-                const uint4 mm = *reinterpret_cast<const uint4*>(km + 16 * r + 4 * tid);   // (s, z) of 4 channels
-                const float4 qq = *reinterpret_cast<const float4*>(sQ + hb * D + 16 * r + 4 * tid);
-                const uint32_t mw[4] = {mm.x, mm.y, mm.z, mm.w};
-                const float qa[4] = {qq.x, qq.y, qq.z, qq.w};
-                float t[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  const float2 sz = __half22float2(as_h2(mw[j]));
-                  t[j] = qa[j] * sz.x;
-                  zsum = fmaf(qa[j], sz.y, zsum);
-                }
-                uint32_t w0, w1;
-                fixed_point_bytes3(t, scale, gid & 1, w0, w1);
-                sB[(((buf * NH + nh) * 2 + 0) * NR + r) * 32 + lane] = w0;
-                sB[(((buf * NH + nh) * 2 + 1) * NR + r) * 32 + lane] = w1;
-              }
-            }
-            zsum += __shfl_xor_sync(FULL, zsum, 1);
-            zsum += __shfl_xor_sync(FULL, zsum, 2);
-            if (tid == 0 && (gid & 1) == 0 && wq * OWN < NR) sZ[(buf * 8 + hb) * 8 + wq] = zsum;
+        if (!aborted) {
+          const bool got = mbar_wait(bar0 + 8 * (2 * stages + stage), phase, wait_ns);
+          if (!__all_sync(FULL, got)) {
+            aborted = true;
+            *abort_flag = 1;
+            if (lane == 0) atomicOr(c.status, KVQ_STATUS_DEVICE_TIMEOUT);
           }
         }
-        // every warp takes part in the exchange barrier of a full page, also after a timeout
-        if (!tail_k) named_bar_sync(2 + grp, 128);
-        if (!aborted && !tail_k) {
-          constexpr int NWR = (NR / OWN < 4) ? NR / OWN : 4;        // warps that contributed
+        if (!aborted) {
+          constexpr int CSB = NH * 2 * NR * 32 * 4 + 64;
+          const uint32_t* ops = reinterpret_cast<const uint32_t*>(smem + sl.chan_off + stage * CSB);
+          const float* opf = reinterpret_cast<const float*>(ops + NH * 2 * NR * 32);
 #pragma unroll
           for (int nh = 0; nh < NH; ++nh) {
 #pragma unroll
             for (int nt = 0; nt < NTK; ++nt) {
 #pragma unroll
-              for (int r = 0; r < NR; ++r) qB[nh][nt][r] = sB[(((buf * NH + nh) * 2 + nt) * NR + r) * 32 + lane];
+              for (int r = 0; r < NR; ++r) qB[nh][nt][r] = ops[((nh * 2 + nt) * NR + r) * 32 + lane];
             }
-            float z = 0.f;
-#pragma unroll
-            for (int w = 0; w < NWR; ++w) z += sZ[(buf * 8 + tid + 4 * nh) * 8 + w];
-            zq[nh] = c1 * z;
-            hs[nh] = sHS[buf * 8 + tid + 4 * nh];
+            zq[nh] = opf[tid + 4 * nh];
+            hs[nh] = opf[8 + tid + 4 * nh];
           }
         }
       }
@@ -563,26 +625,21 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
             vld[u][0] = !MASKED || tok0 < nv;
             vld[u][1] = !MASKED || tok0 + 8 < nv;
             if (KAXIS == 1 && tail_k) {
-              // tokens of the incomplete block: fp16 keys from the tail against q as fp16 high + low parts;
-              // column gid of the operand = (head gid/2 + 4 nh, part gid%2), so lane columns 2 tid, 2 tid + 1 are the
-              // two parts of head tid + 4 nh
+              // tokens of the incomplete block: fp16 keys from the tail against q as fp16 high + low parts (operand
+              // column gid = (head gid/2 + 4 nh, part gid%2), so lane columns 2 tid, 2 tid + 1 are the two parts of
+              // head tid + 4 nh)
               const uint16_t* tl = c.k_tail + ((size_t)stream * kPageTokens + tok0) * D;
 #pragma unroll
               for (int nh = 0; nh < NH; ++nh) {
-                const int hb = (gid >> 1) + 4 * nh;
                 float S[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                 for (int r = 0; r < NR; ++r) {
                   uint2 ra = make_uint2(0u, 0u), rb = make_uint2(0u, 0u);
                   if (vld[u][0]) ra = *reinterpret_cast<const uint2*>(tl + 16 * r + 4 * tid);
                   if (vld[u][1]) rb = *reinterpret_cast<const uint2*>(tl + 8 * D + 16 * r + 4 * tid);
-                  const float4 qq = *reinterpret_cast<const float4*>(sQ + hb * D + 16 * r + 4 * tid);
-                  uint32_t h0, l0_, h1, l1_;
-                  split_h2(qq.x, qq.z, h0, l0_);
-                  split_h2(qq.y, qq.w, h1, l1_);
                   const uint32_t a0 = __byte_perm(ra.x, ra.y, 0x5410), a1 = __byte_perm(rb.x, rb.y, 0x5410);
                   const uint32_t a2 = __byte_perm(ra.x, ra.y, 0x7632), a3 = __byte_perm(rb.x, rb.y, 0x7632);
-                  mma16816(S, a0, a1, a2, a3, (gid & 1) ? l0_ : h0, (gid & 1) ? l1_ : h1);
+                  mma16816(S, a0, a1, a2, a3, qB[nh][0][r], qB[nh][NTK - 1][r]);    // q's fp16 parts, made by the preparation warp
                 }
                 L[u][0][nh] = c1 * (S[0] + S[1]);
                 L[u][1][nh] = c1 * (S[2] + S[3]);
@@ -909,14 +966,15 @@ int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, 
                     void* out, int out_dtype, unsigned long long call_id, unsigned long long wait_ns, long long skip_x,
                     cudaStream_t stream) {
   const int budget = (227 * 1024) / MINB - 1024;            // shared memory per CTA for MINB resident CTAs per SM
-  int stages = (budget - smem_layout(0, 0, NW, g.B, D, NH, KAXIS == 1).total) / ((g.page_bytes + 127) & ~127);
-  if (stages > 16) stages = 16;
+  int stages = (budget - smem_layout(0, 0, NW, g.B, D, NH, KAXIS == 1).total) /
+               (((g.page_bytes + 127) & ~127) + (KAXIS == 1 ? chan_stage_bytes(D, NH) : 0));
+  if (stages > (KAXIS == 1 ? 10 : 16)) stages = KAXIS == 1 ? 10 : 16;      // 32 barriers: two or three per stage
   if (stages < 2 || stages < NW / 4) return KVQ_ERR_UNSUPPORTED;
   const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, g.B, D, NH, KAXIS == 1);
   auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
     return KVQ_ERR_CUDA_LAUNCH;
-  kern<<<148 * MINB, (NW + 1) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap,
+  kern<<<148 * MINB, (NW + 1 + (KAXIS == 1 ? 1 : 0)) * 32, sl.total, stream>>>(g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap,
                                                          stages, out, out_dtype, call_id, wait_ns, skip_x);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
