@@ -17,6 +17,14 @@ int kvq_debug_decode_generic(const kvq_config* cfg, const kvq_cache* cache, cons
                              int32_t out_dtype, float softmax_scale, void* workspace, size_t workspace_bytes,
                              void* cuda_stream);
 
+/* kvq_decode_attention_rows through a chosen implementation of the fast path: impl 0 = the library's own
+ * choice, 1 = the warp-level integer-MMA kernel, 2 = the tcgen05 / tensor-memory kernel
+ * (KVQ_ERR_UNSUPPORTED where that kernel does not serve the configuration).  Lets the tests hold both
+ * kernels against the oracle on the same cache and the benchmark time them side by side. */
+int kvq_debug_decode_impl(const kvq_config* cfg, const kvq_cache* cache, const void* q, int32_t n_rows, void* out,
+                          int32_t out_dtype, float softmax_scale, void* workspace, size_t workspace_bytes,
+                          int32_t impl, void* cuda_stream);
+
 /* kvq_decode_attention on the fast path with every device-side wait limited to wait_us microseconds
  * (1 .. 100000) and the copy of flat page number skip_page (counted over all streams in (batch, kv-head, page)
  * order; -1: none) never issued.  The warps that wait for that page give up after wait_us, set

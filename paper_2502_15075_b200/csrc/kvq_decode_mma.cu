@@ -78,6 +78,11 @@ int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* ou
     int rc = launch_decode_window(g, c, q, out, out_dtype, c1, ws, s_cap, stream);
     if (rc != KVQ_OK) return rc;
   }
+  const bool tc_ok = decode_tc_supported(g, c);
+  if (dbg.fast_impl == 2 && !tc_ok) return KVQ_ERR_UNSUPPORTED;
+  if (tc_ok && dbg.fast_impl == 2)
+    return launch_decode_tc(g, c, q, c1, ws, s_cap, out, out_dtype, next_call_id(),
+                            dbg.wait_us ? 1000ull * dbg.wait_us : mma::kWaitTimeoutNs, dbg.skip_page, stream);
   return pick(g, c, q, c1, ws, s_cap, out, out_dtype, dbg, stream, false, &grid);
 }
 

@@ -8,27 +8,6 @@
 namespace kvq {
 namespace mma {
 
-constexpr int kMaxBatchFlat = 1024;   // the flat partition keeps a per-batch prefix in shared memory
-
-// Flat split of all pages over the grid.
-struct FlatPlan {
-  long long N;       // total pages over all streams
-  int c_eff;         // CTAs that take part
-  __device__ __forceinline__ int cta_of(long long x) const { return (int)(((x + 1) * c_eff - 1) / N); }
-  __device__ __forceinline__ long long lo(int c) const { return (long long)c * N / c_eff; }
-};
-
-__device__ __forceinline__ FlatPlan make_plan(long long N, int pages_max, int grid, int s_cap) {
-  FlatPlan p;
-  p.N = N;
-  long long cap = pages_max > 0 ? (long long)(s_cap - 1) * N / pages_max : 0;
-  long long ce = grid;
-  if (ce > N) ce = N;
-  if (ce > cap) ce = cap;
-  p.c_eff = (int)ce;
-  return p;
-}
-
 // Shared-memory carve-up (dynamic): ring | barriers | prefix | misc | per-warp fp32 masters | (m, l) | channel-wise scratch
 struct SmemLayout {
   int page_stride, ring_bytes, bar_off, pref_off, misc_off, master_off, ml_off, chan_off, total;
@@ -80,24 +59,6 @@ __device__ __forceinline__ uint32_t fixed_point_limb(const float (&t)[4], float 
     qsum += Q;
   }
   return w;
-}
-
-// Split partials of a stream are merged by whichever CTA publishes the last of them: after storing its partial a
-// CTA counts itself in the stream's word, which holds (launch id << 24 | count).  A word that carries another id
-// (stale contents, an earlier launch) restarts at 1, so the workspace needs no initialisation; the CTA that
-// reaches the expected count merges and clears the word, so that a replayed launch with the same id starts clean.
-__device__ __forceinline__ unsigned tagged_count(unsigned long long* p, unsigned long long id40) {
-  unsigned long long old = *reinterpret_cast<volatile unsigned long long*>(p);
-  while (true) {
-    const unsigned long long nw = ((old >> 24) == id40) ? old + 1ull : ((id40 << 24) | 1ull);
-    const unsigned long long r = atomicCAS(p, old, nw);
-    if (r == old) return (unsigned)(nw & 0xFFFFFFull);
-    old = r;
-  }
-}
-// Offset (in floats) of the count words behind the partials: [streams] 64-bit words.
-__host__ __device__ inline size_t tag_offset_floats(int streams, int s_cap, int G, int D) {
-  return ((size_t)streams * s_cap * G * (D + 2) + 3) & ~(size_t)3;
 }
 
 constexpr float kQFix = 32512.0f;          // largest |Q| of the 16-bit fixed-point q (hi limb stays within +-127)

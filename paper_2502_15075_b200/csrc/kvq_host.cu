@@ -268,13 +268,16 @@ int kvq_decode_attention_rows(const kvq_config* cfg, const kvq_cache* cache, con
 // ---------------------------------------------------------------------------
 static int decode_with(const kvq_config* cfg, const kvq_cache* cache, const void* q, void* out, int32_t out_dtype,
                        float softmax_scale, void* workspace, size_t workspace_bytes, void* cuda_stream,
-                       const DecodeDebug& dbg) {
+                       const DecodeDebug& dbg, int n_rows = 1) {
   Geom g;
   CachePtrs c;
   int rc = make_geom(cfg, &g);
   if (rc != KVQ_OK) return rc;
   rc = make_cache(g, cache, &c);
   if (rc != KVQ_OK) return rc;
+  if (n_rows * g.G > kMaxGroupHeads) return KVQ_ERR_UNSUPPORTED;
+  g.rows = n_rows;
+  if (n_rows > 1 && !decode_mma_supported(g)) return KVQ_ERR_UNSUPPORTED;
   if (!q || !out || !workspace) return KVQ_ERR_INVALID_ARG;
   if (out_dtype != KVQ_FP16 && out_dtype != KVQ_BF16 && out_dtype != KVQ_FP32) return KVQ_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out) || !aligned16(workspace)) return KVQ_ERR_MISALIGNED;
@@ -289,6 +292,15 @@ int kvq_debug_decode_generic(const kvq_config* cfg, const kvq_cache* cache, cons
   DecodeDebug dbg;
   dbg.force_generic = true;
   return decode_with(cfg, cache, q, out, out_dtype, softmax_scale, workspace, workspace_bytes, cuda_stream, dbg);
+}
+
+int kvq_debug_decode_impl(const kvq_config* cfg, const kvq_cache* cache, const void* q, int32_t n_rows, void* out,
+                          int32_t out_dtype, float softmax_scale, void* workspace, size_t workspace_bytes,
+                          int32_t impl, void* cuda_stream) {
+  if (impl < 0 || impl > 2 || n_rows < 1) return KVQ_ERR_INVALID_ARG;
+  DecodeDebug dbg;
+  dbg.fast_impl = impl;
+  return decode_with(cfg, cache, q, out, out_dtype, softmax_scale, workspace, workspace_bytes, cuda_stream, dbg, n_rows);
 }
 
 int kvq_debug_decode_stall(const kvq_config* cfg, const kvq_cache* cache, const void* q, void* out, int32_t out_dtype,

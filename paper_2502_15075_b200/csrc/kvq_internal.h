@@ -20,6 +20,7 @@ size_t decode_workspace_bytes(const Geom& g);
 // Test hooks of a decode launch (all zero / -1 in the product path).
 struct DecodeDebug {
   bool force_generic = false;    // run the plain-ALU kernel whatever the configuration
+  int fast_impl = 0;             // fast path: 0 = the library's choice, 1 = the warp-level MMA kernel, 2 = the tcgen05 kernel
   uint32_t wait_us = 0;          // limit of every device-side wait in microseconds (0: the default, 2 s)
   long long skip_page = -1;      // flat page index whose copy is never issued (-1: none)
 };
@@ -45,4 +46,9 @@ int launch_decode_window(const Geom& g, const CachePtrs& c, const void* q, void*
                          float scale_log2e, float* ws, int s_cap, cudaStream_t stream);
 int launch_decode_mma(const Geom& g, const CachePtrs& c, const void* q, void* out, int out_dtype,
                       float scale_log2e, float* ws, const DecodeDebug& dbg, cudaStream_t stream);
+// tcgen05 / tensor-memory variant of the fast path (same split, workspace and merge)
+bool decode_tc_supported(const Geom& g, const CachePtrs& c);
+int launch_decode_tc(const Geom& g, const CachePtrs& c, const void* q, float scale_log2e, float* ws, int s_cap,
+                     void* out, int out_dtype, unsigned long long call_id, unsigned long long wait_ns, long long skip_x,
+                     cudaStream_t stream);
 }  // namespace kvq
