@@ -4,7 +4,7 @@
 // 2- or 4-bit values and up to four (virtual) query heads per KV head.
 //
 // One CTA = four consumer warps (thread x = token x of the page for QK^T and the softmax, = channel x for PV),
-// a producer warp and an MMA warp; two CTAs per SM, each with 256 columns of tensor memory.
+// a producer warp and an MMA warp; two or three CTAs per SM, each with 128 columns of tensor memory.
 //  * The producer streams whole 128-token pages into a shared-memory ring with tiled TMA copies (the page seen
 //    as rows of 64 bytes, 64-byte swizzle: row-per-thread 16-byte reads are then free of bank conflicts).
 //  * A consumer thread turns its token's packed key row into the A operand of QK^T and stores it to tensor
@@ -36,11 +36,11 @@ using namespace mma;
 
 constexpr int kThreads = 192;        // warps 0-3 consumers, 4 producer, 5 MMA issue + tensor-memory allocation
 constexpr int kNCons = 128;
-constexpr int kTmemCols = 256;       // per CTA; two CTAs per SM share the 512 columns
-constexpr int kColKa = 0;            // key operand, two buffers of 32 columns
-constexpr int kColVa = 64;           // value operand, two buffers of 32 columns
-constexpr int kColS = 128;           // logits accumulators, two buffers of 16 columns
-constexpr int kColO = 160;           // output accumulator, 16 columns
+constexpr int kTmemCols = 128;       // per CTA; up to four CTAs per SM share the 512 columns
+constexpr int kColKa = 0;            // key operand, 32 columns
+constexpr int kColVa = 32;           // value operand, two buffers of 32 columns
+constexpr int kColS = 96;            // logits accumulator, 16 columns
+constexpr int kColO = 112;           // output accumulator, 16 columns
 constexpr float kQFixTc = 32512.0f;  // largest |Q| of the 16-bit fixed-point q
 constexpr float kPOne = 2147483648.0f;   // 2^31: the softmax weights are 31-bit fixed point
 constexpr float kHeadroomTc = 6.0f;
@@ -151,8 +151,8 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, uns
   }
 }
 
-template <int KB, int VB>
-__global__ void __launch_bounds__(kThreads, 2)
+template <int KB, int VB, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB)
 decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
                  float* __restrict__ ws, int s_cap, int stages, int box_rows, void* __restrict__ out, int out_dtype,
                  unsigned long long call_id, unsigned long long wait_ns, long long skip_x) {
@@ -181,7 +181,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, 
 
   const int tid_ = threadIdx.x, lane = tid_ & 31, warp = tid_ >> 5;
   const int B = g.B, Hkv = g.Hkv, Gq = g.G, G = g.G * g.rows;
-  // barrier map: full[s], empty[s], then ops_ready[2], s_ready[2], p_ready[2], pv_done[2], drain
+  // barrier map: full[s], empty[s], then k_ready, s_ready, p_ready[2], pv_done[2], drain
   const uint32_t bar0 = smem_u32(bars);
   const uint32_t bar_ops = bar0 + 8 * (2 * stages), bar_s = bar_ops + 16, bar_p = bar_ops + 32, bar_pv = bar_ops + 48,
                  bar_drain = bar_ops + 64;
@@ -213,9 +213,9 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, 
       mbar_init(bar0 + 8 * s, 1);
       mbar_init(bar0 + 8 * (stages + s), 4);
     }
+    mbar_init(bar_ops, 4);
+    mbar_init(bar_s, 1);
     for (int k = 0; k < 2; ++k) {
-      mbar_init(bar_ops + 8 * k, 4);
-      mbar_init(bar_s + 8 * k, 1);
       mbar_init(bar_p + 8 * k, 4);
       mbar_init(bar_pv + 8 * k, 1);
     }
@@ -313,39 +313,28 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, 
   } else if (warp == 5) {
     // =========================================================== MMA issue
     if (lane == 0 && active) {
-      int itb = 0;
       bool ok = true;
-      for (long long x = x_lo; x < x_hi && ok;) {
-        const int seg_pages = (int)min((long long)(pages_b - page), x_hi - x);
-        for (int i = 0; i <= seg_pages && ok; ++i) {
-          if (i < seg_pages) {
-            const int it = itb + i, buf = it & 1;
-            ok = wait_or_abort(bar_ops + 8 * buf, (it >> 1) & 1, wait_ns, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
+      const int n_pages_cta = (int)(x_hi - x_lo);
+      for (int it = 0; it < n_pages_cta; ++it) {
+        const int buf = it & 1;
+        ok = wait_or_abort(bar_ops, it & 1, wait_ns, abort_flag);               // the page's key operand is in tensor memory
+        if (!ok) break;
+        tc_fence_after();
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              tc_mma_i8_ts(tmem + kColS + 16 * buf, tmem + kColKa + 32 * buf + 8 * kk,
-                           smem_desc(smem_u32(sQop) + 512 * kk, 256, 128), kIdescQK, kk > 0 ? 1u : 0u);
-            tc_commit(bar_s + 8 * buf);
-          }
-          if (i >= 1) {
-            const int it = itb + i - 1, buf = it & 1;
-            ok = wait_or_abort(bar_p + 8 * buf, (it >> 1) & 1, wait_ns, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t fresh = (uint32_t)sFresh[buf];
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_i8_ts(tmem + kColS, tmem + kColKa + 8 * kk, smem_desc(smem_u32(sQop) + 512 * kk, 256, 128), kIdescQK,
+                       kk > 0 ? 1u : 0u);
+        tc_commit(bar_s);
+        ok = wait_or_abort(bar_p + 8 * buf, (it >> 1) & 1, wait_ns, abort_flag);   // value operand and weights are ready
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t fresh = (uint32_t)sFresh[buf];
 #pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-              tc_mma_i8_ts(tmem + kColO, tmem + kColVa + 32 * buf + 8 * kk,
-                           smem_desc(smem_u32(sPop) + 2048 * buf + 512 * kk, 128, 128), kIdescPV,
-                           (kk > 0 || !fresh) ? 1u : 0u);
-            tc_commit(bar_pv + 8 * buf);
-          }
-        }
-        itb += seg_pages;
-        x += seg_pages;
-        advance(seg_pages);
+        for (int kk = 0; kk < 4; ++kk)
+          tc_mma_i8_ts(tmem + kColO, tmem + kColVa + 32 * buf + 8 * kk,
+                       smem_desc(smem_u32(sPop) + 2048 * buf + 512 * kk, 128, 128), kIdescPV,
+                       (kk > 0 || !fresh) ? 1u : 0u);
+        tc_commit(bar_pv + 8 * buf);
       }
       if (!ok) {
         *abort_flag = 1;
@@ -463,7 +452,6 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, 
       float sscale = kPOne / 9.094947e-13f;       // 2^31 / s_lim, s_lim a power of two above every value scale so far
       bool o_dirty = false;
       int since_fold = 0;
-      uint32_t km_cur = 0, vm_cur = 0, km_nxt = 0, vm_nxt = 0;
       int lim_hv[4];
 #pragma unroll
       for (int hv = 0; hv < 4; ++hv) lim_hv[hv] = n_all - (g.rows - 1 - min(hv / Gq, g.rows - 1));
@@ -490,70 +478,69 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, 
         since_fold = 0;
       };
 
-      for (int i = 0; i <= seg_pages; ++i) {
-        // ------------------------------------------------------------ operands of page i
-        if (i < seg_pages) {
-          const int itp = it + i, buf = itp & 1;
-          cons_wait(bar0 + 8 * stage, phase);
-          if (itp >= 2) cons_wait(bar_pv + 8 * buf, ((itp - 2) >> 1) & 1);      // the buffers' last readers are done
-          tc_fence_after();
-          const uint8_t* sp = smem + stage * PAGE;
-          uint32_t r[32];
-          if constexpr (KB == 4) {
+      for (int i = 0; i < seg_pages; ++i) {
+        const int itp = it + i, buf = itp & 1;
+        const int pg = page + i;                                  // page index inside the sequence
+        const int nv = min(kPageTokens, n_tok - pg * kPageTokens);
+        const int tokg = pg * kPageTokens + x_;
+        // ------------------------------------------------------------ key operand (thread = token); the earlier
+        // page's QK^T is complete and its logits are read: this thread waited for them in its softmax
+        cons_wait(bar0 + 8 * stage, phase);
+        tc_fence_after();
+        const uint8_t* sp = smem + stage * PAGE;
+        uint32_t r[32];
+        if constexpr (KB == 4) {
+#pragma unroll
+          for (int cch = 0; cch < 4; ++cch) {
+            const uint4 w = *reinterpret_cast<const uint4*>(sp + swz64(x_ * 64 + cch * 16));
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+            for (int wd = 0; wd < 4; ++wd) {
+              r[cch * 8 + wd * 2] = ww[wd];
+              r[cch * 8 + wd * 2 + 1] = ww[wd] & 0xF0F0F0F0u;
+            }
+          }
+        } else {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
 #pragma unroll
             for (int cch = 0; cch < 4; ++cch) {
-              const uint4 w = *reinterpret_cast<const uint4*>(sp + swz64(x_ * 64 + cch * 16));
-              const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-              for (int wd = 0; wd < 4; ++wd) {
-                r[cch * 8 + wd * 2] = ww[wd];
-                r[cch * 8 + wd * 2 + 1] = ww[wd] & 0xF0F0F0F0u;
-              }
-            }
-          } else {
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-#pragma unroll
-              for (int cch = 0; cch < 4; ++cch) {
-                const uint4 w = *reinterpret_cast<const uint4*>(sp + swz64(x_ * 128 + half * 64 + cch * 16));
-                r[half * 16 + cch * 4 + 0] = w.x; r[half * 16 + cch * 4 + 1] = w.y;
-                r[half * 16 + cch * 4 + 2] = w.z; r[half * 16 + cch * 4 + 3] = w.w;
-              }
+              const uint4 w = *reinterpret_cast<const uint4*>(sp + swz64(x_ * 128 + half * 64 + cch * 16));
+              r[half * 16 + cch * 4 + 0] = w.x; r[half * 16 + cch * 4 + 1] = w.y;
+              r[half * 16 + cch * 4 + 2] = w.z; r[half * 16 + cch * 4 + 3] = w.w;
             }
           }
-          tmem_st32(lane_taddr + kColKa + 32 * buf, r);
-#pragma unroll
-          for (int blk = 0; blk < 4; ++blk) {
-#pragma unroll
-            for (int tq = 0; tq < 4; ++tq) {
-              const uint2 w = *reinterpret_cast<const uint2*>(
-                  sp + swz64(V_CODES_OFF + blk * V_BLOCK + v_mw * 512 + (4 * v_gq + tq) * 16 + 8 * v_rh));
-              r[(blk * 4 + tq) * 2 + 0] = w.x & v_mask;
-              r[(blk * 4 + tq) * 2 + 1] = w.y & v_mask;
-            }
-          }
-          tmem_st32(lane_taddr + kColVa + 32 * buf, r);
-          km_nxt = *reinterpret_cast<const uint32_t*>(sp + swz64(K_META_OFF + 4 * x_));
-          vm_nxt = *reinterpret_cast<const uint32_t*>(sp + swz64(V_META_OFF + 4 * x_));
-          tc_wait_st();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(bar_ops + 8 * buf);
-            mbar_arrive(bar0 + 8 * (stages + stage));
-          }
-          if (++stage == stages) { stage = 0; phase ^= 1; }
         }
-        // ------------------------------------------------------------ softmax of page i - 1
-        if (i >= 1) {
-          const int itp = it + i - 1, buf = itp & 1;
-          const int pg = page + i - 1;                              // page index inside the sequence
-          const int nv = min(kPageTokens, n_tok - pg * kPageTokens);
-          const int tokg = pg * kPageTokens + x_;
-          cons_wait(bar_s + 8 * buf, (itp >> 1) & 1);
+        tmem_st32(lane_taddr + kColKa, r);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_ops);
+        // ------------------------------------------------------------ value operand (thread = channel), while QK^T runs
+        const uint32_t km_cur = *reinterpret_cast<const uint32_t*>(sp + swz64(K_META_OFF + 4 * x_));
+        const uint32_t vm_cur = *reinterpret_cast<const uint32_t*>(sp + swz64(V_META_OFF + 4 * x_));
+#pragma unroll
+        for (int blk = 0; blk < 4; ++blk) {
+#pragma unroll
+          for (int tq = 0; tq < 4; ++tq) {
+            const uint2 w = *reinterpret_cast<const uint2*>(
+                sp + swz64(V_CODES_OFF + blk * V_BLOCK + v_mw * 512 + (4 * v_gq + tq) * 16 + 8 * v_rh));
+            r[(blk * 4 + tq) * 2 + 0] = w.x & v_mask;
+            r[(blk * 4 + tq) * 2 + 1] = w.y & v_mask;
+          }
+        }
+        if (itp >= 2) cons_wait(bar_pv + 8 * buf, ((itp - 2) >> 1) & 1);       // the buffer's last reader is done
+        tc_fence_after();
+        tmem_st32(lane_taddr + kColVa + 32 * buf, r);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar0 + 8 * (stages + stage));               // the page's bytes are all in registers
+        if (++stage == stages) { stage = 0; phase ^= 1; }
+        // ------------------------------------------------------------ softmax (thread = token)
+        {
+          cons_wait(bar_s, itp & 1);
           tc_fence_after();
           uint32_t a[16];
-          tmem_ld16(lane_taddr + kColS + 16 * buf, a);
+          tmem_ld16(lane_taddr + kColS, a);
           tc_wait_ld();
           const bool tok_ok = x_ < nv;
           const float2 km = __half22float2(as_h2(tok_ok ? km_cur : 0u));
@@ -616,14 +603,13 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, 
           }
           *reinterpret_cast<uint4*>(sPop + 2048 * buf + 16 * p_row) = pw;
           fence_async_smem();
+          tc_wait_st();                          // the value operand stored above
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_p + 8 * buf);
           o_dirty = true;
           ++since_fold;
         }
-        km_cur = km_nxt;
-        vm_cur = vm_nxt;
       }
       it += seg_pages;
 
@@ -768,7 +754,7 @@ static int make_page_map(const Geom& g, const CachePtrs& c, int box_rows, CUtens
   return r == CUDA_SUCCESS ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
 
-template <int KB, int VB>
+template <int KB, int VB, int MINB>
 static int launch_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap, void* out,
                        int out_dtype, unsigned long long call_id, unsigned long long wait_ns, long long skip_x,
                        cudaStream_t stream) {
@@ -777,18 +763,21 @@ static int launch_inst(const Geom& g, const CachePtrs& c, const void* q, float c
   const int rows64 = g.page_bytes / 64;
   const int box_rows = rows64 <= 256 ? rows64 : rows64 / 2;
   if (g.page_bytes % 1024 || (box_rows * 64) % 512 || box_rows > 256) return KVQ_ERR_UNSUPPORTED;
-  const int budget = (227 * 1024) / 2 - 1024;
+  const int budget = (227 * 1024) / MINB - 1024;
   int stages = (budget - smem_tc(0, 0, g.B).total) / g.page_bytes;
   if (stages > 12) stages = 12;
   if (stages < 2) return KVQ_ERR_UNSUPPORTED;
-  const SmemTc sl = smem_tc(g.page_bytes, stages, g.B);
+  SmemTc sl = smem_tc(g.page_bytes, stages, g.B);
+  // A CTA allocates 128 of the SM's 512 tensor-memory columns and would wait for ever as the fifth CTA on an SM:
+  // asking for more than a fifth of the shared memory keeps the resident CTAs at four or fewer.
+  if (sl.total < 48 * 1024) sl.total = 48 * 1024;
   CUtensorMap tm;
   int rc = make_page_map(g, c, box_rows, &tm);
   if (rc != KVQ_OK) return rc;
-  auto kern = decode_tc_kernel<KB, VB>;
+  auto kern = decode_tc_kernel<KB, VB, MINB>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, sl.total) != cudaSuccess)
     return KVQ_ERR_CUDA_LAUNCH;
-  kern<<<148 * 2, kThreads, sl.total, stream>>>(tm, g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap, stages, box_rows,
+  kern<<<148 * MINB, kThreads, sl.total, stream>>>(tm, g, c, static_cast<const uint16_t*>(q), c1, ws, s_cap, stages, box_rows,
                                                out, out_dtype, call_id, wait_ns, skip_x);
   return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
 }
@@ -801,18 +790,16 @@ bool decode_tc_supported(const Geom& g, const CachePtrs& c) {
   if (g.G * g.rows > 4 || g.B > mma::kMaxBatchFlat) return false;
   if (c.k_signs != nullptr) return false;                       // rotated keys: the warp-level kernel
   if ((long long)g.B * g.Hkv * g.n_pages > 0x7fffffffLL) return false;
-  // two CTAs per SM at most (each owns half of the tensor memory): a CTA must need more than a third of the
-  // shared memory, which the ring guarantees for these page sizes
   return true;
 }
 
 int launch_decode_tc(const Geom& g, const CachePtrs& c, const void* q, float c1, float* ws, int s_cap, void* out,
                      int out_dtype, unsigned long long call_id, unsigned long long wait_ns, long long skip_x,
                      cudaStream_t stream) {
-  if (g.kb == 4 && g.vb == 2) return tc::launch_inst<4, 2>(g, c, q, c1, ws, s_cap, out, out_dtype, call_id, wait_ns, skip_x, stream);
-  if (g.kb == 4 && g.vb == 4) return tc::launch_inst<4, 4>(g, c, q, c1, ws, s_cap, out, out_dtype, call_id, wait_ns, skip_x, stream);
-  if (g.kb == 8 && g.vb == 4) return tc::launch_inst<8, 4>(g, c, q, c1, ws, s_cap, out, out_dtype, call_id, wait_ns, skip_x, stream);
-  if (g.kb == 8 && g.vb == 2) return tc::launch_inst<8, 2>(g, c, q, c1, ws, s_cap, out, out_dtype, call_id, wait_ns, skip_x, stream);
+  if (g.kb == 4 && g.vb == 2) return tc::launch_inst<4, 2, 3>(g, c, q, c1, ws, s_cap, out, out_dtype, call_id, wait_ns, skip_x, stream);
+  if (g.kb == 4 && g.vb == 4) return tc::launch_inst<4, 4, 3>(g, c, q, c1, ws, s_cap, out, out_dtype, call_id, wait_ns, skip_x, stream);
+  if (g.kb == 8 && g.vb == 4) return tc::launch_inst<8, 4, 2>(g, c, q, c1, ws, s_cap, out, out_dtype, call_id, wait_ns, skip_x, stream);
+  if (g.kb == 8 && g.vb == 2) return tc::launch_inst<8, 2, 2>(g, c, q, c1, ws, s_cap, out, out_dtype, call_id, wait_ns, skip_x, stream);
   return KVQ_ERR_UNSUPPORTED;
 }
 
