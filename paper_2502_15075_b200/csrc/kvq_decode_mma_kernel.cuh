@@ -278,6 +278,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       int it = 0, stage = 0;
       uint32_t phase = 1;                // parity of the previous round of `empty`
       bool ok = true;
+      const uint64_t policy = l2_evict_first_policy();
       for (long long x = x_lo; x < x_hi; ++x, ++it) {
         if (it >= stages) {
           ok = mbar_wait(bar0 + 8 * (stages + stage), phase, wait_ns);
@@ -287,7 +288,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
         const uint32_t fb = bar0 + 8 * stage;
         if (x != skip_x) {          // (skip_x: test hook - a page that never arrives makes the consumers' bounded wait expire)
           mbar_expect_tx(fb, (uint32_t)g.page_bytes);
-          bulk_load(ring + stage * sl.page_stride, src, (uint32_t)g.page_bytes, fb);
+          bulk_load(ring + stage * sl.page_stride, src, (uint32_t)g.page_bytes, fb, policy);
         }
         if (++stage == stages) { stage = 0; phase ^= 1; }
         if (++page == pages_b) {
@@ -929,7 +930,9 @@ int launch_mma_inst(const Geom& g, const CachePtrs& c, const void* q, float c1, 
   const int budget = (227 * 1024) / MINB - 1024;            // shared memory per CTA for MINB resident CTAs per SM
   int stages = (budget - smem_layout(0, 0, NW, g.B, D, NH, KAXIS == 1).total) /
                (((g.page_bytes + 127) & ~127) + (KAXIS == 1 ? chan_stage_bytes(D, NH) : 0));
-  if (stages > (KAXIS == 1 ? 10 : 16)) stages = KAXIS == 1 ? 10 : 16;      // 32 barriers: two or three per stage
+  // Deeper rings do not help: the kernel is bound by its arithmetic, not by copy latency, and more bytes in
+  // flight cost DRAM efficiency (8B shape, K4V2: 5 stages 95 us, 3-4 stages 91-92 us, 2 stages 97 us).
+  if (stages > 4) stages = 4;
   if (stages < 2 || stages < NW / 4) return KVQ_ERR_UNSUPPORTED;
   const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, g.B, D, NH, KAXIS == 1);
   auto kern = decode_mma_kernel<D, KB, VB, KAXIS, NGK, NGV, NH, NW, MINB>;
