@@ -68,9 +68,11 @@ __host__ __device__ inline SmemTc smem_tc(int page_bytes, int stages, int batch)
 }
 
 // ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-               ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int c0, int c1, int c2, uint32_t bar,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -283,6 +285,7 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, 
       int it = 0, stage = 0;
       uint32_t phase = 1;
       bool ok = true;
+      const uint64_t policy = l2_evict_first_policy();
       for (long long x = x_lo; x < x_hi; ++x, ++it) {
         if (it >= stages) {
           ok = wait_or_abort(bar0 + 8 * (stages + stage), phase, wait_ns, abort_flag);
@@ -293,8 +296,8 @@ decode_tc_kernel(const __grid_constant__ CUtensorMap tmap, Geom g, CachePtrs c, 
         if (x != skip_x) {      // (skip_x: test hook - a page that never arrives makes the consumers' bounded wait expire)
           mbar_expect_tx(fb, (uint32_t)PAGE);
           const uint32_t dst = ring + stage * PAGE;
-          tma_load_3d(dst, &tmap, 0, 0, gpage, fb);
-          if (box_rows * 64 < PAGE) tma_load_3d(dst + box_rows * 64, &tmap, 0, box_rows, gpage, fb);
+          tma_load_3d(dst, &tmap, 0, 0, gpage, fb, policy);
+          if (box_rows * 64 < PAGE) tma_load_3d(dst + box_rows * 64, &tmap, 0, box_rows, gpage, fb, policy);
         }
         if (++stage == stages) { stage = 0; phase ^= 1; }
         advance(1);
