@@ -95,7 +95,7 @@ __device__ __forceinline__ void quantize_task(const RowSrc& rsrc, int gsz, int l
 #pragma unroll
     for (int f = 0; f < FPB; ++f) {
       raw[k][f] = make_uint4(0u, 0u, 0u, 0u);
-      if (valid) raw[k][f] = *reinterpret_cast<const uint4*>(rsrc.row(tau) + 16 * (FPB * mw + f) + 8 * rh);
+      if (valid) raw[k][f] = __ldcs(reinterpret_cast<const uint4*>(rsrc.row(tau) + 16 * (FPB * mw + f) + 8 * rh));
     }
   }
 
@@ -347,7 +347,7 @@ __device__ __forceinline__ void quantize_task_fast(const RowSrc& rsrc, int gsz, 
 #pragma unroll
       for (int f = 0; f < FPB; ++f) {
         raw[kk][f] = make_uint4(0u, 0u, 0u, 0u);
-        if (valid[kk]) raw[kk][f] = *reinterpret_cast<const uint4*>(rsrc.row(tau) + 16 * (FPB * mw + f) + 8 * rh);
+        if (valid[kk]) raw[kk][f] = __ldcs(reinterpret_cast<const uint4*>(rsrc.row(tau) + 16 * (FPB * mw + f) + 8 * rh));
       }
     }
     // ---- phase 1: minima / maxima of the lane's fields, per token and per set
