@@ -422,6 +422,23 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
         if r:
             deq_ms.append(a.elapsed_time(b_))
     dq_us = stats_us(deq_ms)
+
+    # ---- the two kernels of the fast decode path side by side (decode calls only, layers rotating): the
+    # warp-level integer-MMA kernel, which is the product path, and the tcgen05 / tensor-memory kernel
+    variants = {}
+    for label, impl in (("warp_mma", kvq.IMPL_WARP_MMA), ("tcgen05", kvq.IMPL_TCGEN05)):
+        try:
+            pairs = []
+            for r in range(3 * max(L, 4) + 2):
+                a, b_ = ev(), ev()
+                a.record()
+                kvq.kvq_debug_decode_impl(cfg, caches[r % L], qs[r % L], outs[r % L], ws_buf, impl)
+                b_.record()
+                pairs.append((a, b_))
+            torch.cuda.synchronize()
+            variants[label] = stats_us([a.elapsed_time(b_) for a, b_ in pairs[2:]])
+        except kvq.KvqError as e:
+            variants[label] = {"unsupported": e.code}
     if kvq.kvq_check_status(caches[0]) != 0:
         raise RuntimeError("library reported a status error")
 
@@ -446,7 +463,12 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
                         decode_bytes_per_layer(w, T) + source_bytes_per_layer(w, T), dq_us, peak, peak_src)
 
     cpu = oracle_leg(kvq, w, cfg, caches[0], qs[0], outs[0], oracle_budget_s)
-    kern_per_layer = (2 if w.k_axis == 0 else 3) + 1 + 1      # append (quantize [+ channel-wise K] + bump), decode, dequantize
+    fast_bits = lambda b: b in (2, 4, 8)  # noqa: E731
+    deq_launches = ((1 if w.head_dim == 128 and fast_bits(w.vb) else 0) +
+                    (1 if w.head_dim == 128 and w.k_axis == 0 and fast_bits(w.kb) else 0))
+    deq_launches = deq_launches if deq_launches == 2 else deq_launches + 1        # the general kernel serves what is left
+    # append (quantize [+ channel-wise K] + bump), decode, dequantize (one kernel per side on its fast path)
+    kern_per_layer = (2 if w.k_axis == 0 else 3) + 1 + deq_launches
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "int32 accumulate over 8-bit operands (fp32 softmax and merge)",
@@ -456,7 +478,7 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
             "gpu_launches": L * kern_per_layer * steps,
             "quantize": {"tokens_per_s": world * B * bulk / (q_us["median"] * 1e-6), "us_per_layer_bulk": q_us,
                          "tokens_per_call": B * bulk},
-            "clocks": clocks}
+            "decode_kernels_us": variants, "clocks": clocks}
     if e2e_ms is not None:
         line["e2e"] = {"value": whole_job_gbs(bytes_step, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": L * (2 * k1s[0].numel() * 2 + qs[0].numel() * 2),

@@ -674,6 +674,67 @@ __device__ __forceinline__ void pack_k_rows(const uint8_t* codes, int code_strid
   }
 }
 
+// Channel-wise quantization of one complete 128-token block held as fp16 in shared memory, head_dim 128, 4- or
+// 8-bit codes.  Thread = (token quarter, slice pair rp, channel pair pi): the four channels 32 rp + 2 pi + {0, 1}
+// and 32 rp + 16 + 2 pi + {0, 1}, whose codes share two adjacent bytes (4 bits) or two adjacent byte pairs
+// (8 bits) of every token row.  Minimum and maximum are taken two channels at a time in fp16 (exact), the
+// parameters once per channel, and the codes are written as whole bytes into a shared image of the page's key
+// region, which leaves with 16-byte stores.
+template <int KB>
+__device__ __forceinline__ void kchan_block_fast(const uint16_t* sX, uint8_t* sImg, uint8_t* pg, const Geom& g, int tid) {
+  constexpr int D = 128, ROW = D * KB / 8;
+  const __half2* sX2 = reinterpret_cast<const __half2*>(sX);            // [128][64]
+  __half2* sRed = reinterpret_cast<__half2*>(sImg);                    // [4 quarters][32][4], dead before the image is written
+  const int q = tid >> 5, l32 = tid & 31, rp = l32 >> 3, pi = l32 & 7;
+  const int w_lo = 16 * rp + pi, w_hi = w_lo + 8;
+  const float qmax = (float)((1 << KB) - 1);
+  __half2 mn_lo = sX2[(32 * q) * 64 + w_lo], mx_lo = mn_lo, mn_hi = sX2[(32 * q) * 64 + w_hi], mx_hi = mn_hi;
+#pragma unroll 8
+  for (int t = 32 * q + 1; t < 32 * q + 32; ++t) {
+    const __half2 a = sX2[t * 64 + w_lo], b = sX2[t * 64 + w_hi];
+    mn_lo = __hmin2(mn_lo, a); mx_lo = __hmax2(mx_lo, a);
+    mn_hi = __hmin2(mn_hi, b); mx_hi = __hmax2(mx_hi, b);
+  }
+  sRed[(q * 32 + l32) * 4 + 0] = mn_lo; sRed[(q * 32 + l32) * 4 + 1] = mx_lo;
+  sRed[(q * 32 + l32) * 4 + 2] = mn_hi; sRed[(q * 32 + l32) * 4 + 3] = mx_hi;
+  __syncthreads();
+#pragma unroll
+  for (int qq = 0; qq < 4; ++qq) {
+    mn_lo = __hmin2(mn_lo, sRed[(qq * 32 + l32) * 4 + 0]); mx_lo = __hmax2(mx_lo, sRed[(qq * 32 + l32) * 4 + 1]);
+    mn_hi = __hmin2(mn_hi, sRed[(qq * 32 + l32) * 4 + 2]); mx_hi = __hmax2(mx_hi, sRed[(qq * 32 + l32) * 4 + 3]);
+  }
+  const GroupParams p0 = group_params(__low2float(mn_lo), __low2float(mx_lo), qmax);     // channel 32 rp + 2 pi
+  const GroupParams p1 = group_params(__high2float(mn_lo), __high2float(mx_lo), qmax);   // ... + 1
+  const GroupParams p2 = group_params(__low2float(mn_hi), __low2float(mx_hi), qmax);     // ... + 16
+  const GroupParams p3 = group_params(__high2float(mn_hi), __high2float(mx_hi), qmax);   // ... + 17
+  if (q == 0) {
+    uint32_t* meta = reinterpret_cast<uint32_t*>(pg + g.k_meta_off);
+    const int d0 = 32 * rp + 2 * pi;
+    meta[d0] = p0.meta; meta[d0 + 1] = p1.meta; meta[d0 + 16] = p2.meta; meta[d0 + 17] = p3.meta;
+  }
+  __syncthreads();                       // every thread has read the reduction scratch: the image may overwrite it
+#pragma unroll 4
+  for (int t = 32 * q; t < 32 * q + 32; ++t) {
+    const float2 a = __half22float2(sX2[t * 64 + w_lo]), b = __half22float2(sX2[t * 64 + w_hi]);
+    const uint32_t c0 = code_of_fast(a.x, p0, qmax), c1 = code_of_fast(a.y, p1, qmax);
+    const uint32_t c2 = code_of_fast(b.x, p2, qmax), c3 = code_of_fast(b.y, p3, qmax);
+    if constexpr (KB == 4) {
+      // bytes 2 (pi % 2) + {0, 1} of word rp in chunk pi / 2: low nibble slice 2 rp, high nibble slice 2 rp + 1
+      *reinterpret_cast<uint16_t*>(sImg + t * ROW + (pi >> 1) * 16 + rp * 4 + 2 * (pi & 1)) =
+          (uint16_t)((c0 | (c2 << 4)) | ((c1 | (c3 << 4)) << 8));
+    } else {
+      const int wa = 2 * rp, wb = 2 * rp + 1;                      // words = slices 2 rp and 2 rp + 1
+      *reinterpret_cast<uint16_t*>(sImg + t * ROW + (wa >> 2) * 64 + (pi >> 1) * 16 + (wa & 3) * 4 + 2 * (pi & 1)) =
+          (uint16_t)(c0 | (c1 << 8));
+      *reinterpret_cast<uint16_t*>(sImg + t * ROW + (wb >> 2) * 64 + (pi >> 1) * 16 + (wb & 3) * 4 + 2 * (pi & 1)) =
+          (uint16_t)(c2 | (c3 << 8));
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < kPageTokens * ROW / 16; i += kThreads)
+    reinterpret_cast<uint4*>(pg)[i] = reinterpret_cast<const uint4*>(sImg)[i];
+}
+
 // Channel-wise quantization of K over 128-token blocks with the fp16 tail.
 // CTA j of a stream handles the j-th block touched by this append.  CTA 0 also
 // handles the final block when that one is incomplete (it writes the tail, which
@@ -750,6 +811,10 @@ quant_kchan_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ k_new,
     if (!complete) continue;
     __syncthreads();
     uint8_t* pg = c.pages + ((size_t)bh * g.n_pages + page) * g.page_bytes;
+    if (D == 128 && (g.kb == 4 || g.kb == 8)) {
+      if (g.kb == 4) kchan_block_fast<4>(sX, sC, pg, g, tid); else kchan_block_fast<8>(sX, sC, pg, g, tid);
+      continue;
+    }
     for (int d = tid; d < D; d += kThreads) {
       float mn = INFINITY, mx = -INFINITY;
       for (int t = 0; t < kPageTokens; ++t) {
