@@ -36,6 +36,13 @@ int kvq_debug_decode_stall(const kvq_config* cfg, const kvq_cache* cache, const 
                            int32_t out_dtype, float softmax_scale, void* workspace, size_t workspace_bytes,
                            int64_t skip_page, uint32_t wait_us, void* cuda_stream);
 
+/* kvq_debug_decode_stall through a chosen kernel of the fast path (impl as in kvq_debug_decode_impl): the
+ * tcgen05 kernel's bounded waits, its drain of copies and MMAs in flight and the release of its tensor memory
+ * are exercised the same way as the warp-level kernel's. */
+int kvq_debug_decode_stall_impl(const kvq_config* cfg, const kvq_cache* cache, const void* q, void* out,
+                                int32_t out_dtype, float softmax_scale, void* workspace, size_t workspace_bytes,
+                                int64_t skip_page, uint32_t wait_us, int32_t impl, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -313,6 +313,17 @@ int kvq_debug_decode_stall(const kvq_config* cfg, const kvq_cache* cache, const 
   return decode_with(cfg, cache, q, out, out_dtype, softmax_scale, workspace, workspace_bytes, cuda_stream, dbg);
 }
 
+int kvq_debug_decode_stall_impl(const kvq_config* cfg, const kvq_cache* cache, const void* q, void* out,
+                                int32_t out_dtype, float softmax_scale, void* workspace, size_t workspace_bytes,
+                                int64_t skip_page, uint32_t wait_us, int32_t impl, void* cuda_stream) {
+  if (wait_us == 0 || wait_us > 100000u || impl < 0 || impl > 2) return KVQ_ERR_INVALID_ARG;
+  DecodeDebug dbg;
+  dbg.skip_page = skip_page;
+  dbg.wait_us = wait_us;
+  dbg.fast_impl = impl;
+  return decode_with(cfg, cache, q, out, out_dtype, softmax_scale, workspace, workspace_bytes, cuda_stream, dbg);
+}
+
 int kvq_dequantize(const kvq_config* cfg, const kvq_cache* cache, void* k_out, void* v_out, int32_t t_begin,
                    int32_t t_end, void* cuda_stream) {
   Geom g;

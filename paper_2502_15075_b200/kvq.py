@@ -68,13 +68,16 @@ _lib.kvq_debug_decode_stall.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_
 _lib.kvq_debug_decode_impl.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
                                        ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
                                        ctypes.c_int32, ctypes.c_void_p]
+_lib.kvq_debug_decode_stall_impl.argtypes = [_P(kvq_config), _P(kvq_cache), ctypes.c_void_p, ctypes.c_void_p,
+                                             ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
+                                             ctypes.c_int64, ctypes.c_uint32, ctypes.c_int32, ctypes.c_void_p]
 _lib.kvq_check_status.argtypes = [_P(kvq_cache), ctypes.c_void_p]
 _lib.kvq_strerror.argtypes = [ctypes.c_int]
 _lib.kvq_strerror.restype = ctypes.c_char_p
 for _f in ("kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes", "kvq_quantize_append",
            "kvq_decode_attention", "kvq_decode_attention_static", "kvq_dequantize", "kvq_check_status",
            "kvq_quant_error", "kvq_bit_balance", "kvq_debug_decode_generic", "kvq_debug_decode_stall",
-           "kvq_debug_decode_impl", "kvq_workspace_bytes_rows", "kvq_decode_attention_rows"):
+           "kvq_debug_decode_impl", "kvq_debug_decode_stall_impl", "kvq_workspace_bytes_rows", "kvq_decode_attention_rows"):
     getattr(_lib, _f).restype = ctypes.c_int
 
 EXPORTS = ("kvq_layout_version", "kvq_page_bytes", "kvq_cache_bytes", "kvq_workspace_bytes",
@@ -300,6 +303,15 @@ def kvq_debug_decode_stall(cfg: kvq_config, cache: Cache, q: torch.Tensor, out: 
                                        _dtype_code(out.dtype), 0.0, workspace.data_ptr(),
                                        workspace.numel() * workspace.element_size(), int(skip_page), int(wait_us),
                                        _stream_ptr(None)), "kvq_debug_decode_stall")
+
+
+def kvq_debug_decode_stall_impl(cfg: kvq_config, cache: Cache, q: torch.Tensor, out: torch.Tensor,
+                                workspace: torch.Tensor, skip_page: int, wait_us: int, impl: int):
+    """Test hook: kvq_debug_decode_stall through a chosen kernel of the fast path."""
+    _check(_lib.kvq_debug_decode_stall_impl(ctypes.byref(cfg), ctypes.byref(cache.c), q.data_ptr(), out.data_ptr(),
+                                            _dtype_code(out.dtype), 0.0, workspace.data_ptr(),
+                                            workspace.numel() * workspace.element_size(), int(skip_page), int(wait_us),
+                                            int(impl), _stream_ptr(None)), "kvq_debug_decode_stall_impl")
 
 
 def kvq_check_status(cache: Cache, stream: Optional[torch.cuda.Stream] = None) -> int:

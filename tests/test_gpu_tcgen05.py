@@ -88,3 +88,23 @@ def test_tcgen05_refuses_configurations_it_does_not_serve(kvq):
     with pytest.raises(kvq.KvqError) as e:
         kvq.kvq_debug_decode_impl(cfg, gc, q, out, ws, kvq.IMPL_TCGEN05)
     assert e.value.code == -2
+
+
+def test_tcgen05_wait_that_runs_out_sets_the_status_and_frees_its_tensor_memory(kvq):
+    w = wl.LLAMA_8B.with_(n_kv_heads=2, n_q_heads=8)
+    B, T = 2, 128 * 40
+    k, v = wl.make_kv(w, tokens=T, batch=B)
+    cfg, gc, _ = tl.build_both(kvq, w, k, v, [T], T)
+    q = wl.make_q(w, batch=B).cuda()
+    ws = torch.empty(max(16, kvq.kvq_workspace_bytes(cfg)), dtype=torch.uint8, device="cuda")
+    out = torch.zeros(tuple(q.shape), dtype=torch.float32, device="cuda")
+    good = decode_impl(kvq, cfg, gc, q, kvq.IMPL_TCGEN05)
+    # page 57 of the 160 pages never arrives; every wait gives up after 2 ms
+    kvq.kvq_debug_decode_stall_impl(cfg, gc, q, out, ws, 57, 2000, kvq.IMPL_TCGEN05)
+    torch.cuda.synchronize()                                   # returns: nothing hangs
+    assert kvq.kvq_check_status(gc) == -7                      # KVQ_ERR_DEVICE_TIMEOUT
+    gc.status.zero_()
+    # the next launches find the SMs' tensor memory free again and give the same result as before
+    for _ in range(3):
+        again = decode_impl(kvq, cfg, gc, q, kvq.IMPL_TCGEN05)
+        assert np.array_equal(again, good)
