@@ -108,3 +108,15 @@ def test_tcgen05_wait_that_runs_out_sets_the_status_and_frees_its_tensor_memory(
     for _ in range(3):
         again = decode_impl(kvq, cfg, gc, q, kvq.IMPL_TCGEN05)
         assert np.array_equal(again, good)
+
+
+@pytest.mark.parametrize("R,T,chunks", [(64, 64 * 5 + 37, [64 * 5 + 37]), (128, 128 * 2 + 100, [300, 56]), (64, 40, [40])])
+def test_tcgen05_decode_merges_the_residual_window(kvq, R, T, chunks):
+    w = wl.LLAMA_8B.with_(n_kv_heads=2, n_q_heads=8)
+    B = 2
+    cap = ((T + 127) // 128) * 128 + 128
+    k, v = wl.make_kv(w, tokens=T, batch=B)
+    cfg, gc, _ = tl.build_both(kvq, w, k, v, chunks, cap, residual=R)
+    q = wl.make_q(w, batch=B)
+    want = tl.oracle_on_gpu_codes(gc, w).decode(tl.bits_of(q))
+    tl.assert_attention_close(decode_impl(kvq, cfg, gc, q, kvq.IMPL_TCGEN05), want)
