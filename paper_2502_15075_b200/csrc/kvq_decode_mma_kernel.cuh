@@ -23,7 +23,7 @@ __host__ __device__ inline SmemLayout smem_layout(int page_bytes, int stages, in
   s.ring_bytes = s.page_stride * stages;
   s.bar_off = s.ring_bytes;
   s.pref_off = s.bar_off + 16 * 8 * 2;                      // up to 32 barriers: (full, empty[, ready]) per stage
-  s.misc_off = (s.pref_off + (batch + 1) * 4 + 15) & ~15;
+  s.misc_off = (s.pref_off + 2 * (batch + 1) * 4 + 15) & ~15;      // two prefixes: pages, and pages + stream gaps
   s.master_off = s.misc_off + 64;
   s.ml_off = s.master_off + nw * 4 * nh * (D + 8) * 4;
   s.chan_off = s.ml_off + nw * 4 * nh * 2 * 4;
@@ -61,6 +61,20 @@ __device__ __forceinline__ uint32_t fixed_point_limb(const float (&t)[4], float 
   return w;
 }
 
+// The split balances time, not pages.  Ending one stream and starting the next (fold and combine the warps'
+// state, store and publish the partial, perhaps merge; load and convert the next queries) costs a CTA as much as
+// ~9 pages (8.4 us on the 8B-shaped layer: CTAs whose share crosses a stream boundary ended at 81.2 us, the others
+// at 72.8 us), and of the three CTAs that share an SM the hardware favours the older ones (launch waves ended at
+// 68.9 / 72.7 / 76.8 us with equal work).  So every stream is given kGapPages virtual pages in front of its real
+// ones and the shares of the launch waves are weighted; the split is taken on that virtual axis.
+#ifndef KVQ_GAP_PAGES
+#define KVQ_GAP_PAGES 10
+#endif
+#ifndef KVQ_WAVE_W0
+#define KVQ_WAVE_W0 1040
+#endif
+constexpr int kGapPages = KVQ_GAP_PAGES;
+constexpr int kWaveWeight0 = KVQ_WAVE_W0;  // share of a first-wave CTA in thousandths of the mean (third wave: 2000 - this)
 constexpr float kQFix = 32512.0f;          // largest |Q| of the 16-bit fixed-point q (hi limb stays within +-127)
 constexpr float kQFix3 = 8300000.0f;       // ... of the 24-bit fixed-point q * s of channel-wise keys (three limbs)
 
@@ -154,6 +168,46 @@ __device__ __forceinline__ float load_q_lane(const Geom& g, const CachePtrs& c, 
   return amax;
 }
 
+// Weighted position of a CTA on the virtual axis in units of 1 / kWaveUnits of the whole: three launch waves of 148
+// CTAs with weights W0, 1000, 2000 - W0.
+constexpr long long kWaveUnits = 148ll * 3000;
+__device__ __forceinline__ long long wave_prefix(int cta) {
+  constexpr int W0 = kWaveWeight0, W1 = 1000, W2 = 2000 - kWaveWeight0;
+  const int k = cta / 148, r = cta % 148;
+  return (k == 0 ? 0 : k == 1 ? W0 : k == 2 ? W0 + W1 : W0 + W1 + W2) * 148ll + (long long)r * (k == 0 ? W0 : k == 1 ? W1 : W2);
+}
+// First virtual page of a CTA's share: equal shares, or shares weighted by launch wave (three CTAs per SM).
+
+static __device__ __forceinline__ long long share_start_virtual(const FlatPlan& plan, bool waves, int cta) {
+  if (!waves) return plan.lo(cta);
+  return plan.N * wave_prefix(cta) / kWaveUnits;
+}
+// The CTA whose share holds virtual page v (no division in the search: floor(a / W) <= v  <=>  a < (v + 1) W).
+static __device__ __forceinline__ int cta_of_virtual(const FlatPlan& plan, bool waves, long long v) {
+  if (!waves) return plan.cta_of(v);
+  const long long bound = (v + 1) * kWaveUnits;
+  int lo_ = 0, hi_ = 3 * 148 - 1;
+  while (lo_ < hi_) {
+    const int mid = (lo_ + hi_ + 1) >> 1;
+    if (plan.N * wave_prefix(mid) < bound) lo_ = mid; else hi_ = mid - 1;
+  }
+  return lo_;
+}
+// Flat index of the first real page at or after the start of a CTA's share (sPref: pages, sVPref: pages + gaps).
+static __device__ __forceinline__ long long share_start(const FlatPlan& plan, bool waves, int cta, const int* sPref,
+                                                     const int* sVPref, int B, int Hkv, int gap) {
+  const long long v = share_start_virtual(plan, waves, cta);
+  if (v >= plan.N) return sPref[B];
+  int lo_ = 0, hi_ = B - 1;                        // last batch entry with sVPref <= v
+  while (lo_ < hi_) {
+    const int mid = (lo_ + hi_ + 1) >> 1;
+    if (sVPref[mid] <= v) lo_ = mid; else hi_ = mid - 1;
+  }
+  const int pb = (sPref[lo_ + 1] - sPref[lo_]) / Hkv, len = pb + gap;
+  const int vs = (int)(v - sVPref[lo_]), hh = vs / len, off = vs % len;
+  return (long long)sPref[lo_] + (long long)hh * pb + max(0, off - gap);
+}
+
 // Template parameters: head_dim, key bits, value bits, key axis (0 token-wise, 1 channel-wise), key / value groups
 // per row, NH = query heads per lane (1: up to 4 heads per KV head, 2: up to 8), consumer warps (4: one per
 // 32-token block of a page), resident CTAs per SM.
@@ -187,6 +241,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   constexpr int NCONS = NW * 32;
   constexpr int NG = NW / 4;                // groups of four consumer warps; a group takes every NG-th page
   constexpr uint32_t FULL = 0xffffffffu;
+  // The time-balanced split (stream gaps, wave weights) pays where the arithmetic per page limits the kernel; pages
+  // of 12 bits per element pair and more are bound by their bytes and keep the plain split by pages.
+  constexpr int GAP = (KAXIS == 0 && KB + VB <= 8) ? kGapPages : 0;
   static_assert(NW % 4 == 0, "four consumer warps per page, one per 32-token block");
   static_assert(KAXIS == 0 || KB != 2, "channel-wise 2-bit keys are not instantiated");
   static_assert(MT % FPBV == 0, "value m-tiles come in groups that share a byte");
@@ -195,6 +252,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   const SmemLayout sl = smem_layout(g.page_bytes, stages, NW, g.B, D, NH, KAXIS == 1);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sl.bar_off);   // full[0..stages), empty[0..stages)
   int* sPref = reinterpret_cast<int*>(smem + sl.pref_off);
+  int* sVPref = sPref + (g.B + 1);                                   // the same prefix with kGapPages more per stream
   int* sMisc = reinterpret_cast<int*>(smem + sl.misc_off);           // [0] pages_max, [1] abort flag
   float* sMaster = reinterpret_cast<float*>(smem + sl.master_off);   // [NW][NHEADS][MSTRIDE]
   float* sML = reinterpret_cast<float*>(smem + sl.ml_off);           // [NW][NHEADS][2] = (reference, l)
@@ -206,7 +264,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   const int B = g.B, Hkv = g.Hkv, Gq = g.G, G = g.G * g.rows;
 
   // ---- plan: pages per sequence, prefix over the batch
-  if (tid_ == 0) { sPref[0] = 0; sMisc[0] = 0; sMisc[1] = 0; }
+  if (tid_ == 0) { sPref[0] = 0; sVPref[0] = 0; sMisc[0] = 0; sMisc[1] = 0; }
   __syncthreads();
   for (int b = tid_; b < B; b += blockDim.x) {
     int pages = (paged_len(c.seq_len, b, g.capacity, g.R) + kPageTokens - 1) >> 7;
@@ -215,18 +273,22 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   }
   __syncthreads();
   if (warp == 0) {
-    int carry = 0;
+    int carry = 0, vcarry = 0;
     for (int base = 0; base < B; base += 32) {
       int i = base + lane;
       int v = (i < B) ? sPref[i + 1] : 0;
+      int vv = v > 0 ? v + GAP * Hkv : 0;
       for (int off = 1; off < 32; off <<= 1) {
-        int u = __shfl_up_sync(FULL, v, off);
-        if (lane >= off) v += u;
+        int u = __shfl_up_sync(FULL, v, off), uu = __shfl_up_sync(FULL, vv, off);
+        if (lane >= off) { v += u; vv += uu; }
       }
-      if (i < B) sPref[i + 1] = v + carry;
+      if (i < B) { sPref[i + 1] = v + carry; sVPref[i + 1] = vv + vcarry; }
       carry += __shfl_sync(FULL, v, 31);
+      vcarry += __shfl_sync(FULL, vv, 31);
     }
   }
+  const int s_plan = s_cap - (g.R ? 1 : 0);       // the last partial slot of a stream belongs to its residual window
+  if (warp == 0) __syncwarp();
   if (tid_ == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(smem_u32(&bars[s]), 1);
@@ -234,6 +296,21 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       if constexpr (KAXIS == 1) mbar_init(smem_u32(&bars[2 * stages + s]), 1);     // ready: operands of the page made
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // this CTA's share of the pages, worked out once (sMisc[4..7] = first page, end)
+    const FlatPlan p0 = make_plan(sVPref[B], sMisc[0] + GAP, gridDim.x, s_plan);
+    long long lo0 = 0, hi0 = 0;
+    if (p0.N != 0 && (int)blockIdx.x < p0.c_eff) {
+      if constexpr (GAP == 0) {
+        lo0 = p0.lo(blockIdx.x);
+        hi0 = p0.lo(blockIdx.x + 1);
+      } else {
+        const bool w0 = MINB == 3 && gridDim.x == 3 * 148 && p0.c_eff == (int)gridDim.x && p0.N >= 8ll * gridDim.x;
+        lo0 = share_start(p0, w0, (int)blockIdx.x, sPref, sVPref, B, Hkv, GAP);
+        hi0 = share_start(p0, w0, (int)blockIdx.x + 1, sPref, sVPref, B, Hkv, GAP);
+      }
+    }
+    *reinterpret_cast<long long*>(sMisc + 4) = lo0;
+    *reinterpret_cast<long long*>(sMisc + 6) = hi0;
   }
   __syncthreads();
   // an empty sequence has no page and therefore no CTA of its own: its output rows are zero (with a residual
@@ -247,11 +324,13 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       }
     }
   }
-  const int s_plan = s_cap - (g.R ? 1 : 0);       // the last partial slot of a stream belongs to its residual window
-  const FlatPlan plan = make_plan(sPref[B], sMisc[0], gridDim.x, s_plan);
+  // the plan lives on the virtual axis (pages + a gap in front of every stream)
+  const FlatPlan plan = make_plan(sVPref[B], sMisc[0] + GAP, gridDim.x, s_plan);
   if (plan.N == 0 || (int)blockIdx.x >= plan.c_eff) return;
   unsigned long long* counts = reinterpret_cast<unsigned long long*>(ws + tag_offset_floats(B * Hkv, s_cap, G, D));
-  const long long x_lo = plan.lo(blockIdx.x), x_hi = plan.lo(blockIdx.x + 1);
+  const bool waves = GAP != 0 && MINB == 3 && gridDim.x == 3 * 148 && plan.c_eff == (int)gridDim.x && plan.N >= 8ll * gridDim.x;
+  const long long x_lo = *reinterpret_cast<const long long*>(sMisc + 4), x_hi = *reinterpret_cast<const long long*>(sMisc + 6);
+  if (x_lo >= x_hi) return;                          // a share that lies inside a gap (tiny problems only)
 
   // ---- cursor: first page of this CTA -> (b, h, page)
   int b = 0;
@@ -475,7 +554,6 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     // row r sees the first n - (rows - 1 - r) tokens of the n the sequence holds, window included)
     const int n_unmasked = min(n_tok, clamped_len(c.seq_len, b, g.capacity) - (g.rows - 1));
     const int stream = b * Hkv + h;
-
     // ---- segment start: q operands, group sums and a clean state for this stream's heads
     {
 #pragma unroll
@@ -823,14 +901,17 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           sML[(warp * NHEADS + tid + 4 * nh) * 2 + 1] = l[nh];
         }
       }
+      if (tid_ == 0) {       // which of the stream's partials this CTA writes, and how many there are
+        const long long xs = (long long)sVPref[b] + (long long)h * (pages_b + GAP) + GAP;   // first real page of this stream, virtual axis
+        const int c_first = cta_of_virtual(plan, waves, xs);
+        sMisc[8] = (int)blockIdx.x - c_first;
+        sMisc[9] = cta_of_virtual(plan, waves, xs + pages_b - 1) - c_first + 1;
+      }
       named_bar_sync(1, NCONS);
       // The flat split gives a stream to a run of consecutive CTAs, one partial slot each.  A CTA that holds the
       // whole stream writes the output at once; otherwise it stores its partial, counts itself in, and the CTA
       // that completes the count merges all partials of the stream by log-sum-exp and stores the output.
-      const long long xs = (long long)sPref[b] + (long long)h * pages_b;     // first page of this stream
-      const int c_first = plan.cta_of(xs);
-      const int slot = (int)blockIdx.x - c_first;
-      const int n_part = plan.cta_of(xs + pages_b - 1) - c_first + 1;        // partials of this stream
+      const int slot = sMisc[8], n_part = sMisc[9];
       const bool has_win = clamped_len(c.seq_len, b, g.capacity) > n_tok;    // the window kernel left a partial in slot s_cap - 1
       if (slot >= 0 && slot < s_plan) {
         for (int idx = tid_; idx < G * D; idx += NCONS) {
