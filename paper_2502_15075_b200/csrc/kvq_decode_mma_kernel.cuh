@@ -554,6 +554,15 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     // row r sees the first n - (rows - 1 - r) tokens of the n the sequence holds, window included)
     const int n_unmasked = min(n_tok, clamped_len(c.seq_len, b, g.capacity) - (g.rows - 1));
     const int stream = b * Hkv + h;
+    // which of the stream's partials this CTA writes, and how many there are: one thread works it out now, everybody
+    // reads it after the barrier at the segment's end (the barrier that closed the last segment keeps its readers apart)
+    if (tid_ == 0) {
+      const long long xs = (long long)sVPref[b] + (long long)h * (pages_b + GAP) + GAP;   // first real page of this stream, virtual axis
+      const int c_first = cta_of_virtual(plan, waves, xs);
+      sMisc[8] = (int)blockIdx.x - c_first;
+      sMisc[9] = cta_of_virtual(plan, waves, xs + pages_b - 1) - c_first + 1;
+    }
+
     // ---- segment start: q operands, group sums and a clean state for this stream's heads
     {
 #pragma unroll
@@ -900,12 +909,6 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
           sML[(warp * NHEADS + tid + 4 * nh) * 2 + 0] = m_ref[nh];
           sML[(warp * NHEADS + tid + 4 * nh) * 2 + 1] = l[nh];
         }
-      }
-      if (tid_ == 0) {       // which of the stream's partials this CTA writes, and how many there are
-        const long long xs = (long long)sVPref[b] + (long long)h * (pages_b + GAP) + GAP;   // first real page of this stream, virtual axis
-        const int c_first = cta_of_virtual(plan, waves, xs);
-        sMisc[8] = (int)blockIdx.x - c_first;
-        sMisc[9] = cta_of_virtual(plan, waves, xs + pages_b - 1) - c_first + 1;
       }
       named_bar_sync(1, NCONS);
       // The flat split gives a stream to a run of consecutive CTAs, one partial slot each.  A CTA that holds the
