@@ -3,8 +3,9 @@
 // reconstructed inside the contraction.
 //
 // Structure (one CTA = 4 consumer warps + 1 producer warp, several CTAs per SM):
-//  * the producer streams whole 128-token pages into a shared-memory ring with
-//    cp.async.bulk (one bulk copy per page, completion on an mbarrier);
+//  * the producer streams whole 128-token pages into a four-stage shared-memory ring
+//    with cp.async.bulk (one bulk copy per page with an L2 evict-first policy,
+//    completion on an mbarrier);
 //  * each consumer warp owns one 32-token block of every page and loads its operand
 //    fragments with 16-byte shared loads (the page layout already is fragment order);
 //  * both contractions are integer tensor-core MMAs on the raw code bytes
@@ -14,10 +15,12 @@
 //    three for 8 heads); the 8 MMA columns carry (head, limb) pairs;
 //  * scale and zero-point never touch the codes:  q.K^_t = s_t (q.c_t) + z_t sum(q)
 //    and  o = sum_t (p_t s_t) c_t + sum_t p_t z_t ;
-//  * the sequence is split flat over the grid: CTA i takes the i-th equal share of
-//    all pages of all streams and writes one unnormalised partial (m, l, o) per stream
-//    it touches; the CTA that publishes the last partial of a stream merges them by
-//    log-sum-exp and writes the output (no second kernel, nobody waits).
+//  * the sequence is split flat over the grid: CTA i takes the i-th share of all pages
+//    of all streams (shares balanced by time where the arithmetic limits the kernel: a
+//    stream boundary counts as ten pages, the launch waves of an SM are weighted) and
+//    writes one unnormalised partial (m, l, o) per stream it touches; the CTA that
+//    publishes the last partial of a stream merges them by log-sum-exp and writes the
+//    output (no second kernel, nobody waits).
 // Every wait on an mbarrier is bounded in time; on expiry the kernel sets
 // KVQ_STATUS_DEVICE_TIMEOUT, keeps arriving at its barriers without computing, and returns.
 #pragma once
