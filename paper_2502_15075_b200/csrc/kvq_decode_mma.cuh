@@ -200,7 +200,12 @@ __device__ __forceinline__ FlatPlan make_plan(long long N, int pages_max, int gr
 // (stale contents, an earlier launch) restarts at 1, so the workspace needs no initialisation; the CTA that
 // reaches the expected count merges and clears the word, so that a replayed launch with the same id starts clean.
 __device__ __forceinline__ unsigned tagged_count(unsigned long long* p, unsigned long long id40) {
-  unsigned long long old = *reinterpret_cast<volatile unsigned long long*>(p);
+  // the usual case in one round trip: the word already carries this launch's id
+  unsigned long long old = atomicAdd(p, 1ull);
+  if ((old >> 24) == id40) return (unsigned)((old + 1ull) & 0xFFFFFFull);
+  // otherwise the addition went into a word of another launch (or a cleared one): start it, or count into it once
+  // somebody else has started it (whatever the stray additions left is overwritten by the start)
+  old += 1ull;
   while (true) {
     const unsigned long long nw = ((old >> 24) == id40) ? old + 1ull : ((id40 << 24) | 1ull);
     const unsigned long long r = atomicCAS(p, old, nw);

@@ -182,16 +182,17 @@ static __device__ __forceinline__ long long share_start_virtual(const FlatPlan& 
   if (!waves) return plan.lo(cta);
   return plan.N * wave_prefix(cta) / kWaveUnits;
 }
-// The CTA whose share holds virtual page v (no division in the search: floor(a / W) <= v  <=>  a < (v + 1) W).
+// The CTA whose share holds virtual page v: the largest c with N prefix(c) < (v + 1) U, found wave by wave (the
+// prefix is linear inside a wave), one division.
 static __device__ __forceinline__ int cta_of_virtual(const FlatPlan& plan, bool waves, long long v) {
   if (!waves) return plan.cta_of(v);
-  const long long bound = (v + 1) * kWaveUnits;
-  int lo_ = 0, hi_ = 3 * 148 - 1;
-  while (lo_ < hi_) {
-    const int mid = (lo_ + hi_ + 1) >> 1;
-    if (plan.N * wave_prefix(mid) < bound) lo_ = mid; else hi_ = mid - 1;
-  }
-  return lo_;
+  constexpr int W0 = kWaveWeight0, W1 = 1000, W2 = 2000 - kWaveWeight0;
+  const long long a = (v + 1) * kWaveUnits - 1;                  // N prefix(c) <= a
+  const long long b1 = plan.N * (148ll * W0), b2 = plan.N * (148ll * (W0 + W1));
+  const int k = a >= b2 ? 2 : a >= b1 ? 1 : 0;
+  const long long base = k == 2 ? b2 : k == 1 ? b1 : 0;
+  const long long r = (a - base) / (plan.N * (k == 2 ? W2 : k == 1 ? W1 : W0));
+  return 148 * k + (int)(r < 147 ? r : 147);
 }
 // Flat index of the first real page at or after the start of a CTA's share (sPref: pages, sVPref: pages + gaps).
 static __device__ __forceinline__ long long share_start(const FlatPlan& plan, bool waves, int cta, const int* sPref,
