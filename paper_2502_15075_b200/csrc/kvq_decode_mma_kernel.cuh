@@ -168,36 +168,44 @@ __device__ __forceinline__ float load_q_lane(const Geom& g, const CachePtrs& c, 
   return amax;
 }
 
-// Weighted position of a CTA on the virtual axis in units of 1 / kWaveUnits of the whole: three launch waves of 148
-// CTAs with weights W0, 1000, 2000 - W0.
-constexpr long long kWaveUnits = 148ll * 3000;
+// Weighted position of a CTA on the virtual axis in units of 1 / (148 * 1000 * waves) of the whole: two or three launch
+// waves of 148 CTAs (one per CTA that an SM holds) with weights W0, [1000,] 2000 - W0.
+#ifndef KVQ_WAVE2_W0
+#define KVQ_WAVE2_W0 1000   /* two CTAs per SM: weighting the waves did not pay (70B-shaped layer: 147.8 us equal, 149.9 us at 1040, 154.1 us at 1080) */
+#endif
+template <int WAVES> struct WaveWeights;
+template <> struct WaveWeights<3> { static constexpr int w[3] = {kWaveWeight0, 1000, 2000 - kWaveWeight0}; };
+template <> struct WaveWeights<2> { static constexpr int w[3] = {KVQ_WAVE2_W0, 2000 - KVQ_WAVE2_W0, 0}; };
+template <int WAVES>
 __device__ __forceinline__ long long wave_prefix(int cta) {
-  constexpr int W0 = kWaveWeight0, W1 = 1000, W2 = 2000 - kWaveWeight0;
+  constexpr int W0 = WaveWeights<WAVES>::w[0], W1 = WaveWeights<WAVES>::w[1], W2 = WaveWeights<WAVES>::w[2];
   const int k = cta / 148, r = cta % 148;
   return (k == 0 ? 0 : k == 1 ? W0 : k == 2 ? W0 + W1 : W0 + W1 + W2) * 148ll + (long long)r * (k == 0 ? W0 : k == 1 ? W1 : W2);
 }
-// First virtual page of a CTA's share: equal shares, or shares weighted by launch wave (three CTAs per SM).
-
+// First virtual page of a CTA's share: equal shares, or shares weighted by launch wave.
+template <int WAVES>
 static __device__ __forceinline__ long long share_start_virtual(const FlatPlan& plan, bool waves, int cta) {
   if (!waves) return plan.lo(cta);
-  return plan.N * wave_prefix(cta) / kWaveUnits;
+  return plan.N * wave_prefix<WAVES>(cta) / (148ll * 1000 * WAVES);
 }
 // The CTA whose share holds virtual page v: the largest c with N prefix(c) < (v + 1) U, found wave by wave (the
 // prefix is linear inside a wave), one division.
+template <int WAVES>
 static __device__ __forceinline__ int cta_of_virtual(const FlatPlan& plan, bool waves, long long v) {
   if (!waves) return plan.cta_of(v);
-  constexpr int W0 = kWaveWeight0, W1 = 1000, W2 = 2000 - kWaveWeight0;
-  const long long a = (v + 1) * kWaveUnits - 1;                  // N prefix(c) <= a
+  constexpr int W0 = WaveWeights<WAVES>::w[0], W1 = WaveWeights<WAVES>::w[1], W2 = WaveWeights<WAVES>::w[2];
+  const long long a = (v + 1) * (148ll * 1000 * WAVES) - 1;      // N prefix(c) <= a
   const long long b1 = plan.N * (148ll * W0), b2 = plan.N * (148ll * (W0 + W1));
-  const int k = a >= b2 ? 2 : a >= b1 ? 1 : 0;
+  const int k = (WAVES == 3 && a >= b2) ? 2 : a >= b1 ? 1 : 0;
   const long long base = k == 2 ? b2 : k == 1 ? b1 : 0;
   const long long r = (a - base) / (plan.N * (k == 2 ? W2 : k == 1 ? W1 : W0));
   return 148 * k + (int)(r < 147 ? r : 147);
 }
 // Flat index of the first real page at or after the start of a CTA's share (sPref: pages, sVPref: pages + gaps).
+template <int WAVES>
 static __device__ __forceinline__ long long share_start(const FlatPlan& plan, bool waves, int cta, const int* sPref,
                                                      const int* sVPref, int B, int Hkv, int gap) {
-  const long long v = share_start_virtual(plan, waves, cta);
+  const long long v = share_start_virtual<WAVES>(plan, waves, cta);
   if (v >= plan.N) return sPref[B];
   int lo_ = 0, hi_ = B - 1;                        // last batch entry with sVPref <= v
   while (lo_ < hi_) {
@@ -245,6 +253,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   // The time-balanced split (stream gaps, wave weights) pays where the arithmetic per page limits the kernel; pages
   // of 12 bits per element pair and more are bound by their bytes and keep the plain split by pages.
   constexpr int GAP = (KAXIS == 0 && KB + VB <= 8) ? kGapPages : 0;
+  constexpr int WAVES = MINB == 2 ? 2 : 3;          // CTAs per SM = launch waves (the weights apply to a grid of 148 * WAVES)
   static_assert(NW % 4 == 0, "four consumer warps per page, one per 32-token block");
   static_assert(KAXIS == 0 || KB != 2, "channel-wise 2-bit keys are not instantiated");
   static_assert(MT % FPBV == 0, "value m-tiles come in groups that share a byte");
@@ -297,21 +306,20 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       if constexpr (KAXIS == 1) mbar_init(smem_u32(&bars[2 * stages + s]), 1);     // ready: operands of the page made
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // this CTA's share of the pages, worked out once (sMisc[4..7] = first page, end)
+  }
+  if (warp == 0 && lane < 2) {
+    // this CTA's share of the pages, worked out once: lane 0 its first page, lane 1 its end (sMisc[4..7])
     const FlatPlan p0 = make_plan(sVPref[B], sMisc[0] + GAP, gridDim.x, s_plan);
-    long long lo0 = 0, hi0 = 0;
+    long long x0 = 0;
     if (p0.N != 0 && (int)blockIdx.x < p0.c_eff) {
       if constexpr (GAP == 0) {
-        lo0 = p0.lo(blockIdx.x);
-        hi0 = p0.lo(blockIdx.x + 1);
+        x0 = p0.lo(blockIdx.x + lane);
       } else {
-        const bool w0 = MINB == 3 && gridDim.x == 3 * 148 && p0.c_eff == (int)gridDim.x && p0.N >= 8ll * gridDim.x;
-        lo0 = share_start(p0, w0, (int)blockIdx.x, sPref, sVPref, B, Hkv, GAP);
-        hi0 = share_start(p0, w0, (int)blockIdx.x + 1, sPref, sVPref, B, Hkv, GAP);
+        const bool w0 = gridDim.x == WAVES * 148 && p0.c_eff == (int)gridDim.x && p0.N >= 8ll * gridDim.x;
+        x0 = share_start<WAVES>(p0, w0, (int)blockIdx.x + lane, sPref, sVPref, B, Hkv, GAP);
       }
     }
-    *reinterpret_cast<long long*>(sMisc + 4) = lo0;
-    *reinterpret_cast<long long*>(sMisc + 6) = hi0;
+    *reinterpret_cast<long long*>(sMisc + 4 + 2 * lane) = x0;
   }
   __syncthreads();
   // an empty sequence has no page and therefore no CTA of its own: its output rows are zero (with a residual
@@ -329,7 +337,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   const FlatPlan plan = make_plan(sVPref[B], sMisc[0] + GAP, gridDim.x, s_plan);
   if (plan.N == 0 || (int)blockIdx.x >= plan.c_eff) return;
   unsigned long long* counts = reinterpret_cast<unsigned long long*>(ws + tag_offset_floats(B * Hkv, s_cap, G, D));
-  const bool waves = GAP != 0 && MINB == 3 && gridDim.x == 3 * 148 && plan.c_eff == (int)gridDim.x && plan.N >= 8ll * gridDim.x;
+  const bool waves = GAP != 0 && gridDim.x == WAVES * 148 && plan.c_eff == (int)gridDim.x && plan.N >= 8ll * gridDim.x;
   const long long x_lo = *reinterpret_cast<const long long*>(sMisc + 4), x_hi = *reinterpret_cast<const long long*>(sMisc + 6);
   if (x_lo >= x_hi) return;                          // a share that lies inside a gap (tiny problems only)
 
@@ -559,9 +567,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     // reads it after the barrier at the segment's end (the barrier that closed the last segment keeps its readers apart)
     if (tid_ == 0) {
       const long long xs = (long long)sVPref[b] + (long long)h * (pages_b + GAP) + GAP;   // first real page of this stream, virtual axis
-      const int c_first = cta_of_virtual(plan, waves, xs);
+      const int c_first = cta_of_virtual<WAVES>(plan, waves, xs);
       sMisc[8] = (int)blockIdx.x - c_first;
-      sMisc[9] = cta_of_virtual(plan, waves, xs + pages_b - 1) - c_first + 1;
+      sMisc[9] = cta_of_virtual<WAVES>(plan, waves, xs + pages_b - 1) - c_first + 1;
     }
 
     // ---- segment start: q operands, group sums and a clean state for this stream's heads
