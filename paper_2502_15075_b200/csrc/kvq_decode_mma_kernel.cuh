@@ -263,7 +263,7 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + sl.bar_off);   // full[0..stages), empty[0..stages)
   int* sPref = reinterpret_cast<int*>(smem + sl.pref_off);
   int* sVPref = sPref + (g.B + 1);                                   // the same prefix with kGapPages more per stream
-  int* sMisc = reinterpret_cast<int*>(smem + sl.misc_off);           // [0] pages_max, [1] abort flag
+  int* sMisc = reinterpret_cast<int*>(smem + sl.misc_off);           // [0] pages_max, [1] abort flag, [2] published count, [4..7] share ends, [8..9] segment slot / partials, [10..13] CTAs taking part, cursor
   float* sMaster = reinterpret_cast<float*>(smem + sl.master_off);   // [NW][NHEADS][MSTRIDE]
   float* sML = reinterpret_cast<float*>(smem + sl.ml_off);           // [NW][NHEADS][2] = (reference, l)
 
@@ -273,20 +273,16 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   // r * Gq + j, with its own causal limit on the tokens it may see.
   const int B = g.B, Hkv = g.Hkv, Gq = g.G, G = g.G * g.rows;
 
-  // ---- plan: pages per sequence, prefix over the batch
-  if (tid_ == 0) { sPref[0] = 0; sVPref[0] = 0; sMisc[0] = 0; sMisc[1] = 0; }
-  __syncthreads();
-  for (int b = tid_; b < B; b += blockDim.x) {
-    int pages = (paged_len(c.seq_len, b, g.capacity, g.R) + kPageTokens - 1) >> 7;
-    sPref[b + 1] = pages * Hkv;
-    atomicMax(&sMisc[0], pages);
-  }
-  __syncthreads();
+  // ---- plan, all of it on warp 0 (the others wait at one barrier): pages per sequence, prefix over the batch,
+  // this CTA's share of the pages and the stream its first page lies in
+  const int s_plan = s_cap - (g.R ? 1 : 0);       // the last partial slot of a stream belongs to its residual window
   if (warp == 0) {
-    int carry = 0, vcarry = 0;
+    int carry = 0, vcarry = 0, pmax = 0;
     for (int base = 0; base < B; base += 32) {
-      int i = base + lane;
-      int v = (i < B) ? sPref[i + 1] : 0;
+      const int i = base + lane;
+      const int pages = (i < B) ? (paged_len(c.seq_len, i, g.capacity, g.R) + kPageTokens - 1) >> 7 : 0;
+      pmax = max(pmax, pages);
+      int v = pages * Hkv;
       int vv = v > 0 ? v + GAP * Hkv : 0;
       for (int off = 1; off < 32; off <<= 1) {
         int u = __shfl_up_sync(FULL, v, off), uu = __shfl_up_sync(FULL, vv, off);
@@ -296,30 +292,45 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
       carry += __shfl_sync(FULL, v, 31);
       vcarry += __shfl_sync(FULL, vv, 31);
     }
-  }
-  const int s_plan = s_cap - (g.R ? 1 : 0);       // the last partial slot of a stream belongs to its residual window
-  if (warp == 0) __syncwarp();
-  if (tid_ == 0) {
-    for (int s = 0; s < stages; ++s) {
-      mbar_init(smem_u32(&bars[s]), 1);
-      mbar_init(smem_u32(&bars[stages + s]), 4);
-      if constexpr (KAXIS == 1) mbar_init(smem_u32(&bars[2 * stages + s]), 1);     // ready: operands of the page made
+    for (int off = 16; off; off >>= 1) pmax = max(pmax, __shfl_xor_sync(FULL, pmax, off));
+    if (lane == 0) {
+      sPref[0] = 0; sVPref[0] = 0; sMisc[0] = pmax; sMisc[1] = 0;
+      for (int s = 0; s < stages; ++s) {
+        mbar_init(smem_u32(&bars[s]), 1);
+        mbar_init(smem_u32(&bars[stages + s]), 4);
+        if constexpr (KAXIS == 1) mbar_init(smem_u32(&bars[2 * stages + s]), 1);     // ready: operands of the page made
+      }
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (warp == 0 && lane < 2) {
-    // this CTA's share of the pages, worked out once: lane 0 its first page, lane 1 its end (sMisc[4..7])
-    const FlatPlan p0 = make_plan(sVPref[B], sMisc[0] + GAP, gridDim.x, s_plan);
-    long long x0 = 0;
-    if (p0.N != 0 && (int)blockIdx.x < p0.c_eff) {
-      if constexpr (GAP == 0) {
-        x0 = p0.lo(blockIdx.x + lane);
-      } else {
-        const bool w0 = gridDim.x == WAVES * 148 && p0.c_eff == (int)gridDim.x && p0.N >= 8ll * gridDim.x;
-        x0 = share_start<WAVES>(p0, w0, (int)blockIdx.x + lane, sPref, sVPref, B, Hkv, GAP);
+    __syncwarp();
+    if (lane < 2) {
+      // lane 0: the share's first page, the CTAs that take part and the cursor; lane 1: the share's end
+      const FlatPlan p0 = make_plan(vcarry, pmax + GAP, gridDim.x, s_plan);
+      long long x0 = 0;
+      if (p0.N != 0 && (int)blockIdx.x < p0.c_eff) {
+        if constexpr (GAP == 0) {
+          x0 = p0.lo(blockIdx.x + lane);
+        } else {
+          const bool w0 = gridDim.x == WAVES * 148 && p0.c_eff == (int)gridDim.x && p0.N >= 8ll * gridDim.x;
+          x0 = share_start<WAVES>(p0, w0, (int)blockIdx.x + lane, sPref, sVPref, B, Hkv, GAP);
+        }
+      }
+      *reinterpret_cast<long long*>(sMisc + 4 + 2 * lane) = x0;
+      if (lane == 0) {
+        int cb = 0, ch = 0, cp = 0;
+        if (x0 < carry) {                      // a real page: (sequence, kv head, page) of the share's first page
+          int lo_ = 0, hi_ = B - 1;            // last sequence with sPref <= x0
+          while (lo_ < hi_) {
+            int mid = (lo_ + hi_ + 1) >> 1;
+            if (sPref[mid] <= x0) lo_ = mid; else hi_ = mid - 1;
+          }
+          cb = lo_;
+          const int pb = (sPref[cb + 1] - sPref[cb]) / Hkv, r = (int)x0 - sPref[cb];
+          if (pb > 0) { ch = r / pb; cp = r % pb; }
+        }
+        sMisc[10] = p0.c_eff; sMisc[11] = cb; sMisc[12] = ch; sMisc[13] = cp;
       }
     }
-    *reinterpret_cast<long long*>(sMisc + 4 + 2 * lane) = x0;
   }
   __syncthreads();
   // an empty sequence has no page and therefore no CTA of its own: its output rows are zero (with a residual
@@ -334,7 +345,9 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
     }
   }
   // the plan lives on the virtual axis (pages + a gap in front of every stream)
-  const FlatPlan plan = make_plan(sVPref[B], sMisc[0] + GAP, gridDim.x, s_plan);
+  FlatPlan plan;
+  plan.N = sVPref[B];
+  plan.c_eff = sMisc[10];
   if (plan.N == 0 || (int)blockIdx.x >= plan.c_eff) return;
   unsigned long long* counts = reinterpret_cast<unsigned long long*>(ws + tag_offset_floats(B * Hkv, s_cap, G, D));
   const bool waves = GAP != 0 && gridDim.x == WAVES * 148 && plan.c_eff == (int)gridDim.x && plan.N >= 8ll * gridDim.x;
@@ -342,18 +355,8 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   if (x_lo >= x_hi) return;                          // a share that lies inside a gap (tiny problems only)
 
   // ---- cursor: first page of this CTA -> (b, h, page)
-  int b = 0;
-  {
-    int lo_ = 0, hi_ = B - 1;            // last b with sPref[b] <= x_lo
-    while (lo_ < hi_) {
-      int mid = (lo_ + hi_ + 1) >> 1;
-      if (sPref[mid] <= x_lo) lo_ = mid; else hi_ = mid - 1;
-    }
-    b = lo_;
-  }
+  int b = sMisc[11], h = sMisc[12], page = sMisc[13];
   int pages_b = (sPref[b + 1] - sPref[b]) / Hkv;
-  int h = (int)((x_lo - sPref[b]) / pages_b);
-  int page = (int)((x_lo - sPref[b]) % pages_b);
   const uint32_t ring = smem_u32(smem);
   const uint32_t bar0 = smem_u32(bars);
   volatile int* abort_flag = sMisc + 1;
