@@ -437,6 +437,16 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
                 pairs.append((a, b_))
             torch.cuda.synchronize()
             variants[label] = stats_us([a.elapsed_time(b_) for a, b_ in pairs[2:]])
+            # the same launches with one pair of events around the whole batch: a kernel's launch overlaps the one
+            # before it, and the event timer's ~2 us steps average out
+            n_batch = 3 * max(L, 4)
+            a, b_ = ev(), ev()
+            a.record()
+            for r in range(n_batch):
+                kvq.kvq_debug_decode_impl(cfg, caches[r % L], qs[r % L], outs[r % L], ws_buf, impl)
+            b_.record()
+            torch.cuda.synchronize()
+            variants[label]["us_per_launch_in_a_batch"] = a.elapsed_time(b_) * 1000.0 / n_batch
         except kvq.KvqError as e:
             variants[label] = {"unsupported": e.code}
     if kvq.kvq_check_status(caches[0]) != 0:
