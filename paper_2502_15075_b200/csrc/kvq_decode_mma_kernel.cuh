@@ -250,9 +250,10 @@ decode_mma_kernel(Geom g, CachePtrs c, const uint16_t* __restrict__ q, float c1,
   constexpr int NCONS = NW * 32;
   constexpr int NG = NW / 4;                // groups of four consumer warps; a group takes every NG-th page
   constexpr uint32_t FULL = 0xffffffffu;
-  // The time-balanced split (stream gaps, wave weights) pays where the arithmetic per page limits the kernel; pages
-  // of 12 bits per element pair and more are bound by their bytes and keep the plain split by pages.
-  constexpr int GAP = (KAXIS == 0 && KB + VB <= 8) ? kGapPages : 0;
+  // The time-balanced split (stream gaps, wave weights) pays where the arithmetic per page limits the kernel
+  // (token-wise and channel-wise keys alike: 14B-shaped channel-wise K4V2 188 -> 184 us); pages of 10 bits per
+  // element pair and more lose with it (channel-wise K8V2 193 -> 197 us) and keep the plain split by pages.
+  constexpr int GAP = (KB + VB <= 8) ? kGapPages : 0;
   constexpr int WAVES = MINB == 2 ? 2 : 3;          // CTAs per SM = launch waves (the weights apply to a grid of 148 * WAVES)
   static_assert(NW % 4 == 0, "four consumer warps per page, one per 32-token block");
   static_assert(KAXIS == 0 || KB != 2, "channel-wise 2-bit keys are not instantiated");
