@@ -42,7 +42,7 @@ NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of one launch of the dominant kernel from an ncu capture (bytes), keyed by the sha256 of the
 # kernel source it was taken from; reported as null once that source has changed.
-NCU_TRAFFIC = {"552190782df12ee790ba975cedb5d0514abdd9090075bd65bfd3f4ee1a6d9d6f": 441355520}   # dram read 436.43 MB + write 4.93 MB
+NCU_TRAFFIC = {"2efc81c41ceb77b2f51a4ef4559fd4451d9eaad89bd5cdea35b5019c7e07870a": 440967424}   # dram read 436.43 MB + write 4.54 MB
 DECODE_KERNEL_SOURCES = ("kvq_decode_mma.cuh", "kvq_decode_mma_kernel.cuh", "kvq_decode_mma_list.inc")
 
 WORKLOADS = {"tiny": wl.TINY, "1b": wl.LLAMA_1B, "8b": wl.LLAMA_8B, "14b": wl.SHAPED_14B, "70b": wl.LLAMA_70B}
