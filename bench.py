@@ -404,6 +404,23 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
     ms_per_step = total_ms / steps
     dec_us = stats_us([a.elapsed_time(b_) for a, b_ in events])
 
+    # ---- the same step captured once in a CUDA graph and replayed (no per-call events, no host launch gaps)
+    graph_ms = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        step_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(step_graph, stream=side):
+                step_device()
+        torch.cuda.current_stream().wait_stream(side)
+        for _ in range(2):
+            step_graph.replay()
+        graph_ms = timed(step_graph.replay, steps) / steps
+        del step_graph
+    except RuntimeError as e:                      # reported, never fatal: the eager numbers above stand
+        graph_ms = "capture failed: " + str(e).splitlines()[0][:120]
+
     e2e_ms = None
     if do_e2e:
         for _ in range(max(1, warmup // 2)):
@@ -493,6 +510,11 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
         line["e2e"] = {"value": whole_job_gbs(bytes_step, e2e_ms, world), "unit": UNIT, "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": L * (2 * k1s[0].numel() * 2 + qs[0].numel() * 2),
                        "d2h_bytes_per_step": L * outs[0].numel() * 4}
+    if isinstance(graph_ms, float):
+        line["cuda_graph"] = {"ms_per_step": graph_ms, "value": whole_job_gbs(bytes_step, graph_ms, world), "unit": UNIT,
+                              "what": "the same step (all layers) captured once in a CUDA graph and replayed"}
+    elif graph_ms is not None:
+        line["cuda_graph"] = {"unavailable": graph_ms}
     if append_ms:
         a_us = stats_us(append_ms[1:] or append_ms)
         line["append"] = {"tokens_per_call": B * append_tokens, "us_per_call": a_us,
