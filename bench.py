@@ -411,7 +411,8 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
         side.wait_stream(torch.cuda.current_stream())
         step_graph = torch.cuda.CUDAGraph()
         with torch.cuda.stream(side):
-            with torch.cuda.graph(step_graph, stream=side):
+            # thread_local: other threads (a collective library's watchdog) may call the runtime meanwhile
+            with torch.cuda.graph(step_graph, stream=side, capture_error_mode="thread_local"):
                 step_device()
         torch.cuda.current_stream().wait_stream(side)
         for _ in range(2):
