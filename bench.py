@@ -494,8 +494,11 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
     fast_bits = lambda b: b in (2, 4, 8)  # noqa: E731
     deq_launches = ((1 if w.head_dim == 128 and fast_bits(w.vb) else 0) +
                     (1 if w.head_dim == 128 and w.k_axis == 0 and fast_bits(w.kb) else 0))
-    deq_launches = deq_launches if deq_launches == 2 else deq_launches + 1        # the general kernel serves what is left
-    # append (quantize [+ channel-wise K] + bump), decode, dequantize (one kernel per side on its fast path)
+    if deq_launches == 2:
+        deq_launches = 1 if B * w.n_kv_heads <= 148 * 8 else 2     # a short range takes both sides in one launch
+    else:
+        deq_launches += 1                                           # the general kernel serves what is left
+    # append (quantize [+ channel-wise K] + bump), decode, dequantize of the newest page
     kern_per_layer = (2 if w.k_axis == 0 else 3) + 1 + deq_launches
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",

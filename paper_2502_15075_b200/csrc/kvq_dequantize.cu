@@ -411,6 +411,21 @@ int launch_dequantize(const Geom& g, const CachePtrs& c, void* k_out, void* v_ou
   const bool fast_v = vo && g.D == 128 && fast_bits(g.vb);
   const bool fast_k = ko && g.D == 128 && g.k_axis == 0 && !c.k_signs && fast_bits(g.kb);
   int rc = KVQ_OK;
+  // A short range (the newest page of every stream in a decode step) is one launch for both sides; a long one
+  // keeps a launch per side, where the key CTAs run without the value side's shared-memory tile.
+  if (fast_v && fast_k && (long long)np * g.B * g.Hkv <= 148 * 8) {
+#define KVQ_DQ_BOTH(KB_, VB_) \
+    if (g.kb == KB_ && g.vb == VB_) rc = launch_fast<KB_, VB_>(g, c, ko, vo, t_begin, t_end, page0, np, 0, 2, stream);
+    KVQ_DQ_BOTH(2, 2) KVQ_DQ_BOTH(2, 4) KVQ_DQ_BOTH(2, 8)
+    KVQ_DQ_BOTH(4, 2) KVQ_DQ_BOTH(4, 4) KVQ_DQ_BOTH(4, 8)
+    KVQ_DQ_BOTH(8, 2) KVQ_DQ_BOTH(8, 4) KVQ_DQ_BOTH(8, 8)
+#undef KVQ_DQ_BOTH
+    if (rc != KVQ_OK) return rc;
+    if (g.R)
+      window_dequant_kernel<<<g.B * g.Hkv, kThreads, 0, stream>>>(g, c, static_cast<uint16_t*>(k_out),
+                                                                  static_cast<uint16_t*>(v_out), t_begin, t_end);
+    return cudaGetLastError() == cudaSuccess ? KVQ_OK : KVQ_ERR_CUDA_LAUNCH;
+  }
   if (fast_v) {
     if (g.vb == 2) rc = launch_fast<0, 2>(g, c, ko, vo, t_begin, t_end, page0, np, 0, 1, stream);
     else if (g.vb == 4) rc = launch_fast<0, 4>(g, c, ko, vo, t_begin, t_end, page0, np, 0, 1, stream);
