@@ -314,9 +314,10 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
     caches, qs, k1s, v1s = [], [], [], []
     quant_ms, append_ms = [], []
     bulk = T - 1 - append_tokens
+    all_lens = torch.zeros((L, B), dtype=torch.int32, device=dev)     # every layer's sequence lengths, one tensor
     for layer in range(L):
         k, v = wl.make_kv(w, layer=layer + 100 * rank, device=dev, tokens=T)
-        c = kvq.Cache(cfg, device=dev)
+        c = kvq.Cache(cfg, device=dev, seq_len=all_lens[layer])
         e0, e1, e2 = ev(), ev(), ev()
         e0.record()
         kvq.kvq_quantize_append(cfg, c, k[:, :, :bulk], v[:, :, :bulk])
@@ -343,16 +344,17 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
     deq_k = torch.empty((B, w.n_kv_heads, cap, w.head_dim), dtype=w.torch_dtype, device=dev)
     deq_v = torch.empty_like(deq_k)
 
-    def reset_len(c):
+    def reset_lens():
+        # a step appends one token to every layer: put all layers back to T - 1 cached tokens, in one operation
         if lens is None:
-            c.seq_len.fill_(T - 1)
+            all_lens.fill_(T - 1)
         else:
-            c.seq_len.copy_(lens - 1)
+            all_lens.copy_((lens - 1).unsqueeze(0).expand(L, B))
 
     def step_device(events=None):
+        reset_lens()
         for i in range(L):
             c = caches[i]
-            reset_len(c)
             kvq.kvq_quantize_append(cfg, c, k1s[i], v1s[i])
             if events is not None:
                 a, b_ = ev(), ev()
@@ -371,9 +373,9 @@ def run_workload(kvq, w: wl.Workload, dev, rank: int, world: int, steps: int, wa
     dk, dv, dq = torch.empty_like(k1s[0]), torch.empty_like(v1s[0]), torch.empty_like(qs[0])
 
     def step_e2e():
+        reset_lens()
         for i in range(L):
             c = caches[i]
-            reset_len(c)
             kvq.quantize_append_host(cfg, c, hk[i], hv[i], dk, dv)
             kvq.decode_attention_host(cfg, c, hq[i], hout[i], dq, outs[i], ws_buf)
             kvq.kvq_dequantize(cfg, c, deq_k, deq_v, page0, T)

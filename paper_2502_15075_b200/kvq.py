@@ -149,15 +149,24 @@ def kvq_workspace_bytes(cfg: kvq_config) -> int:
 class Cache:
     """Caller-owned buffers of one layer's packed cache (torch tensors) plus the POD handed to the library."""
 
-    def __init__(self, cfg: kvq_config, device="cuda", k_signs: Optional[torch.Tensor] = None):
-        """k_signs: optional int8 tensor [head_dim] of +1 / -1: rotate the keys (randomized Hadamard)."""
+    def __init__(self, cfg: kvq_config, device="cuda", k_signs: Optional[torch.Tensor] = None,
+                 seq_len: Optional[torch.Tensor] = None):
+        """k_signs: optional int8 tensor [head_dim] of +1 / -1: rotate the keys (randomized Hadamard).
+        seq_len: optional caller-owned storage of the sequence lengths, a contiguous int32 CUDA tensor [batch]
+        (e.g. a row of one [layers, batch] tensor, so that all layers' lengths can be set by one operation); it
+        is zeroed here."""
         self.cfg = cfg
         self.k_signs = None if k_signs is None else k_signs.to(device=device, dtype=torch.int8).contiguous()
         assert self.k_signs is None or self.k_signs.numel() == cfg.head_dim
         pages_bytes, tail_bytes = kvq_cache_bytes(cfg)
         self.pages = torch.zeros(pages_bytes, dtype=torch.uint8, device=device)
         self.k_tail = torch.zeros(tail_bytes // 2, dtype=torch.float16, device=device) if tail_bytes else None
-        self.seq_len = torch.zeros(cfg.batch, dtype=torch.int32, device=device)
+        if seq_len is None:
+            self.seq_len = torch.zeros(cfg.batch, dtype=torch.int32, device=device)
+        else:
+            assert seq_len.is_cuda and seq_len.dtype == torch.int32 and seq_len.is_contiguous()
+            assert tuple(seq_len.shape) == (cfg.batch,)
+            self.seq_len = seq_len.zero_()
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         win_bytes = kvq_window_bytes(cfg)
         self.kv_win = torch.zeros(win_bytes // 2, dtype=torch.int16, device=device) if win_bytes else None
