@@ -98,3 +98,27 @@ def test_step_captured_once_replays_while_the_cache_grows(kvq, name, w, T0):
         n = T0 + 1 + i
         assert torch.equal(deq_k[:, :, page0:n].view(torch.int16), ek[:, :, page0:n].view(torch.int16)), name
         assert torch.equal(deq_v[:, :, page0:n].view(torch.int16), ev[:, :, page0:n].view(torch.int16)), name
+
+
+def test_caches_can_share_one_tensor_of_sequence_lengths(kvq):
+    """Caller-owned length storage: two layers' caches keep their lengths in the rows of one tensor, so that one
+    operation sets both; the library reads and bumps them there."""
+    w = wl.LLAMA_8B.with_(n_kv_heads=2, n_q_heads=8)
+    B, T = 2, 300
+    lens = torch.full((2, B), 77, dtype=torch.int32, device="cuda")      # stale contents: the constructor zeroes its row
+    cfg = tl.gpu_config_for(kvq, w, B, 384)
+    caches = [kvq.Cache(cfg, seq_len=lens[i]) for i in range(2)]
+    assert int(lens.abs().sum().item()) == 0
+    k, v = wl.make_kv(w, layer=5, tokens=T, batch=B)
+    oc = tl.oracle_cache_for(w, B, 384)
+    oc.append(tl.bits_of(k), tl.bits_of(v))
+    kvq.kvq_quantize_append(cfg, caches[0], k.cuda(), v.cuda())
+    kvq.kvq_quantize_append(cfg, caches[1], k.cuda()[:, :, :100], v.cuda()[:, :, :100])
+    torch.cuda.synchronize()
+    assert lens.cpu().tolist() == [[T] * B, [100] * B]
+    tl.assert_caches_equal(caches[0], oc)
+    lens[:, :] = torch.tensor([[200] * B, [100] * B], dtype=torch.int32)    # one operation sets both rows: layer 0 rewinds to 200 tokens
+    q = wl.make_q(w, layer=5, batch=B).cuda()
+    got = tl.gpu_decode(kvq, cfg, caches[0], q)
+    want = tl.oracle_on_gpu_codes(caches[0], w).decode(tl.bits_of(q))
+    tl.assert_attention_close(got, want)
